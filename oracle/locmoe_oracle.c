@@ -1,0 +1,380 @@
+/*
+ * LocMoE router oracle -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, single-threaded CPU statement of what the LocMoE router and
+ * token dispatch compute, written from the paper (arXiv 2401.13920) and used
+ * only to check the CUDA path and as the timed CPU baseline.  Every floating
+ * point quantity is accumulated in IEEE double.  Nothing here is blocked,
+ * fused, vectorised or re-ordered beyond what the cited definition states,
+ * and nothing is shared with the CUDA sources.
+ *
+ * Stages (zero-based indices everywhere):
+ *   oracle_gate      Sec. 3.2.1: G = ReLU(w_i . x + eps_i) with the fixed
+ *                    grouped-average-pooling weight (the w_i formula), the
+ *                    arg-max of softmax(G) (Eq. "max_expert") and the score
+ *                    R = softmax(G)[i*] (Eq. "gating_score"); the cosine
+ *                    between the token and the chosen gating weight
+ *                    (Lemma 1 and its proof, Appendix A.1).
+ *   oracle_p_delta   Lemma 3 / Appendix A.2: share of the unit sphere inside
+ *                    the two symmetric caps |cos| >= delta.
+ *   oracle_ec_min    Theorem 1: the three forms of the capacity lower bound.
+ *   oracle_capacity  abstract ("maximal angular deviation between the gating
+ *                    weights and the assigned tokens"), Theorem 1, and the
+ *                    conventional rule ec = ceil(b_s c_f / (ep n)) of
+ *                    Sec. 3.2.3.
+ *   oracle_route     capacity-bounded first-come-first-served placement into
+ *                    an All-to-All shaped buffer (Sec. 3.2.3 capacity limit,
+ *                    Sec. 3.2.4 exchange, abstract: intra-node before
+ *                    inter-node).
+ *   oracle_dispatch  row copy into the buffer.
+ *   oracle_combine   y_m = R_m * expert_out (first equation of Sec. 3.2.1,
+ *                    top-1 so a single term; a dropped token has no term).
+ *
+ * Parity pins: every function below is pinned by tests/test_oracle_*.py
+ * (dense-weight identity, closed forms, library incomplete beta, brute force,
+ * round trip).  The locality loss L_loc is not computed here at all.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_F32 0
+#define ORACLE_BF16 1
+
+#define ORACLE_LAYOUT_SEND 0
+#define ORACLE_LAYOUT_RECV 1
+
+#define ORACLE_BOUND_BETA 0
+#define ORACLE_BOUND_ERFC 1
+#define ORACLE_BOUND_EXP 2
+
+#define ORACLE_WARN_CLAMPED 1
+#define ORACLE_WARN_BAD_SRC 2
+
+#define ORACLE_FLAG_DELTA_OVERRIDE 1
+#define ORACLE_FLAG_MIN_SATURATED 2
+#define ORACLE_FLAG_MIN_BINDS 4
+
+typedef struct {
+    double min_mult;        /* multiplier on Theorem 1's minimum            */
+    double capacity_factor; /* c_f of ec = ceil(b_s c_f / (ep n)); 0 = off  */
+    double delta_override;  /* < 0: measure delta from the data             */
+    int32_t bound_form;     /* ORACLE_BOUND_*                               */
+} oracle_rule_t;
+
+typedef struct {
+    double delta, p_delta, ec_min;
+    int32_t C_expert, C_local, n_empty_experts, flags;
+} oracle_capacity_t;
+
+/* Exact widening of one stored element to double. */
+static double widen(const void *x, int dtype, int64_t i)
+{
+    if (dtype == ORACLE_F32) {
+        return (double)((const float *)x)[i];
+    } else {
+        uint32_t bits = ((uint32_t)((const uint16_t *)x)[i]) << 16;
+        float f;
+        memcpy(&f, &bits, sizeof f);
+        return (double)f;
+    }
+}
+
+/* The GrAP weight written out literally: w[i][j] = (n/d) 1{ i d/n <= j < (i+1) d/n }.
+ * Only used by tests to pin the grouped mean against a dense product. */
+void oracle_grap_weight(int32_t n, int32_t d, double *w /* [n][d] */)
+{
+    for (int32_t i = 0; i < n; ++i)
+        for (int32_t j = 0; j < d; ++j) {
+            /* i d/n <= j < (i+1) d/n, in integers (n divides d) */
+            int inside = ((int64_t)i * d <= (int64_t)j * n) && ((int64_t)j * n < (int64_t)(i + 1) * d);
+            w[(int64_t)i * d + j] = inside ? (double)n / (double)d : 0.0;
+        }
+}
+
+/*
+ * Gate for tokens 0..T-1 of x[T][H].
+ *   mean[i] = w_i . x      = (n/d) * sum of the i-th group of d/n entries
+ *   G[i]    = max(mean[i] + eps[i], 0)
+ *   idx     = lowest i attaining max_i softmax(G)_i  (softmax is monotone, so
+ *             the lowest i attaining max G)
+ *   R       = softmax(G)[idx] = 1 / sum_k exp(G[k] - G[idx])
+ *   cos     = <w_idx, x> / (|w_idx| |x|), |w_i| = sqrt(n/d); 0 when |x| = 0
+ *   gap     = largest G minus second largest G (0 when E == 1 is reported as +inf)
+ * Optional outputs G_out[T][E], probs_out[T][E] may be NULL.
+ * Returns 0, or -2 on a shape error.
+ */
+int oracle_gate(const void *x, int dtype, int64_t T, int32_t H, int32_t E, const float *eps,
+                int32_t *idx, double *R, double *cosv, double *gap,
+                double *G_out, double *probs_out)
+{
+    if (T < 0 || H <= 0 || E <= 0 || H % E != 0) return -2;
+    const int32_t g = H / E;
+    double *G = (double *)malloc(sizeof(double) * (size_t)E);
+    double *mean = (double *)malloc(sizeof(double) * (size_t)E);
+    if (!G || !mean) { free(G); free(mean); return -6; }
+    for (int64_t t = 0; t < T; ++t) {
+        double sq = 0.0;
+        for (int32_t i = 0; i < E; ++i) {
+            double s = 0.0;
+            for (int32_t j = 0; j < g; ++j) {
+                double v = widen(x, dtype, t * H + (int64_t)i * g + j);
+                s += v;
+                sq += v * v;
+            }
+            mean[i] = s * ((double)E / (double)H);
+            double pre = mean[i] + (eps ? (double)eps[i] : 0.0);
+            G[i] = pre > 0.0 ? pre : 0.0;
+        }
+        int32_t best = 0;
+        for (int32_t i = 1; i < E; ++i)
+            if (G[i] > G[best]) best = i;
+        double second = -INFINITY;
+        for (int32_t i = 0; i < E; ++i)
+            if (i != best && G[i] > second) second = G[i];
+        double denom = 0.0;
+        for (int32_t i = 0; i < E; ++i) denom += exp(G[i] - G[best]);
+        idx[t] = best;
+        R[t] = 1.0 / denom;
+        double nrm = sqrt(sq);
+        double wnorm = sqrt((double)E / (double)H);
+        cosv[t] = nrm > 0.0 ? mean[best] / (wnorm * nrm) : 0.0;
+        gap[t] = (E > 1) ? G[best] - second : INFINITY;
+        if (G_out)
+            for (int32_t i = 0; i < E; ++i) G_out[t * E + i] = G[i];
+        if (probs_out)
+            for (int32_t i = 0; i < E; ++i) probs_out[t * E + i] = exp(G[i] - G[best]) / denom;
+    }
+    free(G);
+    free(mean);
+    return 0;
+}
+
+/*
+ * p_delta of Lemma 3 by the cap-area argument of its proof (Appendix A.2):
+ * the area of a cap of half-angle phi on the unit sphere in R^d is
+ * A_{d-1} * integral_0^phi sin^{d-2}(theta) d theta, and p_delta is twice that
+ * cap (phi = acos(delta)) over the whole sphere:
+ *   p_delta = [2 Gamma(d/2) / (sqrt(pi) Gamma((d-1)/2))] * integral_0^{acos delta} sin^{d-2} theta d theta
+ * which equals 1 - I_{delta^2}(1/2, (d-1)/2).  Composite Simpson rule.
+ */
+double oracle_p_delta(double delta, int32_t d)
+{
+    if (d < 2) return NAN;
+    if (delta <= 0.0) return 1.0;
+    if (delta >= 1.0) return 0.0;
+    const double phi = acos(delta);
+    const int64_t panels = 400000; /* even */
+    const double h = phi / (double)panels;
+    const double pw = (double)(d - 2);
+    double acc = 0.0;
+    for (int64_t k = 0; k <= panels; ++k) {
+        double th = h * (double)k;
+        double f = (d == 2) ? 1.0 : pow(sin(th), pw);
+        double wgt = (k == 0 || k == panels) ? 1.0 : ((k & 1) ? 4.0 : 2.0);
+        acc += wgt * f;
+    }
+    double integral = acc * h / 3.0;
+    double lognorm = lgamma(0.5 * (double)d) - lgamma(0.5 * (double)(d - 1));
+    double c = 2.0 / sqrt(M_PI) * exp(lognorm);
+    return c * integral;
+}
+
+/*
+ * Theorem 1: ec_min = 1 / (n p_delta)   (exact form), and the two large-d
+ * forms with a = delta^2 d / (2 - delta^2):  1 / (n erfc(sqrt a)),  exp(a) / n.
+ */
+double oracle_ec_min(double delta, int32_t n, int32_t d, int32_t form)
+{
+    double a = delta * delta * (double)d / (2.0 - delta * delta);
+    if (form == ORACLE_BOUND_ERFC) return 1.0 / ((double)n * erfc(sqrt(a)));
+    if (form == ORACLE_BOUND_EXP) return exp(a) / (double)n;
+    return 1.0 / ((double)n * oracle_p_delta(delta, d));
+}
+
+/*
+ * Angular deviation and capacity.
+ *   delta_e[e] = smallest cosine among the tokens routed to e (largest angle);
+ *                1 for an expert with no token;  theta_e = acos(delta_e)
+ *   delta      = min_e delta_e clamped to [0, 1], unless overridden
+ *   ec_min     = Theorem 1 in the chosen form
+ *   Cmin       = ceil(min(min_mult * ec_min, T))
+ *   C_expert   = clamp(max(Cmin, ceil(c_f T / n), 1), 1, T)
+ *   C_local    = clamp(max(ceil(Cmin / D), ceil(c_f T / (D n)), 1), 1, T)
+ * where D = number of source devices (the "ep" of ec = ceil(b_s c_f/(ep n)),
+ * with b_s = T).
+ */
+int oracle_capacity(const int32_t *idx, const double *cosv, int64_t T, int32_t E, int32_t d,
+                    int32_t D, const oracle_rule_t *rule,
+                    double *delta_e, double *theta_e, oracle_capacity_t *out)
+{
+    if (T <= 0 || E <= 0 || D <= 0 || d < 2) return -2;
+    int32_t n_empty = 0;
+    for (int32_t e = 0; e < E; ++e) delta_e[e] = INFINITY;
+    for (int64_t t = 0; t < T; ++t) {
+        int32_t e = idx[t];
+        if (e < 0 || e >= E) return -2;
+        if (cosv[t] < delta_e[e]) delta_e[e] = cosv[t];
+    }
+    double dmin = INFINITY;
+    for (int32_t e = 0; e < E; ++e) {
+        if (delta_e[e] == INFINITY) { delta_e[e] = 1.0; ++n_empty; }
+        else if (delta_e[e] < dmin) dmin = delta_e[e];
+        double c = delta_e[e] > 1.0 ? 1.0 : (delta_e[e] < -1.0 ? -1.0 : delta_e[e]);
+        theta_e[e] = acos(c);
+    }
+    int32_t flags = 0;
+    double delta = dmin < 0.0 ? 0.0 : (dmin > 1.0 ? 1.0 : dmin);
+    if (rule->delta_override >= 0.0) {
+        delta = rule->delta_override > 1.0 ? 1.0 : rule->delta_override;
+        flags |= ORACLE_FLAG_DELTA_OVERRIDE;
+    }
+    double p = oracle_p_delta(delta, d);
+    double ec = oracle_ec_min(delta, E, d, rule->bound_form);
+    double m = rule->min_mult * ec;
+    if (!(m < (double)T)) { m = (double)T; flags |= ORACLE_FLAG_MIN_SATURATED; }
+    if (m < 0.0) m = 0.0;
+    double Cmin = ceil(m);
+    double cf = rule->capacity_factor;
+    double conv_e = ceil(cf * (double)T / (double)E);
+    double conv_l = ceil(cf * (double)T / ((double)D * (double)E));
+    double ce = Cmin > conv_e ? Cmin : conv_e;
+    double min_l = ceil(Cmin / (double)D);
+    double cl = min_l > conv_l ? min_l : conv_l;
+    if (min_l > conv_l) flags |= ORACLE_FLAG_MIN_BINDS;
+    if (ce < 1.0) ce = 1.0;
+    if (cl < 1.0) cl = 1.0;
+    if (ce > (double)T) ce = (double)T;
+    if (cl > (double)T) cl = (double)T;
+    out->delta = delta;
+    out->p_delta = p;
+    out->ec_min = ec;
+    out->C_expert = (int32_t)ce;
+    out->C_local = (int32_t)cl;
+    out->n_empty_experts = n_empty;
+    out->flags = flags;
+    return 0;
+}
+
+/* Destination rank seen from device a: itself first, then the rest of its own
+ * node, then the other nodes in cyclic order ("intra-node first"). */
+static int32_t dest_rank(int32_t a, int32_t b, int32_t N, int32_t Dn)
+{
+    int32_t dn = ((b / Dn - a / Dn) % N + N) % N;
+    int32_t dl = ((b % Dn - a % Dn) % Dn + Dn) % Dn;
+    return dn * Dn + dl;
+}
+
+void oracle_dest_order(int32_t N, int32_t Dn, int32_t *r /* [D][D] */)
+{
+    int32_t D = N * Dn;
+    for (int32_t a = 0; a < D; ++a)
+        for (int32_t b = 0; b < D; ++b) r[a * D + b] = dest_rank(a, b, N, Dn);
+}
+
+/* pos_t straight from its definition, O(T^2): how many earlier tokens share
+ * both the source device and the chosen expert. */
+void oracle_pos_bruteforce(const int32_t *idx, const int32_t *src, int64_t T, int32_t *pos)
+{
+    for (int64_t t = 0; t < T; ++t) {
+        int32_t c = 0;
+        for (int64_t u = 0; u < t; ++u)
+            if (src[u] == src[t] && idx[u] == idx[t]) ++c;
+        pos[t] = c;
+    }
+}
+
+/*
+ * Route.  E experts placed contiguously on D = N * Dn devices (Ed = E / D per
+ * device).  Token t comes from device src[t] and goes to expert idx[t].
+ *   pos[t]   = number of earlier tokens with the same (src, idx)
+ *   drop[t]  = pos[t] >= C,  C = min(C_local, C_alloc)
+ *   slot[t]  = row in the buffer (row stride C_alloc), -1 when dropped:
+ *     SEND: ((src * D + r(src, dev(e))) * Ed + el) * C_alloc + pos
+ *     RECV: ((dev(e) * Ed + el) * D + r(dev(e), src)) * C_alloc + pos
+ *   inv[row] = t for an occupied row, else -1           [D * E * C_alloc]
+ *   counts[s][e] raw demand, kept[s][e] = min(counts, C), load[e] = sum_s counts
+ *   send_counts[s][b] = kept tokens from s to the experts of device b
+ *   locality[0][c] raw / locality[1][c] kept token counts by class c:
+ *     0 same device, 1 same node, 2 other node
+ * A token whose src is outside [0, D) is dropped (pos = -1) and flagged.
+ */
+int oracle_route(const int32_t *idx, const int32_t *src, int64_t T, int32_t E, int32_t N, int32_t Dn,
+                 int32_t C_local, int32_t C_alloc, int32_t layout,
+                 int32_t *pos, int32_t *slot, uint8_t *drop, int32_t *inv,
+                 int32_t *counts, int32_t *kept, int32_t *send_counts, int32_t *load,
+                 int64_t *locality, int32_t *status)
+{
+    const int32_t D = N * Dn;
+    if (T < 0 || E <= 0 || N <= 0 || Dn <= 0 || E % D != 0 || C_alloc <= 0 || C_local <= 0) return -2;
+    const int32_t Ed = E / D;
+    int32_t C = C_local;
+    int32_t st = 0;
+    if (C > C_alloc) { C = C_alloc; st |= ORACLE_WARN_CLAMPED; }
+    const int64_t rows = (int64_t)D * E * C_alloc;
+    for (int64_t r = 0; r < rows; ++r) inv[r] = -1;
+    memset(counts, 0, sizeof(int32_t) * (size_t)D * E);
+    memset(send_counts, 0, sizeof(int32_t) * (size_t)D * D);
+    memset(load, 0, sizeof(int32_t) * (size_t)E);
+    for (int i = 0; i < 6; ++i) locality[i] = 0;
+    for (int64_t t = 0; t < T; ++t) {
+        int32_t e = idx[t], s = src[t];
+        if (e < 0 || e >= E) return -2;
+        if (s < 0 || s >= D) {
+            st |= ORACLE_WARN_BAD_SRC;
+            pos[t] = -1; slot[t] = -1; drop[t] = 1;
+            continue;
+        }
+        int32_t p = counts[s * E + e]++;
+        load[e]++;
+        int32_t b = e / Ed, el = e % Ed;
+        int cls = (b == s) ? 0 : ((b / Dn == s / Dn) ? 1 : 2);
+        locality[cls]++;
+        pos[t] = p;
+        if (p >= C) { drop[t] = 1; slot[t] = -1; continue; }
+        drop[t] = 0;
+        locality[3 + cls]++;
+        send_counts[s * D + b]++;
+        int64_t row;
+        if (layout == ORACLE_LAYOUT_SEND)
+            row = (((int64_t)s * D + dest_rank(s, b, N, Dn)) * Ed + el) * C_alloc + p;
+        else
+            row = (((int64_t)b * Ed + el) * D + dest_rank(b, s, N, Dn)) * C_alloc + p;
+        slot[t] = (int32_t)row;
+        inv[row] = (int32_t)t;
+    }
+    for (int64_t k = 0; k < (int64_t)D * E; ++k) kept[k] = counts[k] < C ? counts[k] : C;
+    *status = st;
+    return 0;
+}
+
+/* Dispatch: buf[slot[t]] = x[t] bit for bit; every other row zero. */
+int oracle_dispatch(const void *x, int dtype, int64_t T, int32_t H, const int32_t *slot,
+                    int64_t rows, void *buf)
+{
+    const size_t rb = (size_t)H * (dtype == ORACLE_F32 ? 4 : 2);
+    memset(buf, 0, rb * (size_t)rows);
+    for (int64_t t = 0; t < T; ++t) {
+        if (slot[t] < 0) continue;
+        if (slot[t] >= rows) return -2;
+        memcpy((char *)buf + rb * (size_t)slot[t], (const char *)x + rb * (size_t)t, rb);
+    }
+    return 0;
+}
+
+/* Combine: out[t][j] = R[t] * y[slot[t]][j] (double), 0 for a dropped token;
+ * with accumulate != 0 the product is added to prev[t][j] (prev in out dtype
+ * semantics is the caller's business: prev is given in double). */
+int oracle_combine(const void *y, int y_dtype, int64_t T, int32_t H, const int32_t *slot,
+                   const double *R, const double *prev /* [T][H] or NULL */, double *out /* [T][H] */)
+{
+    for (int64_t t = 0; t < T; ++t)
+        for (int32_t j = 0; j < H; ++j) {
+            double v = 0.0;
+            if (slot[t] >= 0) v = R[t] * widen(y, y_dtype, (int64_t)slot[t] * H + j);
+            if (prev) v += prev[t * H + j];
+            out[t * H + j] = v;
+        }
+    return 0;
+}
