@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the LocMoE router hot path on B200: routed tokens/s and achieved HBM GB/s.
+
+One "step" is one pass of the whole path -- gate, capacity, route, dispatch,
+combine -- over one batch of T synthetic tokens.  Default workload: the
+PanGu-Sigma-like layer (T = 65536, H = 5120, E = 64, bf16 tokens, 8 x 8 logical
+devices, capacity factor 1.0).  With N > 1 (torchrun) every rank routes its own
+batch on its own GPU (the path needs no exchange step on one logical-device
+map), so the reported value is the aggregate and scaling is weak.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--cf F] [--impl reference]
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "routed tokens/sec (gate+dispatch+combine) and achieved HBM GB/s vs B200 peak, 1 GPU"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", type=int, default=2, help="workload 1..5 (default 2, the metric's configuration)")
+    ap.add_argument("--cf", type=float, default=1.0, help="capacity factor (both knobs)")
+    ap.add_argument("--layout", choices=["send", "recv"], default="send")
+    ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=8)
+    return ap.parse_args()
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Reads SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop_evt.wait(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def route_passes(D: int, E: int) -> int:
+    """Radix passes the route stage uses for D * E keys (mirrors the library's plan: one pass up to 1024
+    keys, then 8 bits per pass)."""
+    kb = 1
+    while (1 << kb) < D * E:
+        kb += 1
+    return 1 if kb <= 10 else (kb + 7) // 8
+
+
+def oracle_step(oracle, xh, srch, dtype_code, w, cf, layout):
+    """One pass of the whole path in the CPU oracle on host arrays; returns kept tokens."""
+    T = xh.shape[0]
+    g = oracle.gate(xh, dtype_code, w.E)
+    cap = oracle.capacity(g.idx, g.cos, w.E, w.H, w.D, min_mult=cf, capacity_factor=cf)
+    C = cap.C_local
+    r = oracle.route(g.idx, srch, w.E, w.n_nodes, w.dev_per_node, C, C, layout)
+    rows = w.D * w.E * C
+    buf = oracle.dispatch(xh, dtype_code, r.slot, rows)
+    out = oracle.combine(buf, dtype_code, r.slot, g.R)
+    return int((r.slot >= 0).sum()), out.shape
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: same metric, bounded sample per step, host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    from paper_2401_13920_b200 import workloads as W
+    oracle.build()
+    w = W.CONFIGS[args.config]
+    dtc = 0 if w.dtype == "f32" else 1
+    layout = 0 if args.layout == "send" else 1
+    # calibrate on a small sample, then size the per-step sample so that the run ends within ~2 minutes
+    probe = w.scaled(min(w.T, 1024))
+    xh = W.host_bits(W.make_tokens(probe, "cpu"))
+    sh = W.make_src(probe, "cpu").numpy()
+    t0 = time.perf_counter()
+    oracle_step(oracle, xh, sh, dtc, probe, args.cf, layout)
+    per_tok = (time.perf_counter() - t0) / probe.T
+    total_steps = args.steps + args.warmup
+    n = int(max(256, min(w.T, 120.0 / max(total_steps, 1) / per_tok)))
+    n -= n % w.D if n >= w.D else 0
+    sub = w.scaled(n)
+    xh = W.host_bits(W.make_tokens(sub, "cpu"))
+    sh = W.make_src(sub, "cpu").numpy()
+    for _ in range(args.warmup):
+        oracle_step(oracle, xh, sh, dtc, sub, args.cf, layout)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(oracle, xh, sh, dtc, sub, args.cf, layout)
+    dt = time.perf_counter() - t0
+    val = n * args.steps / dt
+    sample = "first %d tokens of the workload per step, whole path, single thread, gcc -O2" % n
+    line = {
+        "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "impl": "reference",
+        "config": workload_config(w, args, n_tokens=n),
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "host_cores": os.cpu_count(),
+    }
+    print(json.dumps(line))
+
+
+def workload_config(w, args, n_tokens=None):
+    return {
+        "workload": "config %d (%s): T=%d H=%d E=%d %s tokens, %dx%d logical devices, c_f=%g, %s layout" % (
+            w.config, w.name, n_tokens or w.T, w.H, w.E, w.dtype, w.n_nodes, w.dev_per_node, args.cf, args.layout),
+        "T": n_tokens or w.T, "H": w.H, "E": w.E, "token_dtype": w.dtype, "n_nodes": w.n_nodes,
+        "dev_per_node": w.dev_per_node, "capacity_factor": args.cf, "layout": args.layout,
+        "l2": "inputs exceed the 126 MB L2, no flush" if (n_tokens or w.T) * w.H * (2 if w.dtype == "bf16" else 4) > 126e6
+        else "inputs fit in L2 (latency-bound configuration)",
+        "stands_in_for": "the paper's private corpus activations (not available); i.i.d. synthetic tokens",
+    }
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    from paper_2401_13920_b200 import binding as B   # raises if the CUDA library cannot be built / loaded
+    from paper_2401_13920_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = W.CONFIGS[args.config]
+    if world > 1:
+        # every rank routes its own batch: same shape, its own seed
+        w = W.Workload(**{**w.__dict__, "config": w.config + 10 * rank, "name": w.name})
+    layout = B.LAYOUT_SEND if args.layout == "send" else B.LAYOUT_RECV
+    x = W.make_tokens(w, dev)
+    src = W.make_src(w, dev)
+    shape = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, layout)
+    rule = B.CapacityRule(args.cf, args.cf, -1.0, B.BOUND_BETA, 0)
+    C_alloc = B.conventional_capacity(w.T, shape.D, w.E, args.cf)
+    st = B.make_router(shape, C_alloc, rule, dev)
+    y = None
+    if w.y_dtype == "f32":
+        y = W.make_expert_out(w, st.rows, dev, "f32")
+    ysrc = st.buf if y is None else y
+
+    stream = torch.cuda.current_stream()
+    stages = ["gate", "capacity", "route", "dispatch", "combine"]
+
+    def step(ev=None):
+        sh, Ca = st.shape, st.C_alloc
+        if ev: ev[0].record(stream)
+        B.locmoe_gate(sh, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
+        if ev: ev[1].record(stream)
+        B.locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
+        if ev: ev[2].record(stream)
+        B.locmoe_route(sh, st.idx, src, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
+                       st.send_counts, st.load, st.locality, st.status, st.ws, stream)
+        if ev: ev[3].record(stream)
+        B.locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream)
+        if ev: ev[4].record(stream)
+        B.locmoe_combine(sh, Ca, ysrc, st.slot, st.gate_w, st.out, False, stream)
+        if ev: ev[5].record(stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    # ---- timed region: exactly K steps, device-timed, per-stage events on the launching stream ----
+    K = args.steps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(K)]
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for k in range(K):
+        step(evs[k])
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t_start.elapsed_time(t_end)
+    if dist is not None:
+        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / K
+    value = world * w.T * K / (total_ms * 1e-3)
+
+    stage_ms = {s: float(np.mean([evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(K)])) for i, s in enumerate(stages)}
+
+    # ---- algorithmic bytes per launch (per token: see the per-kernel byte model in the design notes) ----
+    kept = int((st.slot >= 0).sum().item())
+    bx = x.element_size()
+    by = ysrc.element_size()
+    rows = st.rows
+    bytes_per_launch = {
+        "gate": w.T * w.H * bx + 12 * w.T,
+        "dispatch": kept * w.H * bx + rows * w.H * bx + 4 * rows,
+        "combine": kept * w.H * by + w.T * w.H * bx + 8 * w.T,
+    }
+    peak, peak_kind = measured_peak()
+    kernels = {}
+    for s in ("gate", "dispatch", "combine"):
+        gbs = bytes_per_launch[s] / (stage_ms[s] * 1e-3) / 1e9
+        kernels[s] = {"ms": stage_ms[s], "bytes": bytes_per_launch[s], "achieved_gbs": gbs, "frac": gbs / peak}
+    dominant = max(("gate", "dispatch", "combine"), key=lambda s: stage_ms[s])
+    traffic = ncu_traffic(dominant, w)
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["achieved_gbs"], "peak": peak,
+                "peak_kind": peak_kind + " (copy, MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
+                "unit": "GB/s", "frac": kernels[dominant]["frac"], "traffic": traffic,
+                "path_bytes": sum(bytes_per_launch.values()),
+                "path_frac": sum(bytes_per_launch.values()) / (ms_per_step * 1e-3) / 1e9 / peak,
+                "kernels": kernels, "stage_ms": stage_ms}
+
+    passes = route_passes(shape.D, w.E)
+    launches_per_step = 1 + 2 + (1 + 3 * passes) + 1 + 1
+    cap = B.locmoe_capacity_read(st.cap_dev)
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
+    e2e = None
+    if args.e2e_steps > 0:
+        xh = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
+        xh.copy_(x)
+        srch = torch.empty(src.shape, dtype=src.dtype, pin_memory=True)
+        srch.copy_(src)
+        outh = torch.empty(st.out.shape, dtype=st.out.dtype, pin_memory=True)
+        xd = torch.empty_like(x)
+        srcd = torch.empty_like(src)
+
+        def e2e_step():
+            xd.copy_(xh, non_blocking=True)
+            srcd.copy_(srch, non_blocking=True)
+            B.router_forward(st, xd, srcd, y=y, stream=stream)
+            outh.copy_(st.out, non_blocking=True)
+
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        ems = a.elapsed_time(b)
+        if dist is not None:
+            tt = torch.tensor([ems], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ems = float(tt.item())
+        e2e = {"value": world * w.T * args.e2e_steps / (ems * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": xh.numel() * xh.element_size() + srch.numel() * 4,
+               "d2h_bytes_per_step": outh.numel() * outh.element_size(), "steps": args.e2e_steps,
+               "api": "binding.router_forward on pinned host tensors (copy in, five C-ABI calls, copy out)"}
+
+    # ---- CPU baseline: the oracle, as it stands, on the host cores (rank 0, N = 1 only) ----
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        n = min(w.T, 32768)
+        xs = W.host_bits(x[:n])
+        ss = src[:n].cpu().numpy()
+        sub = w.scaled(n)
+        t0 = time.perf_counter()
+        oracle_step(oracle, xs, ss, shape.x_dtype, sub, args.cf, layout)
+        dt = time.perf_counter() - t0
+        cpu_baseline = {"value": n / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
+                        "sample": "first %d tokens of the workload, whole path once, single thread (host has %d cores)"
+                                  % (n, os.cpu_count())}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "config": workload_config(w, args),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K,
+            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "routing": {"kept_fraction": kept / w.T, "C_local": cap.C_local, "C_expert": cap.C_expert, "delta": cap.delta,
+                        "ec_min": cap.ec_min, "rows": rows, "kept_tokens_per_s": value * kept / w.T},
+            "context": "the paper reports a 12.68%-22.24% per-epoch training-time reduction on 64-256 Ascend 910A NPUs; "
+                       "it gives no number for this path",
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def ncu_traffic(kernel: str, w) -> float | None:
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if one covers this workload."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    try:
+        with open(path) as f:
+            tab = json.load(f)
+        return tab.get("config%d" % w.config, {}).get(kernel)
+    except Exception:
+        return None
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,189 @@
+/*
+ * locmoe.h -- C ABI of the B200 (sm_100a) LocMoE router path.
+ *
+ * One MoE layer's routing, as defined in "LocMoE: A Low-Overhead MoE for Large
+ * Language Model Training" (arXiv 2401.13920), split into five calls:
+ *
+ *   locmoe_gate      Sec. 3.2.1  GrAP gate, ReLU, softmax, top-1 and its score
+ *   locmoe_capacity  abstract + Sec. 3.2.3 (Lemma 3, Theorem 1) capacity rule
+ *   locmoe_route     Sec. 3.2.3 / 3.2.4  capacity-bounded placement of tokens
+ *                    into an All-to-All shaped buffer, intra-node first
+ *   locmoe_dispatch  row gather into that buffer
+ *   locmoe_combine   first equation of Sec. 3.2.1: y_m = R_m * expert output
+ *
+ * Conventions
+ *   - Every array pointer is a DEVICE pointer owned by the caller unless the
+ *     parameter is documented as host memory.  The shape / rule structs
+ *     passed by pointer are HOST memory and are read before the call returns.
+ *   - The library allocates no device memory, keeps no state between calls and
+ *     never synchronises (locmoe_capacity_read excepted).  All work is queued
+ *     on the CUDA stream given as `stream` (a cudaStream_t cast to void*;
+ *     NULL = the default stream).  Scratch memory comes from the caller:
+ *     `ws` with at least locmoe_workspace_bytes() bytes, 256-byte aligned.
+ *   - Return value: 0 = LOCMOE_OK, < 0 = error found on the host before any
+ *     launch (nothing was queued), except LOCMOE_ERR_CUDA which reports a
+ *     failed launch.  Conditions met on the device (capacity clamped, a token
+ *     with an impossible source device) set LOCMOE_WARN_* bits in the
+ *     caller's int32 status word; no kernel traps or asserts.
+ *   - Row-major, densely packed arrays.  T tokens, H hidden size (the paper's
+ *     d), E experts (n), g = H / E group width.  Logical devices
+ *     D = n_nodes * dev_per_node; E % D == 0; expert e lives on device
+ *     e / (E / D) ("expert_num_per_dp_dim x expert_parallel", Appendix D).
+ */
+#ifndef LOCMOE_H
+#define LOCMOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { LOCMOE_F32 = 0, LOCMOE_BF16 = 1 };
+enum { LOCMOE_LAYOUT_SEND = 0, LOCMOE_LAYOUT_RECV = 1 };
+enum { LOCMOE_BOUND_BETA = 0, LOCMOE_BOUND_ERFC = 1, LOCMOE_BOUND_EXP = 2 };
+enum {
+    LOCMOE_OK = 0,
+    LOCMOE_ERR_NULL = -1,      /* a required pointer is NULL                           */
+    LOCMOE_ERR_SHAPE = -2,     /* T < 1, H % E != 0, E % D != 0, rows overflow int32...*/
+    LOCMOE_ERR_DTYPE = -3,     /* unknown dtype / layout / bound form                  */
+    LOCMOE_ERR_ALIGN = -4,     /* a pointer lacks the stated alignment                 */
+    LOCMOE_ERR_WORKSPACE = -5, /* ws too small or misaligned                           */
+    LOCMOE_ERR_CUDA = -6       /* a CUDA call failed (launch error is cleared)         */
+};
+enum {                         /* bits of the device status word                       */
+    LOCMOE_WARN_CLAMPED = 1,   /* C_local > C_alloc: capacity clamped to C_alloc       */
+    LOCMOE_WARN_BAD_SRC = 2,   /* a token's source device is outside [0, D): dropped   */
+    LOCMOE_WARN_BAD_IDX = 4    /* a token's expert index is outside [0, E): dropped    */
+};
+enum {                         /* bits of locmoe_capacity_t.flags                      */
+    LOCMOE_FLAG_DELTA_OVERRIDE = 1, /* delta came from the rule, not the data          */
+    LOCMOE_FLAG_MIN_SATURATED = 2,  /* min_mult * ec_min >= T (or overflowed): T used  */
+    LOCMOE_FLAG_MIN_BINDS = 4       /* Theorem 1's minimum set C_local                 */
+};
+
+/* Problem shape (host struct). */
+typedef struct {
+    int32_t T;            /* tokens in the batch, >= 1                                 */
+    int32_t H;            /* hidden size d, a multiple of E                            */
+    int32_t E;            /* experts n                                                 */
+    int32_t n_nodes;      /* logical nodes N                                           */
+    int32_t dev_per_node; /* logical devices per node Dn; D = N * Dn divides E         */
+    int32_t x_dtype;      /* LOCMOE_F32 | LOCMOE_BF16: tokens, buffer and combined out */
+    int32_t layout;       /* LOCMOE_LAYOUT_SEND | LOCMOE_LAYOUT_RECV                   */
+} locmoe_shape_t;
+
+/* Capacity rule (host struct).  Capacity = max(Theorem 1's minimum * min_mult,
+ * conventional ec = ceil(T * capacity_factor / (D * n))), see locmoe_capacity. */
+typedef struct {
+    double min_mult;        /* multiplier on ec_min of Theorem 1                       */
+    double capacity_factor; /* c_f of Sec. 3.2.3; 0 = use the minimum alone            */
+    double delta_override;  /* < 0: measure delta from the batch; else use this value  */
+    int32_t bound_form;     /* LOCMOE_BOUND_*: which form of Theorem 1                 */
+    int32_t reserved;       /* must be 0                                               */
+} locmoe_capacity_rule_t;
+
+/* Capacity record (written on the device by locmoe_capacity). */
+typedef struct {
+    double delta;            /* cosine threshold: min over experts of delta_e, >= 0    */
+    double p_delta;          /* Lemma 3: 1 - I_{delta^2}(1/2, (d-1)/2)                 */
+    double ec_min;           /* Theorem 1 in the chosen form                           */
+    int32_t C_expert;        /* slots per expert over all sources                      */
+    int32_t C_local;         /* slots per (source device, expert) pair                 */
+    int32_t n_empty_experts; /* experts that received no token                         */
+    int32_t flags;           /* LOCMOE_FLAG_*                                          */
+} locmoe_capacity_t;
+
+/* Scratch size for locmoe_capacity and locmoe_route on this shape (they may
+ * share one workspace; calls on one stream run in order).  `bytes` is host
+ * memory.  C_alloc is the row stride the caller will pass to locmoe_route. */
+int locmoe_workspace_bytes(const locmoe_shape_t *shape, int32_t C_alloc, size_t *bytes);
+
+/*
+ * GrAP gate (Sec. 3.2.1).  For each token t, with the fixed weight
+ * w_i = (n/d) 1{i d/n <= j < (i+1) d/n}:
+ *   mean_i = w_i . x_t (average of the i-th group of g entries, fp32 accumulation)
+ *   G_i    = ReLU(mean_i + eps_i)                    (eps == NULL means 0)
+ *   idx[t] = lowest i attaining max_i softmax(G)_i   (Eq. "max_expert")
+ *   gate_w[t] = softmax(G)[idx[t]]                   (Eq. "gating_score")
+ *   cos_sim[t] = <w_idx, x_t> / (|w_idx| |x_t|)      (Lemma 1; 0 for a zero token)
+ *   probs[t][i] = softmax(G)_i                       (optional, NULL to skip)
+ * x: [T][H] of shape->x_dtype.  The fast path needs x 16-byte aligned and
+ * H * sizeof(element) a multiple of 16; other inputs take a slower scalar path.
+ * idx int32[T], gate_w / cos_sim float[T], probs float[T][E], eps float[E].
+ */
+int locmoe_gate(const locmoe_shape_t *shape, const void *x, const float *eps,
+                int32_t *idx, float *gate_w, float *cos_sim, float *probs, void *stream);
+
+/*
+ * Angular deviation and capacity (abstract; Lemma 3; Theorem 1; Sec. 3.2.3).
+ *   delta_e[e] = smallest cos_sim among tokens with idx == e (1 if none),
+ *   theta_e[e] = acos(delta_e[e])  -- the largest angle between expert e's
+ *                gating weight and a token assigned to it,
+ *   delta      = clamp(min_e delta_e, 0, 1) or rule->delta_override,
+ *   p_delta, ec_min = 1 / (n p_delta) (or the erfc / exp form),
+ *   Cmin       = ceil(min(min_mult * ec_min, T)),
+ *   C_expert   = clamp(max(Cmin, ceil(c_f T / n), 1), 1, T),
+ *   C_local    = clamp(max(ceil(Cmin / D), ceil(c_f T / (D n)), 1), 1, T).
+ * delta_e / theta_e: float[E]; cap_dev: device record; ws: see above.
+ */
+int locmoe_capacity(const locmoe_shape_t *shape, const int32_t *idx, const float *cos_sim,
+                    const locmoe_capacity_rule_t *rule, float *delta_e, float *theta_e,
+                    locmoe_capacity_t *cap_dev, void *ws, size_t ws_bytes, void *stream);
+
+/* Copies the device record to host memory and waits for the stream. */
+int locmoe_capacity_read(const locmoe_capacity_t *cap_dev, locmoe_capacity_t *cap_host, void *stream);
+
+/*
+ * Capacity-bounded routing (Sec. 3.2.3 capacity limit; Sec. 3.2.4 exchange).
+ * Token t comes from logical device src_dev[t] and goes to expert idx[t].
+ * C = min(cap_dev->C_local, C_alloc).
+ *   pos[t]  = number of earlier tokens (lower t) with the same (src, expert)
+ *   drop[t] = pos[t] >= C; a dropped token gets slot[t] = -1
+ *   slot[t] = row of the token in the buffer of D * E * C_alloc rows:
+ *     SEND layout  ((src * D + r(src, dev(e))) * Ed + e % Ed) * C_alloc + pos
+ *     RECV layout  ((e * D) + r(dev(e), src)) * C_alloc + pos
+ *     with r(a, b) = ((node(b) - node(a)) mod N) * Dn + ((loc(b) - loc(a)) mod Dn):
+ *     a device lists itself first, then its own node, then the other nodes.
+ *   inv[row] = t for an occupied row, -1 otherwise          int32[D * E * C_alloc]
+ *   counts[s][e] tokens demanded, kept[s][e] = min(counts, C)      int32[D][E]
+ *   send_counts[s][b] = kept tokens from s to the experts of device b  int32[D][D]
+ *   load[e] = sum_s counts[s][e]                                   int32[E]
+ *   locality[0][c] / locality[1][c]: tokens demanded / kept by class c
+ *     (0 same device, 1 same node, 2 other node)                   int64[2][3]
+ *   status: int32 word, LOCMOE_WARN_* bits are OR-ed in (it is zeroed first).
+ * The result is deterministic: it depends only on the inputs.
+ */
+int locmoe_route(const locmoe_shape_t *shape, const int32_t *idx, const int32_t *src_dev,
+                 const locmoe_capacity_t *cap_dev, int32_t C_alloc,
+                 int32_t *pos, int32_t *slot, uint8_t *drop, int32_t *inv,
+                 int32_t *counts, int32_t *kept, int32_t *send_counts, int32_t *load,
+                 int64_t *locality, int32_t *status, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Dispatch: buf[row][:] = x[inv[row]][:] bit for bit for occupied rows; rows
+ * with inv < 0 are zero-filled when zero_pad != 0 and left untouched otherwise.
+ * x [T][H], buf [D * E * C_alloc][H], both of shape->x_dtype.
+ */
+int locmoe_dispatch(const locmoe_shape_t *shape, int32_t C_alloc, const void *x,
+                    const int32_t *inv, void *buf, int32_t zero_pad, void *stream);
+
+/*
+ * Combine: out[t][:] = gate_w[t] * y[slot[t]][:] for a kept token and 0 for a
+ * dropped one; with accumulate != 0 the product is added to out (a dropped
+ * token then leaves out unchanged).  y [D * E * C_alloc][H] of y_dtype,
+ * out [T][H] of shape->x_dtype; the product (and the sum) is formed in fp32
+ * and then rounded to the output type, to nearest-even.
+ */
+int locmoe_combine(const locmoe_shape_t *shape, int32_t C_alloc, const void *y, int32_t y_dtype,
+                   const int32_t *slot, const float *gate_w, void *out, int32_t accumulate,
+                   void *stream);
+
+/* Text for a return code of this library (host string, never NULL). */
+const char *locmoe_status_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOCMOE_H */

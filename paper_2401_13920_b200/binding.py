@@ -1,0 +1,282 @@
+"""Python face of the C-ABI library declared in ``include/locmoe.h``.
+
+Argument marshalling only: every function hands device pointers of torch
+tensors to the entry point of the same name in ``liblocmoe.so``; all of the
+router's arithmetic runs in the CUDA kernels.  There is no CPU fallback -- if
+the library is missing it is built with nvcc, and if that fails the import of
+this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+F32, BF16 = 0, 1
+LAYOUT_SEND, LAYOUT_RECV = 0, 1
+BOUND_BETA, BOUND_ERFC, BOUND_EXP = 0, 1, 2
+WARN_CLAMPED, WARN_BAD_SRC, WARN_BAD_IDX = 1, 2, 4
+FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
+
+EXPORTS = [
+    "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_read", "locmoe_route",
+    "locmoe_dispatch", "locmoe_combine", "locmoe_status_string",
+]
+
+
+class Shape(C.Structure):
+    _fields_ = [("T", C.c_int32), ("H", C.c_int32), ("E", C.c_int32), ("n_nodes", C.c_int32),
+                ("dev_per_node", C.c_int32), ("x_dtype", C.c_int32), ("layout", C.c_int32)]
+
+    @property
+    def D(self) -> int:
+        return self.n_nodes * self.dev_per_node
+
+
+class CapacityRule(C.Structure):
+    _fields_ = [("min_mult", C.c_double), ("capacity_factor", C.c_double), ("delta_override", C.c_double),
+                ("bound_form", C.c_int32), ("reserved", C.c_int32)]
+
+
+class Capacity(C.Structure):
+    _fields_ = [("delta", C.c_double), ("p_delta", C.c_double), ("ec_min", C.c_double),
+                ("C_expert", C.c_int32), ("C_local", C.c_int32), ("n_empty_experts", C.c_int32),
+                ("flags", C.c_int32)]
+
+
+CAPACITY_BYTES = C.sizeof(Capacity)
+
+
+class LocMoEError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        self.code = code
+        super().__init__("%s failed: %d (%s)" % (fn, code, status_string(code)))
+
+
+def _load() -> C.CDLL:
+    path = _build.build()  # raises when nvcc or the sources are missing
+    lib = C.CDLL(path)
+    vp, i32 = C.c_void_p, C.c_int32
+    lib.locmoe_workspace_bytes.argtypes = [C.POINTER(Shape), i32, C.POINTER(C.c_size_t)]
+    lib.locmoe_gate.argtypes = [C.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp]
+    lib.locmoe_capacity.argtypes = [C.POINTER(Shape), vp, vp, C.POINTER(CapacityRule), vp, vp, vp, vp, C.c_size_t, vp]
+    lib.locmoe_capacity_read.argtypes = [vp, C.POINTER(Capacity), vp]
+    lib.locmoe_route.argtypes = [C.POINTER(Shape), vp, vp, vp, i32] + [vp] * 10 + [vp, C.c_size_t, vp]
+    lib.locmoe_dispatch.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, i32, vp]
+    lib.locmoe_combine.argtypes = [C.POINTER(Shape), i32, vp, i32, vp, vp, vp, i32, vp]
+    lib.locmoe_status_string.argtypes = [C.c_int]
+    lib.locmoe_status_string.restype = C.c_char_p
+    for name in EXPORTS[:-1]:
+        getattr(lib, name).restype = C.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def status_string(code: int) -> str:
+    return _lib.locmoe_status_string(int(code)).decode()
+
+
+def dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.float32:
+        return F32
+    if dt == torch.bfloat16:
+        return BF16
+    raise TypeError("tokens must be float32 or bfloat16, got %s" % dt)
+
+
+def make_shape(T, H, E, n_nodes, dev_per_node, x_dtype, layout=LAYOUT_SEND) -> Shape:
+    if isinstance(x_dtype, torch.dtype):
+        x_dtype = dtype_code(x_dtype)
+    return Shape(int(T), int(H), int(E), int(n_nodes), int(dev_per_node), int(x_dtype), int(layout))
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _check(fn: str, rc: int) -> int:
+    if rc < 0:
+        raise LocMoEError(fn, rc)
+    return rc
+
+
+def _want(t, dtype, numel, name):
+    if t.dtype != dtype or t.numel() < numel:
+        raise ValueError("%s: expected %s with at least %d elements, got %s with %d"
+                         % (name, dtype, numel, t.dtype, t.numel()))
+
+
+def locmoe_workspace_bytes(shape: Shape, C_alloc: int) -> int:
+    out = C.c_size_t(0)
+    _check("locmoe_workspace_bytes", _lib.locmoe_workspace_bytes(C.byref(shape), int(C_alloc), C.byref(out)))
+    return out.value
+
+
+def locmoe_gate(shape: Shape, x, eps, idx, gate_w, cos_sim, probs=None, stream=None) -> int:
+    _want(x, torch.float32 if shape.x_dtype == F32 else torch.bfloat16, shape.T * shape.H, "x")
+    _want(idx, torch.int32, shape.T, "idx")
+    _want(gate_w, torch.float32, shape.T, "gate_w")
+    _want(cos_sim, torch.float32, shape.T, "cos_sim")
+    if eps is not None:
+        _want(eps, torch.float32, shape.E, "eps")
+    if probs is not None:
+        _want(probs, torch.float32, shape.T * shape.E, "probs")
+    return _check("locmoe_gate", _lib.locmoe_gate(C.byref(shape), _ptr(x), _ptr(eps), _ptr(idx), _ptr(gate_w),
+                                                  _ptr(cos_sim), _ptr(probs), _stream(stream)))
+
+
+def locmoe_capacity(shape: Shape, idx, cos_sim, rule: CapacityRule, delta_e, theta_e, cap_dev, ws, stream=None) -> int:
+    _want(idx, torch.int32, shape.T, "idx")
+    _want(cos_sim, torch.float32, shape.T, "cos_sim")
+    _want(delta_e, torch.float32, shape.E, "delta_e")
+    _want(theta_e, torch.float32, shape.E, "theta_e")
+    _want(cap_dev, torch.uint8, CAPACITY_BYTES, "cap_dev")
+    return _check("locmoe_capacity", _lib.locmoe_capacity(
+        C.byref(shape), _ptr(idx), _ptr(cos_sim), C.byref(rule), _ptr(delta_e), _ptr(theta_e), _ptr(cap_dev),
+        _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def locmoe_capacity_read(cap_dev, stream=None) -> Capacity:
+    out = Capacity()
+    _check("locmoe_capacity_read", _lib.locmoe_capacity_read(_ptr(cap_dev), C.byref(out), _stream(stream)))
+    return out
+
+
+def locmoe_route(shape: Shape, idx, src_dev, cap_dev, C_alloc, pos, slot, drop, inv, counts, kept, send_counts,
+                 load, locality, status, ws, stream=None) -> int:
+    D, E, T = shape.D, shape.E, shape.T
+    _want(idx, torch.int32, T, "idx")
+    _want(src_dev, torch.int32, T, "src_dev")
+    _want(cap_dev, torch.uint8, CAPACITY_BYTES, "cap_dev")
+    _want(pos, torch.int32, T, "pos")
+    _want(slot, torch.int32, T, "slot")
+    _want(drop, torch.uint8, T, "drop")
+    _want(inv, torch.int32, D * E * C_alloc, "inv")
+    _want(counts, torch.int32, D * E, "counts")
+    _want(kept, torch.int32, D * E, "kept")
+    _want(send_counts, torch.int32, D * D, "send_counts")
+    _want(load, torch.int32, E, "load")
+    _want(locality, torch.int64, 6, "locality")
+    _want(status, torch.int32, 1, "status")
+    return _check("locmoe_route", _lib.locmoe_route(
+        C.byref(shape), _ptr(idx), _ptr(src_dev), _ptr(cap_dev), int(C_alloc), _ptr(pos), _ptr(slot), _ptr(drop),
+        _ptr(inv), _ptr(counts), _ptr(kept), _ptr(send_counts), _ptr(load), _ptr(locality), _ptr(status),
+        _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def locmoe_dispatch(shape: Shape, C_alloc, x, inv, buf, zero_pad=True, stream=None) -> int:
+    rows = shape.D * shape.E * C_alloc
+    dt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
+    _want(x, dt, shape.T * shape.H, "x")
+    _want(inv, torch.int32, rows, "inv")
+    _want(buf, dt, rows * shape.H, "buf")
+    return _check("locmoe_dispatch", _lib.locmoe_dispatch(C.byref(shape), int(C_alloc), _ptr(x), _ptr(inv), _ptr(buf),
+                                                          1 if zero_pad else 0, _stream(stream)))
+
+
+def locmoe_combine(shape: Shape, C_alloc, y, slot, gate_w, out, accumulate=False, stream=None) -> int:
+    rows = shape.D * shape.E * C_alloc
+    _want(y, y.dtype, rows * shape.H, "y")
+    _want(slot, torch.int32, shape.T, "slot")
+    _want(gate_w, torch.float32, shape.T, "gate_w")
+    _want(out, torch.float32 if shape.x_dtype == F32 else torch.bfloat16, shape.T * shape.H, "out")
+    return _check("locmoe_combine", _lib.locmoe_combine(C.byref(shape), int(C_alloc), _ptr(y), dtype_code(y.dtype),
+                                                        _ptr(slot), _ptr(gate_w), _ptr(out), 1 if accumulate else 0,
+                                                        _stream(stream)))
+
+
+def conventional_capacity(T: int, D: int, E: int, capacity_factor: float) -> int:
+    """Host-side row stride to allocate: ceil(c_f T / (D n)), at least 1 (Sec. 3.2.3)."""
+    return max(1, math.ceil(capacity_factor * T / (D * E)))
+
+
+@dataclass
+class RouterState:
+    """Device buffers of one router instance (allocated once, reused every step)."""
+    shape: Shape
+    C_alloc: int
+    rule: CapacityRule
+    idx: torch.Tensor
+    gate_w: torch.Tensor
+    cos_sim: torch.Tensor
+    delta_e: torch.Tensor
+    theta_e: torch.Tensor
+    cap_dev: torch.Tensor
+    pos: torch.Tensor
+    slot: torch.Tensor
+    drop: torch.Tensor
+    inv: torch.Tensor
+    counts: torch.Tensor
+    kept: torch.Tensor
+    send_counts: torch.Tensor
+    load: torch.Tensor
+    locality: torch.Tensor
+    status: torch.Tensor
+    ws: torch.Tensor
+    buf: torch.Tensor
+    out: torch.Tensor
+
+    @property
+    def rows(self) -> int:
+        return self.shape.D * self.shape.E * self.C_alloc
+
+
+def make_router(shape: Shape, C_alloc: int, rule: CapacityRule, device="cuda") -> RouterState:
+    """Allocates every output and scratch tensor of the five calls with torch (memory plumbing only)."""
+    dev = torch.device(device)
+    T, H, E, D = shape.T, shape.H, shape.E, shape.D
+    rows = D * E * C_alloc
+    xdt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
+    i32 = dict(dtype=torch.int32, device=dev)
+    f32 = dict(dtype=torch.float32, device=dev)
+    ws_bytes = locmoe_workspace_bytes(shape, C_alloc)
+    return RouterState(
+        shape=shape, C_alloc=C_alloc, rule=rule,
+        idx=torch.empty(T, **i32), gate_w=torch.empty(T, **f32), cos_sim=torch.empty(T, **f32),
+        delta_e=torch.empty(E, **f32), theta_e=torch.empty(E, **f32),
+        cap_dev=torch.zeros(CAPACITY_BYTES, dtype=torch.uint8, device=dev),
+        pos=torch.empty(T, **i32), slot=torch.empty(T, **i32), drop=torch.empty(T, dtype=torch.uint8, device=dev),
+        inv=torch.empty(rows, **i32), counts=torch.empty(D * E, **i32), kept=torch.empty(D * E, **i32),
+        send_counts=torch.empty(D * D, **i32), load=torch.empty(E, **i32),
+        locality=torch.empty(6, dtype=torch.int64, device=dev), status=torch.zeros(1, **i32),
+        ws=torch.empty(ws_bytes, dtype=torch.uint8, device=dev),
+        buf=torch.empty(rows, H, dtype=xdt, device=dev), out=torch.empty(T, H, dtype=xdt, device=dev),
+    )
+
+
+def router_forward(st: RouterState, x, src_dev, y=None, eps=None, stream=None):
+    """gate -> capacity -> route -> dispatch -> combine on one stream.
+
+    ``y`` are the expert outputs in slot layout; with ``y=None`` the experts are
+    the identity and the dispatched buffer itself is combined.  Returns ``st.out``.
+    """
+    sh, Ca = st.shape, st.C_alloc
+    locmoe_gate(sh, x, eps, st.idx, st.gate_w, st.cos_sim, None, stream)
+    locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
+    locmoe_route(sh, st.idx, src_dev, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
+                 st.send_counts, st.load, st.locality, st.status, st.ws, stream)
+    locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream)
+    locmoe_combine(sh, Ca, st.buf if y is None else y, st.slot, st.gate_w, st.out, False, stream)
+    return st.out

@@ -1,0 +1,154 @@
+// C-ABI front end: argument validation on the host, then the kernel launchers.
+#include "common.cuh"
+
+namespace locmoe {
+
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return kNumSMsB200; }
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+            cudaGetLastError();
+            n = kNumSMsB200;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+namespace {
+
+int check_shape(const locmoe_shape_t* s) {
+    if (!s) return LOCMOE_ERR_NULL;
+    if (s->T < 1 || s->H < 1 || s->E < 1 || s->n_nodes < 1 || s->dev_per_node < 1) return LOCMOE_ERR_SHAPE;
+    if (s->H % s->E != 0) return LOCMOE_ERR_SHAPE;
+    const long long D = (long long)s->n_nodes * s->dev_per_node;
+    if (D > s->E || s->E % D != 0) return LOCMOE_ERR_SHAPE;
+    if (D * s->E > 0x7fffffffll) return LOCMOE_ERR_SHAPE;
+    if (s->x_dtype != LOCMOE_F32 && s->x_dtype != LOCMOE_BF16) return LOCMOE_ERR_DTYPE;
+    if (s->layout != LOCMOE_LAYOUT_SEND && s->layout != LOCMOE_LAYOUT_RECV) return LOCMOE_ERR_DTYPE;
+    return LOCMOE_OK;
+}
+
+// Rows of the buffer for row stride C_alloc, or -1 if they do not fit an int32 row index.
+long long buffer_rows(const locmoe_shape_t* s, int32_t C_alloc) {
+    if (C_alloc < 1) return -1;
+    const long long K = (long long)s->n_nodes * s->dev_per_node * s->E;
+    const long long rows = K * C_alloc;
+    return rows > 0x7fffffffll ? -1 : rows;
+}
+
+}  // namespace
+}  // namespace locmoe
+
+using namespace locmoe;
+
+extern "C" {
+
+int locmoe_workspace_bytes(const locmoe_shape_t* shape, int32_t C_alloc, size_t* bytes) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!bytes) return LOCMOE_ERR_NULL;
+    if (buffer_rows(shape, C_alloc) < 0) return LOCMOE_ERR_SHAPE;
+    RoutePlan p;
+    if ((rc = plan_route(*shape, &p))) return rc;
+    size_t c = capacity_ws_bytes(*shape);
+    *bytes = p.total > c ? p.total : c;
+    return LOCMOE_OK;
+}
+
+int locmoe_gate(const locmoe_shape_t* shape, const void* x, const float* eps, int32_t* idx, float* gate_w,
+                float* cos_sim, float* probs, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!x || !idx || !gate_w || !cos_sim) return LOCMOE_ERR_NULL;
+    const int esz = shape->x_dtype == LOCMOE_F32 ? 4 : 2;
+    if ((uintptr_t)x % esz) return LOCMOE_ERR_ALIGN;
+    return launch_gate(*shape, x, eps, idx, gate_w, cos_sim, probs, static_cast<cudaStream_t>(stream));
+}
+
+int locmoe_capacity(const locmoe_shape_t* shape, const int32_t* idx, const float* cos_sim,
+                    const locmoe_capacity_rule_t* rule, float* delta_e, float* theta_e, locmoe_capacity_t* cap_dev,
+                    void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!idx || !cos_sim || !rule || !delta_e || !theta_e || !cap_dev) return LOCMOE_ERR_NULL;
+    if (shape->H < 2) return LOCMOE_ERR_SHAPE;
+    if (rule->bound_form < LOCMOE_BOUND_BETA || rule->bound_form > LOCMOE_BOUND_EXP) return LOCMOE_ERR_DTYPE;
+    if (!(rule->min_mult >= 0.0) || !(rule->capacity_factor >= 0.0) || rule->delta_override != rule->delta_override)
+        return LOCMOE_ERR_SHAPE;
+    if (!ws || ws_bytes < capacity_ws_bytes(*shape) || (uintptr_t)ws % 256) return LOCMOE_ERR_WORKSPACE;
+    if ((uintptr_t)cap_dev % 8) return LOCMOE_ERR_ALIGN;
+    return launch_capacity(*shape, idx, cos_sim, *rule, delta_e, theta_e, cap_dev, ws, static_cast<cudaStream_t>(stream));
+}
+
+int locmoe_capacity_read(const locmoe_capacity_t* cap_dev, locmoe_capacity_t* cap_host, void* stream) {
+    if (!cap_dev || !cap_host) return LOCMOE_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(cap_host, cap_dev, sizeof(locmoe_capacity_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return LOCMOE_ERR_CUDA;
+    }
+    return LOCMOE_OK;
+}
+
+int locmoe_route(const locmoe_shape_t* shape, const int32_t* idx, const int32_t* src_dev,
+                 const locmoe_capacity_t* cap_dev, int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop,
+                 int32_t* inv, int32_t* counts, int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality,
+                 int32_t* status, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!idx || !src_dev || !cap_dev || !pos || !slot || !drop || !inv || !counts || !kept || !send_counts || !load ||
+        !locality || !status)
+        return LOCMOE_ERR_NULL;
+    if (buffer_rows(shape, C_alloc) < 0) return LOCMOE_ERR_SHAPE;
+    RoutePlan p;
+    if ((rc = plan_route(*shape, &p))) return rc;
+    if (!ws || ws_bytes < p.total || (uintptr_t)ws % 256) return LOCMOE_ERR_WORKSPACE;
+    if ((uintptr_t)locality % 8 || (uintptr_t)cap_dev % 8) return LOCMOE_ERR_ALIGN;
+    return launch_route(*shape, idx, src_dev, cap_dev, C_alloc, pos, slot, drop, inv, counts, kept, send_counts, load,
+                        locality, status, ws, static_cast<cudaStream_t>(stream));
+}
+
+int locmoe_dispatch(const locmoe_shape_t* shape, int32_t C_alloc, const void* x, const int32_t* inv, void* buf,
+                    int32_t zero_pad, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!x || !inv || !buf) return LOCMOE_ERR_NULL;
+    const long long rows = buffer_rows(shape, C_alloc);
+    if (rows < 0) return LOCMOE_ERR_SHAPE;
+    const int esz = shape->x_dtype == LOCMOE_F32 ? 4 : 2;
+    if ((uintptr_t)x % esz || (uintptr_t)buf % esz) return LOCMOE_ERR_ALIGN;
+    return launch_dispatch(*shape, rows, x, inv, buf, zero_pad, static_cast<cudaStream_t>(stream));
+}
+
+int locmoe_combine(const locmoe_shape_t* shape, int32_t C_alloc, const void* y, int32_t y_dtype, const int32_t* slot,
+                   const float* gate_w, void* out, int32_t accumulate, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!y || !slot || !gate_w || !out) return LOCMOE_ERR_NULL;
+    if (y_dtype != LOCMOE_F32 && y_dtype != LOCMOE_BF16) return LOCMOE_ERR_DTYPE;
+    const long long rows = buffer_rows(shape, C_alloc);
+    if (rows < 0) return LOCMOE_ERR_SHAPE;
+    if ((uintptr_t)y % (y_dtype == LOCMOE_F32 ? 4 : 2) || (uintptr_t)out % (shape->x_dtype == LOCMOE_F32 ? 4 : 2))
+        return LOCMOE_ERR_ALIGN;
+    return launch_combine(*shape, rows, y, y_dtype, slot, gate_w, out, accumulate, static_cast<cudaStream_t>(stream));
+}
+
+const char* locmoe_status_string(int code) {
+    switch (code) {
+        case LOCMOE_OK: return "ok";
+        case LOCMOE_ERR_NULL: return "a required pointer is NULL";
+        case LOCMOE_ERR_SHAPE: return "invalid shape or size";
+        case LOCMOE_ERR_DTYPE: return "unknown dtype, layout or bound form";
+        case LOCMOE_ERR_ALIGN: return "pointer alignment";
+        case LOCMOE_ERR_WORKSPACE: return "workspace missing, too small or misaligned";
+        case LOCMOE_ERR_CUDA: return "a CUDA call failed";
+        default: return code > 0 ? "warning bits set" : "unknown error";
+    }
+}
+
+}  // extern "C"

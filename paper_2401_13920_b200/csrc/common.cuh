@@ -1,0 +1,77 @@
+// Internal declarations shared by the LocMoE kernels and the C-ABI front end.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "locmoe.h"
+
+namespace locmoe {
+
+constexpr int kWarp = 32;
+constexpr int kNumSMsB200 = 148;
+
+// Number of SMs of the current device (cached per process; B200 has 148).
+int sm_count();
+
+inline int check_launch() {
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? LOCMOE_OK : LOCMOE_ERR_CUDA;
+}
+
+// ---- launchers (each queues its kernels on `st` and returns a LOCMOE_* code) ----
+int launch_gate(const locmoe_shape_t& s, const void* x, const float* eps, int32_t* idx, float* gate_w,
+                float* cos_sim, float* probs, cudaStream_t st);
+
+int launch_capacity(const locmoe_shape_t& s, const int32_t* idx, const float* cos_sim,
+                    const locmoe_capacity_rule_t& rule, float* delta_e, float* theta_e,
+                    locmoe_capacity_t* cap_dev, void* ws, cudaStream_t st);
+
+struct RoutePlan {
+    int key_bits;     // bits needed for keys 0..K (K = D*E is the "bad token" key)
+    int passes;       // radix passes
+    int bits[4];      // bits per pass, least significant first
+    int tile;         // tokens per tile
+    int rounds;       // 32-token rounds per warp per tile
+    int ntiles;
+    size_t off_keys[2], off_toks[2], off_hist, off_keystart, total;
+};
+int plan_route(const locmoe_shape_t& s, RoutePlan* p);
+size_t capacity_ws_bytes(const locmoe_shape_t& s);
+
+int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src, const locmoe_capacity_t* cap_dev,
+                 int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
+                 int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
+                 void* ws, cudaStream_t st);
+
+int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const int32_t* inv, void* buf,
+                    int zero_pad, cudaStream_t st);
+
+int launch_combine(const locmoe_shape_t& s, int64_t rows, const void* y, int y_dtype, const int32_t* slot, const float* gate_w,
+                   void* out, int accumulate, cudaStream_t st);
+
+// ---- small device helpers ----
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// fp32 -> bf16 bits, round to nearest even (NaN kept quiet).
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
+    uint32_t u = __float_as_uint(f);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (u >> 16) | 0x40u;
+    return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
+}
+
+// 16-byte streaming accesses: every byte of the token matrices is touched once per kernel.
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+}  // namespace locmoe

@@ -1,0 +1,241 @@
+// Dispatch (row gather into the All-to-All shaped buffer) and gate-weighted
+// combine (first equation of Sec. 3.2.1, top-1: y_m = R_m * expert output).
+//
+// Both are row movers: one warp owns one destination row, reads the whole
+// source row with 16-byte streaming loads and writes the destination row with
+// fully coalesced 16-byte streaming stores.  Rows are at least a few KB, so a
+// gather of whole rows runs at the same DRAM efficiency as a flat copy.  The
+// loads of the next chunk are issued before the stores of the current one.
+#include "common.cuh"
+
+namespace locmoe {
+
+namespace {
+
+constexpr int kCH = 4;
+constexpr int kThreads = 256;
+
+// buf[row] = x[inv[row]] or zeros.  V = 16-byte vectors per row.
+__global__ void __launch_bounds__(kThreads) dispatch_vec_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ inv,
+                                                                uint4* __restrict__ buf, long long rows, int V, int T,
+                                                                int zero_pad) {
+    const int lane = threadIdx.x & 31;
+    const long long nw = (long long)gridDim.x * (blockDim.x >> 5);
+    long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int nch = (V + kCH * kWarp - 1) / (kCH * kWarp);
+    int t_next = row < rows ? inv[row] : -1;
+    for (; row < rows; row += nw) {
+        const int t = t_next;
+        if (row + nw < rows) t_next = inv[row + nw];
+        uint4* dst = buf + row * V;
+        if (t < 0 || t >= T) {
+            if (zero_pad)
+                for (int v = lane; v < V; v += kWarp) st_stream(dst + v, make_uint4(0, 0, 0, 0));
+            continue;
+        }
+        const uint4* srcp = x + (long long)t * V;
+        uint4 cur[kCH], nxt[kCH];
+#pragma unroll
+        for (int k = 0; k < kCH; ++k) {
+            int v = k * kWarp + lane;
+            if (v < V) cur[k] = ld_stream(srcp + v);
+        }
+        for (int c = 0; c < nch; ++c) {
+            if (c + 1 < nch) {
+#pragma unroll
+                for (int k = 0; k < kCH; ++k) {
+                    int v = ((c + 1) * kCH + k) * kWarp + lane;
+                    if (v < V) nxt[k] = ld_stream(srcp + v);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < kCH; ++k) {
+                int v = (c * kCH + k) * kWarp + lane;
+                if (v < V) st_stream(dst + v, cur[k]);
+            }
+#pragma unroll
+            for (int k = 0; k < kCH; ++k) cur[k] = nxt[k];
+        }
+    }
+}
+
+// Element-wise fallback for rows that are not a multiple of 16 bytes or misaligned bases.
+template <typename E>
+__global__ void __launch_bounds__(kThreads) dispatch_scalar_kernel(const E* __restrict__ x, const int32_t* __restrict__ inv,
+                                                                   E* __restrict__ buf, long long rows, int H, int T,
+                                                                   int zero_pad) {
+    const int lane = threadIdx.x & 31;
+    const long long nw = (long long)gridDim.x * (blockDim.x >> 5);
+    for (long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); row < rows; row += nw) {
+        const int t = inv[row];
+        E* dst = buf + row * H;
+        if (t < 0 || t >= T) {
+            if (zero_pad) for (int j = lane; j < H; j += kWarp) dst[j] = E(0);
+            continue;
+        }
+        const E* srcp = x + (long long)t * H;
+        for (int j = lane; j < H; j += kWarp) dst[j] = srcp[j];
+    }
+}
+
+// ---- combine ----
+template <int DT> struct Oct;   // 8 consecutive elements
+template <> struct Oct<LOCMOE_F32> {
+    static constexpr int NV = 2;
+    __device__ static __forceinline__ void load(const void* base, long long o, float (&f)[8]) {
+        const uint4* p = reinterpret_cast<const uint4*>(base) + o * 2;
+        uint4 a = ld_stream(p), b = ld_stream(p + 1);
+        f[0] = __uint_as_float(a.x); f[1] = __uint_as_float(a.y); f[2] = __uint_as_float(a.z); f[3] = __uint_as_float(a.w);
+        f[4] = __uint_as_float(b.x); f[5] = __uint_as_float(b.y); f[6] = __uint_as_float(b.z); f[7] = __uint_as_float(b.w);
+    }
+    __device__ static __forceinline__ void store(void* base, long long o, const float (&f)[8]) {
+        uint4* p = reinterpret_cast<uint4*>(base) + o * 2;
+        st_stream(p, make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3])));
+        st_stream(p + 1, make_uint4(__float_as_uint(f[4]), __float_as_uint(f[5]), __float_as_uint(f[6]), __float_as_uint(f[7])));
+    }
+};
+template <> struct Oct<LOCMOE_BF16> {
+    static constexpr int NV = 1;
+    __device__ static __forceinline__ void load(const void* base, long long o, float (&f)[8]) {
+        uint4 a = ld_stream(reinterpret_cast<const uint4*>(base) + o);
+        f[0] = bf16_lo(a.x); f[1] = bf16_hi(a.x); f[2] = bf16_lo(a.y); f[3] = bf16_hi(a.y);
+        f[4] = bf16_lo(a.z); f[5] = bf16_hi(a.z); f[6] = bf16_lo(a.w); f[7] = bf16_hi(a.w);
+    }
+    __device__ static __forceinline__ void store(void* base, long long o, const float (&f)[8]) {
+        st_stream(reinterpret_cast<uint4*>(base) + o,
+                  make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7])));
+    }
+};
+
+// out[t] (+)= gate_w[t] * y[slot[t]]; O = octets (8 elements) per row.
+template <int YDT, int ODT, bool ACC>
+__global__ void __launch_bounds__(kThreads) combine_vec_kernel(const void* __restrict__ y, const int32_t* __restrict__ slot,
+                                                               const float* __restrict__ gate_w, void* __restrict__ out,
+                                                               int T, int O, long long rows) {
+    constexpr int CH = 4;
+    const int lane = threadIdx.x & 31;
+    const int nw = gridDim.x * (blockDim.x >> 5);
+    const int nch = (O + CH * kWarp - 1) / (CH * kWarp);
+    for (int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); t < T; t += nw) {
+        const int s = slot[t];
+        const long long obase = (long long)t * O;
+        if (s < 0 || s >= rows) {
+            if (!ACC) {
+                const float z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                for (int o = lane; o < O; o += kWarp) Oct<ODT>::store(out, obase + o, z);
+            }
+            continue;
+        }
+        const float w = gate_w[t];
+        const long long ybase = (long long)s * O;
+        for (int c = 0; c < nch; ++c) {
+            float f[CH][8], prev[CH][8];
+#pragma unroll
+            for (int k = 0; k < CH; ++k) {
+                int o = (c * CH + k) * kWarp + lane;
+                if (o < O) {
+                    Oct<YDT>::load(y, ybase + o, f[k]);
+                    if (ACC) Oct<ODT>::load(out, obase + o, prev[k]);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < CH; ++k) {
+                int o = (c * CH + k) * kWarp + lane;
+                if (o < O) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) f[k][e] = ACC ? fmaf(w, f[k][e], prev[k][e]) : w * f[k][e];
+                    Oct<ODT>::store(out, obase + o, f[k]);
+                }
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ float load_elem(const void* p, long long i, int dt) {
+    if (dt == LOCMOE_F32) return reinterpret_cast<const float*>(p)[i];
+    return __uint_as_float(((uint32_t) reinterpret_cast<const uint16_t*>(p)[i]) << 16);
+}
+__device__ __forceinline__ void store_elem(void* p, long long i, int dt, float v) {
+    if (dt == LOCMOE_F32) reinterpret_cast<float*>(p)[i] = v;
+    else reinterpret_cast<uint16_t*>(p)[i] = (uint16_t)f32_to_bf16_bits(v);
+}
+
+__global__ void __launch_bounds__(kThreads) combine_scalar_kernel(const void* __restrict__ y, int ydt,
+                                                                  const int32_t* __restrict__ slot,
+                                                                  const float* __restrict__ gate_w, void* __restrict__ out,
+                                                                  int odt, int T, int H, long long rows, int acc) {
+    const int lane = threadIdx.x & 31;
+    const int nw = gridDim.x * (blockDim.x >> 5);
+    for (int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); t < T; t += nw) {
+        const int s = slot[t];
+        const long long ob = (long long)t * H;
+        if (s < 0 || s >= rows) {
+            if (!acc) for (int j = lane; j < H; j += kWarp) store_elem(out, ob + j, odt, 0.0f);
+            continue;
+        }
+        const float w = gate_w[t];
+        const long long yb = (long long)s * H;
+        for (int j = lane; j < H; j += kWarp) {
+            float v = load_elem(y, yb + j, ydt);
+            v = acc ? fmaf(w, v, load_elem(out, ob + j, odt)) : w * v;
+            store_elem(out, ob + j, odt, v);
+        }
+    }
+}
+
+int grid_for(long long units, int warps_per_block, int blocks_per_sm) {
+    long long want = (units + warps_per_block - 1) / warps_per_block;
+    long long cap = (long long)blocks_per_sm * sm_count();
+    if (want > cap) want = cap;
+    return want < 1 ? 1 : (int)want;
+}
+
+}  // namespace
+
+int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const int32_t* inv, void* buf,
+                    int zero_pad, cudaStream_t st) {
+    const int esz = s.x_dtype == LOCMOE_F32 ? 4 : 2;
+    const size_t rb = (size_t)s.H * esz;
+    const bool vec_ok = rb % 16 == 0 && (uintptr_t)x % 16 == 0 && (uintptr_t)buf % 16 == 0;
+    const int grid = grid_for(rows, kThreads / 32, 8);
+    if (vec_ok) {
+        dispatch_vec_kernel<<<grid, kThreads, 0, st>>>(static_cast<const uint4*>(x), inv, static_cast<uint4*>(buf), rows,
+                                                       (int)(rb / 16), s.T, zero_pad);
+    } else if (esz == 4) {
+        dispatch_scalar_kernel<uint32_t><<<grid, kThreads, 0, st>>>(static_cast<const uint32_t*>(x), inv,
+                                                                    static_cast<uint32_t*>(buf), rows, s.H, s.T, zero_pad);
+    } else {
+        dispatch_scalar_kernel<uint16_t><<<grid, kThreads, 0, st>>>(static_cast<const uint16_t*>(x), inv,
+                                                                    static_cast<uint16_t*>(buf), rows, s.H, s.T, zero_pad);
+    }
+    return check_launch();
+}
+
+int launch_combine(const locmoe_shape_t& s, int64_t rows, const void* y, int y_dtype, const int32_t* slot,
+                   const float* gate_w, void* out, int accumulate, cudaStream_t st) {
+    const bool vec_ok = s.H % 8 == 0 && (uintptr_t)y % 16 == 0 && (uintptr_t)out % 16 == 0;
+    const int grid = grid_for(s.T, kThreads / 32, 8);
+    if (!vec_ok) {
+        combine_scalar_kernel<<<grid, kThreads, 0, st>>>(y, y_dtype, slot, gate_w, out, s.x_dtype, s.T, s.H, rows,
+                                                         accumulate);
+        return check_launch();
+    }
+    const int O = s.H / 8;
+#define LOCMOE_COMBINE_CASE(YD, OD, AC)                                                                              \
+    if (y_dtype == YD && s.x_dtype == OD && (accumulate != 0) == AC) {                                               \
+        combine_vec_kernel<YD, OD, AC><<<grid, kThreads, 0, st>>>(y, slot, gate_w, out, s.T, O, rows);               \
+        return check_launch();                                                                                       \
+    }
+    LOCMOE_COMBINE_CASE(LOCMOE_F32, LOCMOE_F32, false)
+    LOCMOE_COMBINE_CASE(LOCMOE_F32, LOCMOE_F32, true)
+    LOCMOE_COMBINE_CASE(LOCMOE_F32, LOCMOE_BF16, false)
+    LOCMOE_COMBINE_CASE(LOCMOE_F32, LOCMOE_BF16, true)
+    LOCMOE_COMBINE_CASE(LOCMOE_BF16, LOCMOE_F32, false)
+    LOCMOE_COMBINE_CASE(LOCMOE_BF16, LOCMOE_F32, true)
+    LOCMOE_COMBINE_CASE(LOCMOE_BF16, LOCMOE_BF16, false)
+    LOCMOE_COMBINE_CASE(LOCMOE_BF16, LOCMOE_BF16, true)
+#undef LOCMOE_COMBINE_CASE
+    return LOCMOE_ERR_DTYPE;
+}
+
+}  // namespace locmoe

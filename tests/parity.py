@@ -1,0 +1,208 @@
+"""Stage-wise comparison of the CUDA path (through the C-ABI binding) with the CPU oracle.
+
+Used by the GPU parity tests and by the smoke check.  One flipped expert index
+would shift the queue position of every later token of two queues, so the
+stages are compared one by one, each oracle stage being fed the indices the
+previous comparison has just validated:
+
+  gate      expert index bit-exact except tokens whose top-2 logit gap (oracle,
+            fp64) is below 1e-6 -- those are counted and the GPU's choice must
+            still be a maximiser within that gap; score 1e-5 relative; cosine
+            1e-5 relative (+1e-6 absolute near zero)
+  capacity  delta_e bit-exact on the GPU's own (idx, cos); delta within the cosine
+            tolerance of the oracle's; p_delta / ec_min 1e-8 relative and the
+            integer capacities exact for the oracle evaluated at the GPU's delta
+  route     every integer output bit-exact
+  dispatch  bit-exact rows
+  combine   bf16: 2e-2 absolute; fp32: 1e-5 relative (+1e-6 absolute)
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2401_13920_b200 import binding as B
+from paper_2401_13920_b200 import workloads as W
+
+GAP_EXCUSE = 1e-6
+GATE_RTOL = 1e-5
+COS_RTOL, COS_ATOL = 1e-5, 1e-6
+BF16_OUT_ATOL = 2e-2
+F32_OUT_RTOL, F32_OUT_ATOL = 1e-5, 1e-6
+CHUNK = 65536
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+def oracle_gate_chunked(x_dev, dtype_code, E, eps=None):
+    """Oracle gate over device tokens, copied to the host chunk by chunk."""
+    T = x_dev.shape[0]
+    idx = np.empty(T, np.int32)
+    R = np.empty(T, np.float64)
+    cs = np.empty(T, np.float64)
+    gap = np.empty(T, np.float64)
+    for s in range(0, T, CHUNK):
+        g = oracle.gate(W.host_bits(x_dev[s:s + CHUNK]), dtype_code, E, eps=eps)
+        n = g.idx.shape[0]
+        idx[s:s + n], R[s:s + n], cs[s:s + n], gap[s:s + n] = g.idx, g.R, g.cos, g.gap
+    return idx, R, cs, gap
+
+
+def check_gate(x, shape, st, eps_dev=None):
+    eps_h = None if eps_dev is None else _np(eps_dev)
+    idx_o, R_o, cos_o, gap = oracle_gate_chunked(x, shape.x_dtype, shape.E, eps_h)
+    idx_g, R_g, cos_g = _np(st.idx), _np(st.gate_w).astype(np.float64), _np(st.cos_sim).astype(np.float64)
+    excused = gap < GAP_EXCUSE
+    differ = idx_g != idx_o
+    bad = differ & ~excused
+    assert not bad.any(), "expert index differs on %d non-excused tokens, first %s" % (bad.sum(), np.nonzero(bad)[0][:5])
+    # an excused token that differs must still have picked a maximiser within the gap
+    for t in np.nonzero(differ)[0]:
+        g = oracle.gate(W.host_bits(x[int(t):int(t) + 1]), shape.x_dtype, shape.E, eps=eps_h, want_G=True)
+        assert 0 <= idx_g[t] < shape.E
+        assert g.G[0, idx_g[t]] >= g.G[0].max() - GAP_EXCUSE, "token %d: GPU expert is not a near-maximiser" % t
+    same = ~differ
+    relR = np.abs(R_g - R_o) / R_o
+    assert relR[same].max() <= GATE_RTOL, "gate score off by %.3g relative" % relR[same].max()
+    assert relR.max() <= 10 * GATE_RTOL
+    okc = np.abs(cos_g - cos_o) <= COS_RTOL * np.abs(cos_o) + COS_ATOL
+    assert okc[same].all(), "cosine off on %d tokens" % (~okc[same]).sum()
+    return dict(idx_o=idx_o, R_o=R_o, cos_o=cos_o, gap=gap, n_excused=int(excused.sum()), n_differ=int(differ.sum()),
+                max_rel_R=float(relR[same].max()), max_abs_cos=float(np.abs(cos_g - cos_o)[same].max()))
+
+
+def check_capacity(shape, st, rule, gate_info):
+    cap = B.locmoe_capacity_read(st.cap_dev)
+    idx_g, cos_g = _np(st.idx), _np(st.cos_sim)
+    D = shape.D
+    own = oracle.capacity(idx_g, cos_g.astype(np.float64), shape.E, shape.H, D, rule.min_mult, rule.capacity_factor,
+                          rule.delta_override, rule.bound_form)
+    assert np.array_equal(_np(st.delta_e), own.delta_e.astype(np.float32)), "delta_e is not the per-expert minimum"
+    assert np.allclose(_np(st.theta_e), np.arccos(np.clip(own.delta_e, -1, 1)), rtol=1e-6, atol=1e-6)
+    assert cap.n_empty_experts == own.n_empty_experts
+    assert cap.delta == own.delta, "delta %r vs %r" % (cap.delta, own.delta)
+    # against the oracle's own gate outputs (fp64 cosines)
+    ref = oracle.capacity(gate_info["idx_o"], gate_info["cos_o"], shape.E, shape.H, D, rule.min_mult,
+                          rule.capacity_factor, rule.delta_override, rule.bound_form)
+    assert abs(cap.delta - ref.delta) <= COS_RTOL * abs(ref.delta) + COS_ATOL
+    # closed forms and the integer rule at the GPU's delta
+    at = oracle.capacity(idx_g, cos_g.astype(np.float64), shape.E, shape.H, D, rule.min_mult, rule.capacity_factor,
+                         cap.delta if rule.delta_override < 0 else rule.delta_override, rule.bound_form)
+    assert math.isclose(cap.p_delta, at.p_delta, rel_tol=1e-8, abs_tol=1e-300), (cap.p_delta, at.p_delta)
+    assert math.isclose(cap.ec_min, at.ec_min, rel_tol=1e-8), (cap.ec_min, at.ec_min)
+    assert (cap.C_expert, cap.C_local) == (at.C_expert, at.C_local), \
+        "capacity (%d,%d) vs oracle (%d,%d)" % (cap.C_expert, cap.C_local, at.C_expert, at.C_local)
+    return cap, ref
+
+
+def check_route(shape, st, src, cap):
+    idx_g = _np(st.idx)
+    ref = oracle.route(idx_g, _np(src), shape.E, shape.n_nodes, shape.dev_per_node, cap.C_local, st.C_alloc, shape.layout)
+    for name in ("pos", "slot", "drop", "inv", "load"):
+        got = _np(getattr(st, name))
+        want = getattr(ref, name)
+        assert np.array_equal(got, want), "%s differs at %s" % (name, np.nonzero(got != want)[0][:5])
+    D, E = shape.D, shape.E
+    assert np.array_equal(_np(st.counts).reshape(D, E), ref.counts)
+    assert np.array_equal(_np(st.kept).reshape(D, E), ref.kept)
+    assert np.array_equal(_np(st.send_counts).reshape(D, D), ref.send_counts)
+    assert np.array_equal(_np(st.locality).reshape(2, 3), ref.locality)
+    assert int(st.status.item()) == ref.status
+    return ref
+
+
+def check_dispatch_full(x, shape, st, ref_route):
+    want = oracle.dispatch(W.host_bits(x), shape.x_dtype, ref_route.slot, st.rows)
+    got = W.host_bits(st.buf)
+    assert np.array_equal(got, want), "dispatched buffer differs"
+
+
+def check_dispatch_sampled(x, shape, st, ref_route, rows_sample):
+    """Rows chosen by the caller: an occupied row holds its token bit for bit, an empty one is zero."""
+    rs = torch.as_tensor(rows_sample, dtype=torch.int64, device=x.device)
+    got = W.host_bits(st.buf[rs])
+    inv = ref_route.inv[rows_sample]
+    toks = np.where(inv >= 0, inv, 0)
+    xs = W.host_bits(x[torch.as_tensor(toks, dtype=torch.int64, device=x.device)])
+    sub_slot = np.where(inv >= 0, np.arange(len(rows_sample)), -1).astype(np.int32)
+    want = oracle.dispatch(xs, shape.x_dtype, sub_slot, len(rows_sample))
+    assert np.array_equal(got, want), "sampled buffer rows differ"
+
+
+def _out_close(got_bits, want64, x_dtype):
+    if x_dtype == B.BF16:
+        got = oracle.bf16_bits_to_f64(got_bits)
+        err = np.abs(got - want64)
+        assert err.max() <= BF16_OUT_ATOL, "combined output off by %.3g" % err.max()
+        # a correctly rounded bf16 result is much closer than the gate: half an ulp
+        half_ulp_bound = np.maximum(np.abs(want64), 2.0 ** -126) * 2.0 ** -8   # half an ulp is at most |v| / 256
+        assert (err <= 1.02 * half_ulp_bound).all(), "combined output is not within half a bf16 ulp"
+    else:
+        err = np.abs(got_bits.astype(np.float64) - want64)
+        assert (err <= F32_OUT_RTOL * np.abs(want64) + F32_OUT_ATOL).all(), "combined output off by %.3g" % err.max()
+    return float(err.max())
+
+
+def check_combine_sampled(y, shape, st, ref_route, gate_info, tokens_sample):
+    """Tokens chosen by the caller: out[t] = R_t * y[slot_t] in fp64 (0 when dropped).
+
+    R is the oracle's score for tokens whose index agrees, the GPU's (validated to 1e-5) otherwise."""
+    ts = np.asarray(tokens_sample)
+    tdev = torch.as_tensor(ts, dtype=torch.int64, device=y.device)
+    slot = ref_route.slot[ts]
+    rows = np.where(slot >= 0, slot, 0)
+    ys = W.host_bits(y[torch.as_tensor(rows, dtype=torch.int64, device=y.device)])
+    sub_slot = np.where(slot >= 0, np.arange(len(ts)), -1).astype(np.int32)
+    R = np.where(gate_info["idx_o"][ts] == _np(st.idx)[ts], gate_info["R_o"][ts], _np(st.gate_w)[ts].astype(np.float64))
+    want = oracle.combine(ys, B.dtype_code(y.dtype), sub_slot, R)
+    got = W.host_bits(st.out[tdev])
+    return _out_close(got, want, shape.x_dtype)
+
+
+def run_staged(w: W.Workload, capacity_factor=1.0, min_mult=None, layout=B.LAYOUT_SEND, delta_override=-1.0,
+               bound_form=B.BOUND_BETA, C_alloc=None, full=True, n_sample=512, y_random=False, eps=None, seed=0):
+    """Runs the five calls on the workload and compares every stage; returns a small report."""
+    dev = torch.device("cuda:0")
+    x = W.make_tokens(w, dev)
+    src = W.make_src(w, dev)
+    shape = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, layout)
+    rule = B.CapacityRule(capacity_factor if min_mult is None else min_mult, capacity_factor, delta_override, bound_form, 0)
+    if C_alloc is None:
+        C_alloc = B.conventional_capacity(w.T, shape.D, w.E, capacity_factor)
+    st = B.make_router(shape, C_alloc, rule, dev)
+    eps_dev = None if eps is None else torch.as_tensor(eps, dtype=torch.float32, device=dev)
+    y = None
+    if y_random:
+        y = W.make_expert_out(w, st.rows, dev, "f32" if w.y_dtype == "f32" else w.dtype)
+    B.router_forward(st, x, src, y=y, eps=eps_dev)
+    torch.cuda.synchronize()
+
+    rep = {"workload": w.name, "T": w.T, "C_alloc": C_alloc}
+    gi = check_gate(x, shape, st, eps_dev)
+    rep.update(n_excused=gi["n_excused"], n_differ=gi["n_differ"], max_rel_R=gi["max_rel_R"])
+    cap, _ = check_capacity(shape, st, rule, gi)
+    rep.update(delta=cap.delta, ec_min=cap.ec_min, C_local=cap.C_local, C_expert=cap.C_expert)
+    rr = check_route(shape, st, src, cap)
+    rep.update(drop_frac=float(rr.drop.mean()), status=rr.status)
+    ysrc = st.buf if y is None else y
+    rng = np.random.default_rng(seed)
+    if full:
+        check_dispatch_full(x, shape, st, rr)
+        rep["max_out_err"] = check_combine_sampled(ysrc, shape, st, rr, gi, np.arange(w.T))
+    else:
+        rows_sample = np.unique(np.concatenate([rng.integers(0, st.rows, n_sample), [0, st.rows - 1]]))
+        check_dispatch_sampled(x, shape, st, rr, rows_sample)
+        dropped = np.nonzero(rr.drop)[0][:n_sample // 4]
+        toks = np.unique(np.concatenate([rng.integers(0, w.T, n_sample), [0, w.T - 1], dropped]))
+        rep["max_out_err"] = check_combine_sampled(ysrc, shape, st, rr, gi, toks)
+        # properties that hold at any size
+        occupied = int((st.inv >= 0).sum().item())
+        assert occupied == w.T - int(rr.drop.sum())
+        assert int((st.buf != 0).any(dim=1).sum().item()) <= occupied
+        assert not st.out[torch.as_tensor(dropped, dtype=torch.int64, device=dev)].any().item()
+    return rep

@@ -1,0 +1,197 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the CPU
+oracle on the same seeded inputs (stage by stage, see tests/parity.py)."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import oracle
+    oracle.build()
+    from tests import parity
+    return parity
+
+
+def _wl(P, **kw):
+    base = dict(name="case", config=9, T=1000, H=256, E=8, n_nodes=2, dev_per_node=2, dtype="bf16",
+                tokens="normal", src="uniform")
+    base.update(kw)
+    return P.W.Workload(**base)
+
+
+# ---- the five configurations at sizes the oracle covers element by element ----
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_config1_tiny_full_size(P, layout):
+    rep = P.run_staged(P.W.CONFIGS[1], 1.0, layout=layout, full=True)
+    assert rep["C_local"] == 64 and 0.02 < rep["drop_frac"] < 0.10
+
+
+@pytest.mark.parametrize("cfg,T", [(2, 6000), (3, 8229), (5, 7001)])
+def test_configs_scaled_full_compare(P, cfg, T):
+    rep = P.run_staged(P.W.CONFIGS[cfg].scaled(T), 1.0, full=True)
+    assert rep["status"] == 0
+
+
+@pytest.mark.parametrize("mult", [1.0, 1.25, 2.0])
+def test_config4_scaled_capacity_multipliers_random_fp32_expert_out(P, mult):
+    # group width 20 bf16 (40 bytes): 16-byte vectors straddle group boundaries
+    rep = P.run_staged(P.W.CONFIGS[4].scaled(5003), mult, full=True, y_random=True)
+    assert rep["C_local"] == int(np.ceil(mult * 5003 / 65536))
+
+
+# ---- full sizes, in the launch configuration the bench times; outputs sampled ----
+
+@pytest.mark.parametrize("cfg", [2, 5, 3])
+def test_configs_full_size_sampled(P, cfg):
+    w = P.W.CONFIGS[cfg]
+    rep = P.run_staged(w, 1.0, full=False, n_sample=1024)
+    assert rep["C_local"] == w.T // (w.D * w.E)
+    if cfg == 3:
+        assert rep["drop_frac"] > 0.3     # the Zipf mixture forces imbalance and drops
+    else:
+        assert 0.03 < rep["drop_frac"] < 0.15
+
+
+def test_config4_full_size_sampled(P):
+    w = P.W.CONFIGS[4]
+    rep = P.run_staged(w, 1.0, full=False, n_sample=1024, y_random=True)
+    assert rep["C_local"] == 16 and 0.05 < rep["drop_frac"] < 0.15
+
+
+# ---- edge cases and degenerate inputs ----
+
+@pytest.mark.parametrize("kw", [
+    dict(T=1, H=64, E=4, n_nodes=1, dev_per_node=2),
+    dict(T=31, H=64, E=1, n_nodes=1, dev_per_node=1),                   # one expert: R = 1
+    dict(T=777, H=60, E=4, n_nodes=1, dev_per_node=4, dtype="f32"),     # odd group width 15 (unit = 1 element)
+    dict(T=777, H=16, E=8, n_nodes=2, dev_per_node=2),                  # group width 2
+    dict(T=777, H=36, E=4, n_nodes=2, dev_per_node=2),                  # rows of 72 bytes: scalar path
+    dict(T=513, H=1024, E=512, n_nodes=4, dev_per_node=8),              # many experts, Ed = 16
+    dict(T=2049, H=2048, E=8, n_nodes=2, dev_per_node=4, dtype="f32"),  # group spans whole warp iterations
+    dict(T=3000, H=4096, E=2048, n_nodes=1, dev_per_node=1),            # > 1024 keys on a single device
+    dict(T=4097, H=2048, E=2048, n_nodes=8, dev_per_node=8),            # 131072 keys: three radix passes; g = 1
+])
+@pytest.mark.parametrize("layout", [0, 1])
+def test_shapes(P, kw, layout):
+    P.run_staged(_wl(P, **kw), 1.0, layout=layout, full=True)
+
+
+def test_literal_minimum_mode_one_slot_per_pair(P):
+    # c_f = 0: capacity = ceil(Theorem 1's minimum) = 1 slot per (source, expert) pair
+    rep = P.run_staged(P.W.CONFIGS[2].scaled(20000), 0.0, min_mult=1.0, C_alloc=1, full=True)
+    assert rep["C_local"] == 1 and rep["drop_frac"] > 0.7
+
+
+def test_minimum_binds_on_aligned_tokens(P):
+    # tokens pushed along their expert's gating direction: large delta, Theorem 1's minimum exceeds T / n
+    w = _wl(P, T=4096, H=1024, E=8, n_nodes=2, dev_per_node=4, dtype="f32", tokens="zipf_mixture", config=8)
+    rep = P.run_staged(w, 0.5, min_mult=1.0, delta_override=0.134, C_alloc=600, full=True)
+    assert rep["C_expert"] == 4096 and rep["C_local"] == 512
+
+
+@pytest.mark.parametrize("form", [1, 2])
+def test_bound_forms_with_the_papers_delta(P, form):
+    rep = P.run_staged(P.W.CONFIGS[2].scaled(3000), 1.0, delta_override=0.03, bound_form=form, full=True)
+    assert rep["delta"] == 0.03
+
+
+def test_capacity_clamped_to_the_allocation(P):
+    rep = P.run_staged(P.W.CONFIGS[1], 2.0, C_alloc=40, full=True)
+    assert rep["status"] & 1 and rep["C_local"] == 128
+
+
+def test_bias_and_probs(P):
+    W, B = P.W, P.B
+    w = _wl(P, T=2000, H=512, E=16, n_nodes=2, dev_per_node=4)
+    eps = np.linspace(-0.05, 0.05, 16).astype(np.float32)
+    P.run_staged(w, 1.0, eps=eps, full=True)
+    dev = torch.device("cuda:0")
+    x = W.make_tokens(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, 2, 4, x.dtype)
+    idx = torch.empty(w.T, dtype=torch.int32, device=dev)
+    gw = torch.empty(w.T, device=dev)
+    cs = torch.empty(w.T, device=dev)
+    probs = torch.empty(w.T, w.E, device=dev)
+    B.locmoe_gate(sh, x, torch.as_tensor(eps, device=dev), idx, gw, cs, probs)
+    ref = P.oracle.gate(W.host_bits(x), sh.x_dtype, w.E, eps=eps, want_probs=True)
+    assert np.allclose(probs.cpu().numpy(), ref.probs, rtol=1e-5, atol=1e-9)
+    assert torch.allclose(probs.sum(1), torch.ones(w.T, device=dev), atol=1e-5)
+
+
+def test_bad_source_device_is_dropped_and_flagged(P):
+    W, B = P.W, P.B
+    w = _wl(P, T=1500, H=128, E=8, n_nodes=2, dev_per_node=2)
+    dev = torch.device("cuda:0")
+    x = W.make_tokens(w, dev)
+    src = W.make_src(w, dev)
+    src[7] = 99
+    src[1200] = -3
+    sh = B.make_shape(w.T, w.H, w.E, 2, 2, x.dtype)
+    rule = B.CapacityRule(1.0, 1.0, -1.0, 0, 0)
+    st = B.make_router(sh, 60, rule, dev)
+    B.router_forward(st, x, src)
+    torch.cuda.synchronize()
+    cap = B.locmoe_capacity_read(st.cap_dev)
+    ref = P.check_route(sh, st, src, cap)
+    assert ref.status == 2 and ref.drop[7] == 1 and ref.pos[1200] == -1
+    assert not st.out[7].any().item()
+
+
+def test_accumulate_adds_to_the_output(P):
+    W, B = P.W, P.B
+    w = _wl(P, T=900, H=256, E=8, n_nodes=2, dev_per_node=2, dtype="f32")
+    dev = torch.device("cuda:0")
+    x = W.make_tokens(w, dev)
+    src = W.make_src(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, 2, 2, x.dtype)
+    st = B.make_router(sh, 20, B.CapacityRule(1.0, 1.0, -1.0, 0, 0), dev)
+    B.router_forward(st, x, src)
+    first = st.out.clone()
+    B.locmoe_combine(sh, 20, st.buf, st.slot, st.gate_w, st.out, accumulate=True)
+    torch.cuda.synchronize()
+    ref = P.oracle.combine(W.host_bits(st.buf), B.F32, st.slot.cpu().numpy(), st.gate_w.double().cpu().numpy(),
+                           prev=first.double().cpu().numpy())
+    assert np.allclose(st.out.cpu().numpy(), ref, rtol=1e-5, atol=1e-6)
+
+
+def test_round_trip_identity_experts_unit_scores(P):
+    # combine(dispatch(x)) with R = 1 returns x bit for bit on kept tokens and 0 on dropped ones
+    W, B = P.W, P.B
+    w = P.W.CONFIGS[5].scaled(9000)
+    dev = torch.device("cuda:0")
+    x = W.make_tokens(w, dev)
+    src = W.make_src(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype)
+    st = B.make_router(sh, 9, B.CapacityRule(1.0, 1.0, -1.0, 0, 0), dev)
+    B.router_forward(st, x, src)
+    ones = torch.ones(w.T, device=dev)
+    B.locmoe_combine(sh, 9, st.buf, st.slot, ones, st.out)
+    torch.cuda.synchronize()
+    keep = st.slot >= 0
+    assert 0 < int(keep.sum()) < w.T
+    assert torch.equal(st.out[keep].view(torch.int16), x[keep].view(torch.int16))
+    assert not st.out[~keep].any().item()
+
+
+def test_route_is_deterministic(P):
+    W, B = P.W, P.B
+    w = P.W.CONFIGS[3].scaled(50000)
+    dev = torch.device("cuda:0")
+    x = W.make_tokens(w, dev)
+    src = W.make_src(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype)
+    st = B.make_router(sh, 4, B.CapacityRule(1.0, 1.0, -1.0, 0, 0), dev)
+    B.router_forward(st, x, src)
+    torch.cuda.synchronize()
+    a = [t.clone() for t in (st.pos, st.slot, st.inv, st.counts, st.send_counts, st.locality)]
+    for _ in range(3):
+        B.router_forward(st, x, src)
+        torch.cuda.synchronize()
+        for u, v in zip(a, (st.pos, st.slot, st.inv, st.counts, st.send_counts, st.locality)):
+            assert torch.equal(u, v)
