@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=8)
+    ap.add_argument("--tokens", type=int, default=0, help="override T (profiling-sized case; not the metric's workload)")
     return ap.parse_args()
 
 
@@ -218,6 +219,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     w = W.CONFIGS[args.config]
+    if args.tokens > 0:
+        w = w.scaled(args.tokens)
     if world > 1:
         # every rank routes its own batch: same shape, its own seed
         w = W.Workload(**{**w.__dict__, "config": w.config + 10 * rank, "name": w.name})

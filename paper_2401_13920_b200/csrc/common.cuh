@@ -64,6 +64,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
 }
 
+// Two floats -> packed bf16x2 (x in the low half), round to nearest even, one instruction.
+__device__ __forceinline__ uint32_t cvt_bf16x2(const float2& f) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(f.y), "f"(f.x));
+    return r;
+}
+
 // 16-byte streaming accesses: every byte of the token matrices is touched once per kernel.
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     uint4 v;

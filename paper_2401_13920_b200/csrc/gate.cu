@@ -16,8 +16,6 @@ namespace locmoe {
 
 namespace {
 
-constexpr int kCH = 4;  // 16-byte vectors per lane per chunk
-
 struct GateArgs {
     const void* x;
     const float* eps;
@@ -30,36 +28,39 @@ struct GateArgs {
     int nch;          // chunks per row
     int PU;           // units per group
     int PS;           // padded strip stride per group (floats)
-    uint32_t magic;   // ceil(2^32 / PU) for p / PU by multiply-high
     int S, logS;      // lanes cooperating on one group in the strip reduction
     int warp_floats;  // shared floats per warp
+    int tab_ints;     // shared ints of the strip-offset table (one per unit of a row)
     float inv_g, sqrt_g;
 };
 
+// A 16-byte vector as NP packed pairs of floats (Blackwell has two-wide fp32 add / fma).
 template <int DT>
 struct Vec;
 template <>
 struct Vec<LOCMOE_F32> {
-    static constexpr int VE = 4;
-    __device__ static __forceinline__ void unpack(const uint4& v, float (&f)[4]) {
-        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
-        f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    static constexpr int NP = 2;
+    __device__ static __forceinline__ void unpack(const uint4& v, float2 (&p)[2]) {
+        p[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+        p[1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
     }
 };
 template <>
 struct Vec<LOCMOE_BF16> {
-    static constexpr int VE = 8;
-    __device__ static __forceinline__ void unpack(const uint4& v, float (&f)[8]) {
-        f[0] = bf16_lo(v.x); f[1] = bf16_hi(v.x); f[2] = bf16_lo(v.y); f[3] = bf16_hi(v.y);
-        f[4] = bf16_lo(v.z); f[5] = bf16_hi(v.z); f[6] = bf16_lo(v.w); f[7] = bf16_hi(v.w);
+    static constexpr int NP = 4;
+    __device__ static __forceinline__ void unpack(const uint4& v, float2 (&p)[4]) {
+        p[0] = make_float2(bf16_lo(v.x), bf16_hi(v.x));
+        p[1] = make_float2(bf16_lo(v.y), bf16_hi(v.y));
+        p[2] = make_float2(bf16_lo(v.z), bf16_hi(v.z));
+        p[3] = make_float2(bf16_lo(v.w), bf16_hi(v.w));
     }
 };
 
-// Sum of U consecutive floats as a balanced tree.
-template <int U>
-__device__ __forceinline__ float tree_sum(const float* f) {
-    if constexpr (U == 1) return f[0];
-    else return tree_sum<U / 2>(f) + tree_sum<U / 2>(f + U / 2);
+// Sum of NPAIR consecutive pairs (a balanced tree of two-wide adds, then one scalar add).
+template <int NPAIR>
+__device__ __forceinline__ float2 pair_tree(const float2* p) {
+    if constexpr (NPAIR == 1) return p[0];
+    else return __fadd2_rn(pair_tree<NPAIR / 2>(p), pair_tree<NPAIR / 2>(p + NPAIR / 2));
 }
 
 // Softmax / arg-max / cosine of one row from the raw group sums in gsum[E].
@@ -103,84 +104,113 @@ __device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gs
     }
 }
 
-template <int DT, int U>
+// DT: token dtype.  U: elements per unit.  CH: vectors per lane per chunk.
+// EXACT: the row is a whole number of chunks (no bounds tests in the loop).
+template <int DT, int U, int CH, bool EXACT>
 __global__ void __launch_bounds__(256) gate_vec_kernel(const GateArgs a) {
-    constexpr int VE = Vec<DT>::VE;
+    constexpr int NP = Vec<DT>::NP;
+    constexpr int VE = 2 * NP;
     constexpr int UPV = VE / U;  // units per vector
     extern __shared__ float smem[];
     const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int wpb = blockDim.x >> 5;
-    float* part = smem + (size_t)wib * a.warp_floats;
+    // strip offset (in floats) of every unit of a row: unit p of group p / PU sits at p + (p / PU) * pad
+    int* tab = reinterpret_cast<int*>(smem);
+    {
+        const int pad = a.PS - a.PU;
+        for (int p = threadIdx.x; p < a.V * UPV; p += blockDim.x) tab[p] = p + (p / a.PU) * pad;
+    }
+    __syncthreads();
+    float* part = smem + a.tab_ints + (size_t)wib * a.warp_floats;
     float* gsum = part + (size_t)a.E * a.PS;
     const int nw = gridDim.x * wpb;
     const uint4* xv = reinterpret_cast<const uint4*>(a.x);
-    const int pad = a.PS - a.PU;
 
-    uint4 cur[kCH], nxt[kCH];
-    int row = blockIdx.x * wpb + wib, ch = 0;
-    float sq = 0.0f;
+    uint4 bufA[CH], bufB[CH];
+    float2 sq2 = make_float2(0.0f, 0.0f);
 
-    auto load = [&](uint4 (&buf)[kCH], int r, int c) {
-        const uint4* base = xv + (size_t)r * a.V;
+    auto load = [&](uint4 (&buf)[CH], int r, int c) {
+        const uint4* base = xv + (size_t)r * a.V + c * (CH * kWarp) + lane;
 #pragma unroll
-        for (int k = 0; k < kCH; ++k) {
-            int v = (c * kCH + k) * kWarp + lane;
-            buf[k] = (v < a.V) ? ld_stream(base + v) : make_uint4(0, 0, 0, 0);
+        for (int k = 0; k < CH; ++k) {
+            if (EXACT || c * (CH * kWarp) + k * kWarp + lane < a.V) buf[k] = ld_stream(base + k * kWarp);
+            else buf[k] = make_uint4(0, 0, 0, 0);
         }
     };
 
-    if (row < a.T) load(cur, row, 0);
-    while (row < a.T) {
+    auto consume = [&](const uint4 (&buf)[CH], int c) {
+        const int v0 = c * (CH * kWarp) + lane;
+        const int* tb = tab + v0 * UPV;
+#pragma unroll
+        for (int k = 0; k < CH; ++k) {
+            if (EXACT || v0 + k * kWarp < a.V) {
+                float2 p[NP];
+                Vec<DT>::unpack(buf[k], p);
+#pragma unroll
+                for (int e = 0; e < NP; ++e) sq2 = __ffma2_rn(p[e], p[e], sq2);
+                if constexpr (U >= 2) {
+                    constexpr int PPU = U / 2;  // pairs per unit
+#pragma unroll
+                    for (int u = 0; u < UPV; ++u) {
+                        float2 s2 = pair_tree<PPU>(p + u * PPU);
+                        part[tb[k * kWarp * UPV + u]] = s2.x + s2.y;
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < NP; ++e) {
+                        part[tb[k * kWarp * UPV + 2 * e]] = p[e].x;
+                        part[tb[k * kWarp * UPV + 2 * e + 1]] = p[e].y;
+                    }
+                }
+            }
+        }
+    };
+
+    auto finish_row = [&](int row) {  // the strip holds a whole row: reduce it group by group
+        __syncwarp();
+        if (a.S == 1) {
+            for (int i = lane; i < a.E; i += kWarp) {
+                const float* pp = part + (size_t)i * a.PS;
+                float s = 0.0f;
+                for (int k = 0; k < a.PU; ++k) s += pp[k];
+                gsum[i] = s;
+            }
+        } else {
+            int i = lane >> a.logS, sl = lane & (a.S - 1);
+            float s = 0.0f;
+            if (i < a.E) {
+                const float* pp = part + (size_t)i * a.PS;
+                for (int k = sl; k < a.PU; k += a.S) s += pp[k];
+            }
+            for (int o = a.S >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(full, s, o);
+            if (i < a.E && sl == 0) gsum[i] = s;
+        }
+        __syncwarp();
+        gate_epilogue(a, gsum, sq2.x + sq2.y, row, lane);
+        __syncwarp();
+        sq2 = make_float2(0.0f, 0.0f);
+    };
+
+    int row = blockIdx.x * wpb + wib, ch = 0;
+    if (row >= a.T) return;
+    load(bufA, row, 0);
+    while (true) {
         int ch2 = ch + 1, row2 = row;
         if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
-        if (row2 < a.T) load(nxt, row2, ch2);
+        if (row2 < a.T) load(bufB, row2, ch2);
+        consume(bufA, ch);
+        if (ch2 == 0) finish_row(row);
+        if (row2 >= a.T) break;
+        row = row2; ch = ch2;
 
-#pragma unroll
-        for (int k = 0; k < kCH; ++k) {
-            int v = (ch * kCH + k) * kWarp + lane;
-            if (v < a.V) {
-                float f[VE];
-                Vec<DT>::unpack(cur[k], f);
-#pragma unroll
-                for (int e = 0; e < VE; ++e) sq = fmaf(f[e], f[e], sq);
-#pragma unroll
-                for (int u = 0; u < UPV; ++u) {
-                    int p = v * UPV + u;
-                    int q = pad ? p + (int)__umulhi((uint32_t)p, a.magic) * pad : p;
-                    part[q] = tree_sum<U>(f + u * U);
-                }
-            }
-        }
-
-        if (ch2 == 0) {  // row complete: reduce the strip group by group
-            __syncwarp();
-            if (a.S == 1) {
-                for (int i = lane; i < a.E; i += kWarp) {
-                    const float* pp = part + (size_t)i * a.PS;
-                    float s = 0.0f;
-                    for (int k = 0; k < a.PU; ++k) s += pp[k];
-                    gsum[i] = s;
-                }
-            } else {
-                int i = lane >> a.logS, sl = lane & (a.S - 1);
-                float s = 0.0f;
-                if (i < a.E) {
-                    const float* pp = part + (size_t)i * a.PS;
-                    for (int k = sl; k < a.PU; k += a.S) s += pp[k];
-                }
-                for (int o = a.S >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(full, s, o);
-                if (i < a.E && sl == 0) gsum[i] = s;
-            }
-            __syncwarp();
-            gate_epilogue(a, gsum, sq, row, lane);
-            __syncwarp();
-            sq = 0.0f;
-        }
-#pragma unroll
-        for (int k = 0; k < kCH; ++k) cur[k] = nxt[k];
-        row = row2;
-        ch = ch2;
+        ch2 = ch + 1; row2 = row;
+        if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
+        if (row2 < a.T) load(bufA, row2, ch2);
+        consume(bufB, ch);
+        if (ch2 == 0) finish_row(row);
+        if (row2 >= a.T) break;
+        row = row2; ch = ch2;
     }
 }
 
@@ -223,7 +253,7 @@ int launch_persistent(K kernel, const GateArgs& a, int max_warps, cudaStream_t s
     int wpb = max_warps;
     size_t smem = 0;
     for (; wpb >= 1; wpb >>= 1) {
-        smem = (size_t)wpb * a.warp_floats * sizeof(float);
+        smem = ((size_t)wpb * a.warp_floats + a.tab_ints) * sizeof(float);
         if (smem <= 200 * 1024) break;
     }
     if (wpb < 1) return LOCMOE_ERR_SHAPE;
@@ -262,17 +292,27 @@ int launch_gate(const locmoe_shape_t& s, const void* x, const float* eps, int32_
     }
     const int U = gcd_int(a.g, VE);
     a.V = s.H / VE;
-    a.nch = (a.V + kCH * kWarp - 1) / (kCH * kWarp);
     a.PU = a.g / U;
     a.S = 1; a.logS = 0;
     while (a.S * 2 * s.E <= kWarp && a.S * 2 <= a.PU) { a.S *= 2; a.logS++; }
     // stride congruent to S modulo 2S keeps the strip reads of a warp in distinct banks
     a.PS = a.PU;
     if (a.PU > 1) while (a.PS % (2 * a.S) != a.S) a.PS++;
-    a.magic = a.PU > 1 ? (uint32_t)((0x100000000ull + a.PU - 1) / a.PU) : 0u;
     a.warp_floats = (s.E * a.PS + s.E + 3) & ~3;
-#define LOCMOE_GATE_CASE(DT, UU) \
-    if (s.x_dtype == DT && U == UU) return launch_persistent(gate_vec_kernel<DT, UU>, a, 8, st);
+    a.tab_ints = (s.H / U + 3) & ~3;
+    // chunk size: prefer one that divides the row exactly (no bounds tests in the loop)
+    const int per_lane = a.V / kWarp;
+    const bool whole = a.V % kWarp == 0;
+    int CH = 4;
+    bool exact = whole && per_lane % 4 == 0;
+    if (!exact && whole && per_lane % 5 == 0) { CH = 5; exact = true; }
+    a.nch = (a.V + CH * kWarp - 1) / (CH * kWarp);
+#define LOCMOE_GATE_CASE(DT, UU)                                                                              \
+    if (s.x_dtype == DT && U == UU) {                                                                         \
+        if (exact && CH == 4) return launch_persistent(gate_vec_kernel<DT, UU, 4, true>, a, 8, st);           \
+        if (exact && CH == 5) return launch_persistent(gate_vec_kernel<DT, UU, 5, true>, a, 8, st);           \
+        return launch_persistent(gate_vec_kernel<DT, UU, 4, false>, a, 8, st);                                \
+    }
     LOCMOE_GATE_CASE(LOCMOE_F32, 4)
     LOCMOE_GATE_CASE(LOCMOE_F32, 2)
     LOCMOE_GATE_CASE(LOCMOE_F32, 1)

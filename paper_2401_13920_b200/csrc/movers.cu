@@ -79,31 +79,34 @@ __global__ void __launch_bounds__(kThreads) dispatch_scalar_kernel(const E* __re
 }
 
 // ---- combine ----
-template <int DT> struct Oct;   // 8 consecutive elements
+// 8 consecutive elements ("octet") as four packed float pairs.
+template <int DT> struct Oct;
 template <> struct Oct<LOCMOE_F32> {
-    static constexpr int NV = 2;
-    __device__ static __forceinline__ void load(const void* base, long long o, float (&f)[8]) {
+    __device__ static __forceinline__ void load(const void* base, long long o, float2 (&f)[4]) {
         const uint4* p = reinterpret_cast<const uint4*>(base) + o * 2;
         uint4 a = ld_stream(p), b = ld_stream(p + 1);
-        f[0] = __uint_as_float(a.x); f[1] = __uint_as_float(a.y); f[2] = __uint_as_float(a.z); f[3] = __uint_as_float(a.w);
-        f[4] = __uint_as_float(b.x); f[5] = __uint_as_float(b.y); f[6] = __uint_as_float(b.z); f[7] = __uint_as_float(b.w);
+        f[0] = make_float2(__uint_as_float(a.x), __uint_as_float(a.y));
+        f[1] = make_float2(__uint_as_float(a.z), __uint_as_float(a.w));
+        f[2] = make_float2(__uint_as_float(b.x), __uint_as_float(b.y));
+        f[3] = make_float2(__uint_as_float(b.z), __uint_as_float(b.w));
     }
-    __device__ static __forceinline__ void store(void* base, long long o, const float (&f)[8]) {
+    __device__ static __forceinline__ void store(void* base, long long o, const float2 (&f)[4]) {
         uint4* p = reinterpret_cast<uint4*>(base) + o * 2;
-        st_stream(p, make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3])));
-        st_stream(p + 1, make_uint4(__float_as_uint(f[4]), __float_as_uint(f[5]), __float_as_uint(f[6]), __float_as_uint(f[7])));
+        st_stream(p, make_uint4(__float_as_uint(f[0].x), __float_as_uint(f[0].y), __float_as_uint(f[1].x), __float_as_uint(f[1].y)));
+        st_stream(p + 1, make_uint4(__float_as_uint(f[2].x), __float_as_uint(f[2].y), __float_as_uint(f[3].x), __float_as_uint(f[3].y)));
     }
 };
 template <> struct Oct<LOCMOE_BF16> {
-    static constexpr int NV = 1;
-    __device__ static __forceinline__ void load(const void* base, long long o, float (&f)[8]) {
+    __device__ static __forceinline__ void load(const void* base, long long o, float2 (&f)[4]) {
         uint4 a = ld_stream(reinterpret_cast<const uint4*>(base) + o);
-        f[0] = bf16_lo(a.x); f[1] = bf16_hi(a.x); f[2] = bf16_lo(a.y); f[3] = bf16_hi(a.y);
-        f[4] = bf16_lo(a.z); f[5] = bf16_hi(a.z); f[6] = bf16_lo(a.w); f[7] = bf16_hi(a.w);
+        f[0] = make_float2(bf16_lo(a.x), bf16_hi(a.x));
+        f[1] = make_float2(bf16_lo(a.y), bf16_hi(a.y));
+        f[2] = make_float2(bf16_lo(a.z), bf16_hi(a.z));
+        f[3] = make_float2(bf16_lo(a.w), bf16_hi(a.w));
     }
-    __device__ static __forceinline__ void store(void* base, long long o, const float (&f)[8]) {
+    __device__ static __forceinline__ void store(void* base, long long o, const float2 (&f)[4]) {
         st_stream(reinterpret_cast<uint4*>(base) + o,
-                  make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7])));
+                  make_uint4(cvt_bf16x2(f[0]), cvt_bf16x2(f[1]), cvt_bf16x2(f[2]), cvt_bf16x2(f[3])));
     }
 };
 
@@ -121,15 +124,16 @@ __global__ void __launch_bounds__(kThreads) combine_vec_kernel(const void* __res
         const long long obase = (long long)t * O;
         if (s < 0 || s >= rows) {
             if (!ACC) {
-                const float z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                const float2 z[4] = {{0, 0}, {0, 0}, {0, 0}, {0, 0}};
                 for (int o = lane; o < O; o += kWarp) Oct<ODT>::store(out, obase + o, z);
             }
             continue;
         }
         const float w = gate_w[t];
+        const float2 w2 = make_float2(w, w);
         const long long ybase = (long long)s * O;
         for (int c = 0; c < nch; ++c) {
-            float f[CH][8], prev[CH][8];
+            float2 f[CH][4], prev[CH][4];
 #pragma unroll
             for (int k = 0; k < CH; ++k) {
                 int o = (c * CH + k) * kWarp + lane;
@@ -143,7 +147,7 @@ __global__ void __launch_bounds__(kThreads) combine_vec_kernel(const void* __res
                 int o = (c * CH + k) * kWarp + lane;
                 if (o < O) {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) f[k][e] = ACC ? fmaf(w, f[k][e], prev[k][e]) : w * f[k][e];
+                    for (int e = 0; e < 4; ++e) f[k][e] = ACC ? __ffma2_rn(w2, f[k][e], prev[k][e]) : __fmul2_rn(w2, f[k][e]);
                     Oct<ODT>::store(out, obase + o, f[k]);
                 }
             }

@@ -142,31 +142,38 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(const RouteArg
         block_exclusive_scan(a.counts, a.keystart, a.K, nullptr);
         return;
     }
-    __shared__ unsigned long long loc[6];
-    if (threadIdx.x < 6) loc[threadIdx.x] = 0ull;
-    __syncthreads();
     int C = a.cap->C_local;
     if (C > a.C_alloc) {
         C = a.C_alloc;
         if (blockIdx.x == 2 && threadIdx.x == 0) atomicOr(a.status, LOCMOE_WARN_CLAMPED);
     }
-    unsigned long long l[6] = {0, 0, 0, 0, 0, 0};
+    unsigned long long raw0 = 0, raw1 = 0, raw2 = 0, kp0 = 0, kp1 = 0, kp2 = 0;
     for (int k = (blockIdx.x - 2) * blockDim.x + threadIdx.x; k < a.K; k += (gridDim.x - 2) * blockDim.x) {
         int c = a.counts[k];
         int kp = c < C ? c : C;
         a.kept[k] = kp;
         if (c == 0) continue;
         int s = k / a.E, e = k - s * a.E, b = e / a.Ed;
-        int cls = (b == s) ? 0 : ((b / a.Dn == s / a.Dn) ? 1 : 2);
-        l[cls] += (unsigned long long)c;
-        l[3 + cls] += (unsigned long long)kp;
+        if (b == s) { raw0 += c; kp0 += kp; }
+        else if (b / a.Dn == s / a.Dn) { raw1 += c; kp1 += kp; }
+        else { raw2 += c; kp2 += kp; }
         atomicAdd(&a.load[e], c);
         if (kp) atomicAdd(&a.send_counts[s * a.D + b], kp);
     }
 #pragma unroll
-    for (int i = 0; i < 6; ++i) if (l[i]) atomicAdd(&loc[i], l[i]);
-    __syncthreads();
-    if (threadIdx.x < 6 && loc[threadIdx.x]) atomicAdd(&a.locality[threadIdx.x], loc[threadIdx.x]);
+    for (int o = 16; o > 0; o >>= 1) {
+        raw0 += __shfl_xor_sync(0xffffffffu, raw0, o); raw1 += __shfl_xor_sync(0xffffffffu, raw1, o);
+        raw2 += __shfl_xor_sync(0xffffffffu, raw2, o); kp0 += __shfl_xor_sync(0xffffffffu, kp0, o);
+        kp1 += __shfl_xor_sync(0xffffffffu, kp1, o); kp2 += __shfl_xor_sync(0xffffffffu, kp2, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (raw0) atomicAdd(&a.locality[0], raw0);
+        if (raw1) atomicAdd(&a.locality[1], raw1);
+        if (raw2) atomicAdd(&a.locality[2], raw2);
+        if (kp0) atomicAdd(&a.locality[3], kp0);
+        if (kp1) atomicAdd(&a.locality[4], kp1);
+        if (kp2) atomicAdd(&a.locality[5], kp2);
+    }
 }
 
 template <bool FIRST, bool LAST>
