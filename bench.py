@@ -116,15 +116,6 @@ def physical_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
-def route_passes(D: int, E: int) -> int:
-    """Radix passes the route stage uses for D * E keys (mirrors the library's plan: one pass up to 1024
-    keys, then 8 bits per pass)."""
-    kb = 1
-    while (1 << kb) < D * E:
-        kb += 1
-    return 1 if kb <= 10 else (kb + 7) // 8
-
-
 def oracle_step(oracle, xh, srch, dtype_code, w, cf, layout):
     """One pass of the whole path in the CPU oracle on host arrays; returns kept tokens."""
     T = xh.shape[0]
@@ -311,8 +302,8 @@ def main():
                 "path_frac": sum(bytes_per_launch.values()) / (ms_per_step * 1e-3) / 1e9 / peak,
                 "kernels": kernels, "stage_ms": stage_ms}
 
-    passes = route_passes(shape.D, w.E)
-    launches_per_step = 1 + 2 + (1 + 3 * passes) + 1 + 1
+    launches = B.locmoe_launch_counts(shape)
+    launches_per_step = sum(launches.values())
     cap = B.locmoe_capacity_read(st.cap_dev)
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
@@ -373,7 +364,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic", "config": workload_config(w, args),
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "launches_per_step": launches,
             "roofline": roofline, "cpu_baseline": cpu_baseline,
             "routing": {"kept_fraction": kept / w.T, "C_local": cap.C_local, "C_expert": cap.C_expert, "delta": cap.delta,
                         "ec_min": cap.ec_min, "rows": rows, "kept_tokens_per_s": value * kept / w.T},

@@ -180,6 +180,11 @@ int locmoe_combine(const locmoe_shape_t *shape, int32_t C_alloc, const void *y, 
                    const int32_t *slot, const float *gate_w, void *out, int32_t accumulate,
                    void *stream);
 
+/* Kernels launched per call of gate, capacity, route, dispatch, combine on this
+ * shape (counts[5], host memory); a bookkeeping aid for benchmarks.  The paper
+ * has no counterpart. */
+int locmoe_launch_counts(const locmoe_shape_t *shape, int32_t counts[5]);
+
 /* Text for a return code of this library (host string, never NULL). */
 const char *locmoe_status_string(int code);
 

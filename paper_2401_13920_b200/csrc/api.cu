@@ -138,6 +138,20 @@ int locmoe_combine(const locmoe_shape_t* shape, int32_t C_alloc, const void* y, 
     return launch_combine(*shape, rows, y, y_dtype, slot, gate_w, out, accumulate, static_cast<cudaStream_t>(stream));
 }
 
+int locmoe_launch_counts(const locmoe_shape_t* shape, int32_t counts[5]) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!counts) return LOCMOE_ERR_NULL;
+    RoutePlan p;
+    if ((rc = plan_route(*shape, &p))) return rc;
+    counts[0] = 1;
+    counts[1] = capacity_cluster_eligible(*shape) ? 1 : 2;
+    counts[2] = p.launches;
+    counts[3] = 1;
+    counts[4] = 1;
+    return LOCMOE_OK;
+}
+
 const char* locmoe_status_string(int code) {
     switch (code) {
         case LOCMOE_OK: return "ok";

@@ -1,13 +1,19 @@
 // Angular deviation per expert and the capacity rule (abstract; Lemma 3; Theorem 1; Sec. 3.2.3).
 //
-// Two small kernels after a memset of the scratch: a grid-wide per-expert minimum
-// of the token cosines (integer atomicMin on an order-preserving encoding, so
-// the result does not depend on scheduling), and a single-CTA finish that
+// Per-expert minimum of the token cosines (integer min on an order-preserving
+// encoding, so the result does not depend on scheduling), then a finish that
 // decodes the minima and evaluates the closed forms in fp64 on one thread.
-// Nothing is read back by the host.
+// Moderate batches run as ONE kernel on one thread-block cluster (hardware
+// cluster barrier between the two steps); large ones as memset + grid-wide
+// minimum + single-CTA finish.  Nothing is read back by the host.
 #include <math.h>
+#include <stdlib.h>
+
+#include <cooperative_groups.h>
 
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace locmoe {
 
@@ -86,36 +92,37 @@ __device__ double p_delta_device(double delta, int d) {
     return 1.0 - beta_cf(0.5, b, x, lnx, lny);
 }
 
-__global__ void __launch_bounds__(256) capacity_finish_kernel(const uint32_t* __restrict__ gmin, int T, int E, int H,
-                                                              int D, locmoe_capacity_rule_t rule,
-                                                              float* __restrict__ delta_e, float* __restrict__ theta_e,
-                                                              locmoe_capacity_t* __restrict__ cap) {
-    __shared__ float s_min[256];
-    __shared__ int s_empty[256];
+// Decodes the per-expert minima (nsets partial arrays of E codes each, combined by min), writes delta_e /
+// theta_e, and lets thread 0 evaluate the closed forms and the integer rule.  One CTA, any block size <= 1024.
+__device__ void capacity_finish(const uint32_t* __restrict__ gmin, int nsets, int T, int E, int H, int D,
+                                const locmoe_capacity_rule_t& rule, float* __restrict__ delta_e,
+                                float* __restrict__ theta_e, locmoe_capacity_t* __restrict__ cap) {
+    __shared__ float s_min[32];
+    __shared__ int s_empty[32];
     float lmin = INFINITY;
     int lempty = 0;
     for (int e = threadIdx.x; e < E; e += blockDim.x) {
-        uint32_t c = gmin[e];
+        uint32_t c = 0xffffffffu;
+        for (int k = 0; k < nsets; ++k) c = min(c, __ldcg(gmin + (size_t)k * E + e));
         float de;
         if (c == 0xffffffffu) { de = 1.0f; ++lempty; }
         else { de = order_decode(c); lmin = fminf(lmin, de); }
         delta_e[e] = de;
         theta_e[e] = acosf(fminf(fmaxf(de, -1.0f), 1.0f));
     }
-    s_min[threadIdx.x] = lmin;
-    s_empty[threadIdx.x] = lempty;
-    __syncthreads();
-    for (int o = 128; o > 0; o >>= 1) {
-        if ((int)threadIdx.x < o) {
-            s_min[threadIdx.x] = fminf(s_min[threadIdx.x], s_min[threadIdx.x + o]);
-            s_empty[threadIdx.x] += s_empty[threadIdx.x + o];
-        }
-        __syncthreads();
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lmin = fminf(lmin, __shfl_xor_sync(0xffffffffu, lmin, o));
+        lempty += __shfl_xor_sync(0xffffffffu, lempty, o);
     }
+    if ((threadIdx.x & 31) == 0) { s_min[threadIdx.x >> 5] = lmin; s_empty[threadIdx.x >> 5] = lempty; }
+    __syncthreads();
     if (threadIdx.x != 0) return;
+    const int nwarps = (blockDim.x + 31) >> 5;
+    for (int w = 1; w < nwarps; ++w) { lmin = fminf(lmin, s_min[w]); lempty += s_empty[w]; }
 
     int flags = 0;
-    double delta = (double)s_min[0];
+    double delta = (double)lmin;
     delta = delta < 0.0 ? 0.0 : (delta > 1.0 ? 1.0 : delta);
     if (rule.delta_override >= 0.0) {
         delta = rule.delta_override > 1.0 ? 1.0 : rule.delta_override;
@@ -148,18 +155,65 @@ __global__ void __launch_bounds__(256) capacity_finish_kernel(const uint32_t* __
     cap->ec_min = ec;
     cap->C_expert = (int32_t)ce;
     cap->C_local = (int32_t)cl;
-    cap->n_empty_experts = s_empty[0];
+    cap->n_empty_experts = lempty;
     cap->flags = flags;
+}
+
+__global__ void __launch_bounds__(256) capacity_finish_kernel(const uint32_t* __restrict__ gmin, int T, int E, int H,
+                                                              int D, locmoe_capacity_rule_t rule,
+                                                              float* __restrict__ delta_e, float* __restrict__ theta_e,
+                                                              locmoe_capacity_t* __restrict__ cap) {
+    capacity_finish(gmin, 1, T, E, H, D, rule, delta_e, theta_e, cap);
+}
+
+// Whole stage in one kernel on one cluster: every CTA reduces its share of the tokens into per-expert minima in
+// shared memory and stores them (plain stores, no initialisation needed) as its own row of the scratch; after the
+// hardware cluster barrier CTA 0 combines the rows and finishes.
+constexpr int kCapCS = 8;
+constexpr int kCapThreads = 1024;
+
+__global__ void __cluster_dims__(kCapCS, 1, 1) __launch_bounds__(kCapThreads, 1)
+capacity_cluster_kernel(const int32_t* __restrict__ idx, const float* __restrict__ cs, uint32_t* __restrict__ part,
+                        int T, int E, int H, int D, locmoe_capacity_rule_t rule, float* __restrict__ delta_e,
+                        float* __restrict__ theta_e, locmoe_capacity_t* __restrict__ cap) {
+    extern __shared__ uint32_t smin[];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int cta = (int)cluster.block_rank();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) smin[e] = 0xffffffffu;
+    __syncthreads();
+    for (int t = cta * kCapThreads + threadIdx.x; t < T; t += kCapCS * kCapThreads) {
+        const int e = idx[t];
+        if (e >= 0 && e < E) atomicMin(&smin[e], order_code(cs[t]));
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) part[(size_t)cta * E + e] = smin[e];
+    cluster.sync();
+    if (cta == 0) capacity_finish(part, kCapCS, T, E, H, D, rule, delta_e, theta_e, cap);
 }
 
 }  // namespace
 
-size_t capacity_ws_bytes(const locmoe_shape_t& s) { return ((size_t)s.E * sizeof(uint32_t) + 255) & ~(size_t)255; }
+// One-cluster kernel when the per-expert minima fit in shared memory and the batch is moderate;
+// LOCMOE_PATH=grid|cluster overrides the size rule (testing aid).
+bool capacity_cluster_eligible(const locmoe_shape_t& s) {
+    if (s.E > kSmemExperts) return false;
+    const char* o = getenv("LOCMOE_PATH");
+    if (o && o[0] == 'g') return false;
+    if (o && o[0] == 'c') return true;
+    return s.T <= (1 << 21);
+}
+
+size_t capacity_ws_bytes(const locmoe_shape_t& s) { return ((size_t)kCapCS * s.E * sizeof(uint32_t) + 255) & ~(size_t)255; }
 
 int launch_capacity(const locmoe_shape_t& s, const int32_t* idx, const float* cos_sim,
                     const locmoe_capacity_rule_t& rule, float* delta_e, float* theta_e,
                     locmoe_capacity_t* cap_dev, void* ws, cudaStream_t st) {
     uint32_t* gmin = static_cast<uint32_t*>(ws);
+    if (capacity_cluster_eligible(s)) {
+        capacity_cluster_kernel<<<kCapCS, kCapThreads, (size_t)s.E * sizeof(uint32_t), st>>>(
+            idx, cos_sim, gmin, s.T, s.E, s.H, s.n_nodes * s.dev_per_node, rule, delta_e, theta_e, cap_dev);
+        return check_launch();
+    }
     if (cudaMemsetAsync(gmin, 0xff, (size_t)s.E * sizeof(uint32_t), st) != cudaSuccess) {
         cudaGetLastError();
         return LOCMOE_ERR_CUDA;

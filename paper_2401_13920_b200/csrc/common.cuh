@@ -34,10 +34,12 @@ struct RoutePlan {
     int tile;         // tokens per tile
     int rounds;       // 32-token rounds per warp per tile
     int ntiles;
-    size_t off_keys[2], off_toks[2], off_hist, off_keystart, total;
+    int launches;     // kernel launches of one route call
+    size_t off_keys[2], off_toks[2], off_hist[4], off_keystart, total;
 };
 int plan_route(const locmoe_shape_t& s, RoutePlan* p);
 size_t capacity_ws_bytes(const locmoe_shape_t& s);
+bool capacity_cluster_eligible(const locmoe_shape_t& s);
 
 int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src, const locmoe_capacity_t* cap_dev,
                  int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,

@@ -3,17 +3,21 @@
 // pos[t] -- the number of earlier tokens with the same (source device, expert)
 // pair -- is the rank of t inside its key class in token order.  It is
 // obtained with a stable least-significant-digit radix sort of the keys
-// key = src * E + expert: per pass a per-tile digit histogram, one exclusive
-// scan over (digit, tile), and a stable in-tile ranking that uses warp match
-// operations and per-warp digit counters.  A token's final sorted position
-// minus the start of its key class is pos.  Every step is integer and order
-// independent, so the result is a function of the inputs only; no kernel waits
-// on another CTA.
+// key = src * E + expert.  A token's final sorted position minus the start of
+// its key class is pos.  Every step is integer and order independent, so the
+// result is a function of the inputs only; no kernel waits on another CTA.
 //
-// Launch sequence (P radix passes, P = 1 for up to 1024 keys, 2 up to 65536):
-//   init -> [hist_p -> scan_p -> scatter_p] for p = 0..P-1
-// scan_0 also turns the per-key demand counts into key-class starts and the
-// count matrices (kept, send_counts, load, locality tallies).
+// Launch sequence for P radix passes (P = 1 up to 1024 keys, 2 up to 65536):
+//   init      inv = -1, accumulators and later-pass histograms = 0
+//   hist0     per-tile histogram of digit 0, per-key demand counts
+//   scatter_p every CTA derives its own (digit, tile) offsets from the
+//             histogram matrix (no separate scan launch), ranks its tile stably
+//             with warp match operations and per-warp digit counters, moves
+//             (key, token) to the sorted position and adds to the next pass's
+//             histogram with integer atomics; the last pass emits the outputs.
+//   extras    key-class starts and count matrices (kept, send_counts, load,
+//             locality tallies): extra CTAs of scatter_0 when P > 1, a launch
+//             of their own before the only scatter when P = 1.
 #include "common.cuh"
 
 namespace locmoe {
@@ -23,7 +27,7 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxRounds = 16;
-constexpr int kScanThreads = 1024;
+constexpr int kMaxPasses = 4;
 
 struct RouteArgs {
     const int32_t* idx;
@@ -36,29 +40,18 @@ struct RouteArgs {
     int32_t* status;
     int T, E, N, Dn, D, Ed, K, layout;
     long long rows;
-    int tile, rounds, ntiles;
+    int tile, rounds, ntiles, passes;
+    int bits[kMaxPasses];
     uint32_t* keys[2];
     int32_t* toks[2];
-    int32_t* hist;       // [nbins][ntiles], digit major
-    int32_t* keystart;   // [K]
-    int32_t* n_valid;    // items that survive pass 0
+    int32_t* hist[kMaxPasses];  // [1 << bits[p]][ntiles], digit major
+    int32_t* keystart;          // [K]
 };
 
 __device__ __forceinline__ int dest_rank(int a, int b, int N, int Dn) {
     int dn = b / Dn - a / Dn; if (dn < 0) dn += N;
     int dl = b % Dn - a % Dn; if (dl < 0) dl += Dn;
     return dn * Dn + dl;
-}
-
-__global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a) {
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    for (long long i = i0; i < a.rows; i += stride) a.inv[i] = -1;
-    for (long long i = i0; i < a.K; i += stride) a.counts[i] = 0;
-    for (long long i = i0; i < (long long)a.D * a.D; i += stride) a.send_counts[i] = 0;
-    for (long long i = i0; i < a.E; i += stride) a.load[i] = 0;
-    if (i0 < 6) a.locality[i0] = 0ull;
-    if (i0 == 0) *a.status = 0;
 }
 
 // Key of token t, or -1 with a warning bit when the token cannot be routed.
@@ -69,40 +62,69 @@ __device__ __forceinline__ int token_key(const RouteArgs& a, int t, int* warn) {
     return s * a.E + e;
 }
 
-template <bool FIRST>
-__global__ void __launch_bounds__(kThreads) route_hist_kernel(const RouteArgs a, int pass, int shift, int nbins) {
-    extern __shared__ int sh[];
-    for (int d = threadIdx.x; d < nbins; d += blockDim.x) sh[d] = 0;
-    __syncthreads();
-    const int n = FIRST ? a.T : *a.n_valid;
-    const int base = blockIdx.x * a.tile;
-    const uint32_t mask = (uint32_t)nbins - 1u;
-    const uint32_t* kin = a.keys[(pass + 1) & 1];
-    int warn = 0;
-    for (int o = threadIdx.x; o < a.tile; o += blockDim.x) {
-        int j = base + o;
-        if (j >= n) break;
-        int key;
-        if (FIRST) {
-            key = token_key(a, j, &warn);
-            if (key < 0) continue;
-            atomicAdd(&a.counts[key], 1);
-        } else {
-            key = (int)kin[j];
-        }
-        atomicAdd(&sh[((uint32_t)key >> shift) & mask], 1);
-    }
-    if (FIRST && warn) atomicOr(a.status, warn);
-    __syncthreads();
-    for (int d = threadIdx.x; d < nbins; d += blockDim.x) a.hist[(size_t)d * a.ntiles + blockIdx.x] = sh[d];
+// Row base (in units of C_alloc rows) of key k = s * E + e in the chosen layout.
+__device__ __forceinline__ long long route_row_base(const RouteArgs& a, int k) {
+    const int s = k / a.E, e = k - s * a.E;
+    const int b = e / a.Ed, el = e - b * a.Ed;
+    if (a.layout == LOCMOE_LAYOUT_SEND) return ((long long)s * a.D + dest_rank(s, b, a.N, a.Dn)) * a.Ed + el;
+    return (long long)e * a.D + dest_rank(b, s, a.N, a.Dn);
 }
 
-// In-place exclusive scan of data[0..n) by one CTA; returns the total in *total (if given).
-__device__ void block_exclusive_scan(const int32_t* in, int32_t* out, int n, int32_t* total) {
-    __shared__ int warp_sums[kScanThreads / 32];
-    __shared__ int carry_all;
+// Final outputs of one token: `dest` is its position in the stable sort by key.
+__device__ __forceinline__ void route_emit(const RouteArgs& a, int k, int t, int dest, int C) {
+    const int p = dest - a.keystart[k];
+    const bool dropped = p >= C;
+    a.pos[t] = p;
+    a.drop[t] = dropped ? 1 : 0;
+    int row = -1;
+    if (!dropped) {
+        row = (int)(route_row_base(a, k) * a.C_alloc + p);
+        a.inv[row] = t;
+    }
+    a.slot[t] = row;
+}
+
+__global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    for (long long i = i0; i < a.rows; i += stride) a.inv[i] = -1;
+    for (long long i = i0; i < a.K; i += stride) a.counts[i] = 0;
+    for (long long i = i0; i < (long long)a.D * a.D; i += stride) a.send_counts[i] = 0;
+    for (long long i = i0; i < a.E; i += stride) a.load[i] = 0;
+    for (int p = 1; p < a.passes; ++p) {
+        const long long n = ((long long)a.ntiles) << a.bits[p];
+        for (long long i = i0; i < n; i += stride) a.hist[p][i] = 0;
+    }
+    if (i0 < 6) a.locality[i0] = 0ull;
+    if (i0 == 0) *a.status = 0;
+}
+
+__global__ void __launch_bounds__(kThreads) route_hist0_kernel(const RouteArgs a) {
+    extern __shared__ int sh[];
+    const int nbins = 1 << a.bits[0];
+    for (int d = threadIdx.x; d < nbins; d += blockDim.x) sh[d] = 0;
+    __syncthreads();
+    const int base = blockIdx.x * a.tile;
+    const uint32_t mask = (uint32_t)nbins - 1u;
+    int warn = 0;
+    for (int o = threadIdx.x; o < a.tile; o += blockDim.x) {
+        const int t = base + o;
+        if (t >= a.T) break;
+        const int key = token_key(a, t, &warn);
+        if (key < 0) { a.pos[t] = -1; a.slot[t] = -1; a.drop[t] = 1; continue; }
+        atomicAdd(&a.counts[key], 1);
+        atomicAdd(&sh[(uint32_t)key & mask], 1);
+    }
+    if (warn) atomicOr(a.status, warn);
+    __syncthreads();
+    for (int d = threadIdx.x; d < nbins; d += blockDim.x) a.hist[0][(size_t)d * a.ntiles + blockIdx.x] = sh[d];
+}
+
+// Exclusive scan of in[0..n) into out[0..n) by one CTA of kThreads threads (in == out allowed).
+__device__ void block_exclusive_scan(const int32_t* in, int32_t* out, int n) {
+    __shared__ int warp_sums[kWarps];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    const int chunk = (n + kScanThreads - 1) / kScanThreads;
+    const int chunk = (n + kThreads - 1) / kThreads;
     const int lo = min(tid * chunk, n), hi = min(lo + chunk, n);
     int s = 0;
     for (int i = lo; i < hi; ++i) s += in[i];
@@ -114,46 +136,32 @@ __device__ void block_exclusive_scan(const int32_t* in, int32_t* out, int n, int
     }
     if (lane == 31) warp_sums[w] = incl;
     __syncthreads();
-    if (w == 0) {
-        int v = warp_sums[lane];
-        int iv = v;
+    int wbase = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int u = __shfl_up_sync(0xffffffffu, iv, o);
-            if (lane >= o) iv += u;
-        }
-        warp_sums[lane] = iv - v;
-        if (lane == 31) carry_all = iv;
-    }
-    __syncthreads();
-    int run = warp_sums[w] + incl - s;
+    for (int ww = 0; ww < kWarps; ++ww) if (ww < w) wbase += warp_sums[ww];
+    int run = wbase + incl - s;
     for (int i = lo; i < hi; ++i) { int v = in[i]; out[i] = run; run += v; }
-    if (total && tid == 0) *total = carry_all;
+    __syncthreads();
 }
 
-// Block 0: offsets for this pass.  With with_stats: block 1 builds the key-class
-// starts, blocks >= 2 the count matrices.
-__global__ void __launch_bounds__(kScanThreads) route_scan_kernel(const RouteArgs a, int nbins, int with_stats) {
-    if (blockIdx.x == 0) {
-        block_exclusive_scan(a.hist, a.hist, nbins * a.ntiles, with_stats ? a.n_valid : nullptr);
-        return;
-    }
-    if (blockIdx.x == 1) {
-        block_exclusive_scan(a.counts, a.keystart, a.K, nullptr);
+// Extra CTAs (index x = 0, 1, ... of nx): x = 0 builds the key-class starts, the others the count matrices.
+__device__ void route_extras(const RouteArgs& a, int x, int nx) {
+    if (x == 0) {
+        block_exclusive_scan(a.counts, a.keystart, a.K);
         return;
     }
     int C = a.cap->C_local;
     if (C > a.C_alloc) {
         C = a.C_alloc;
-        if (blockIdx.x == 2 && threadIdx.x == 0) atomicOr(a.status, LOCMOE_WARN_CLAMPED);
+        if (x == 1 && threadIdx.x == 0) atomicOr(a.status, LOCMOE_WARN_CLAMPED);
     }
     unsigned long long raw0 = 0, raw1 = 0, raw2 = 0, kp0 = 0, kp1 = 0, kp2 = 0;
-    for (int k = (blockIdx.x - 2) * blockDim.x + threadIdx.x; k < a.K; k += (gridDim.x - 2) * blockDim.x) {
-        int c = a.counts[k];
-        int kp = c < C ? c : C;
+    for (int k = (x - 1) * kThreads + threadIdx.x; k < a.K; k += (nx - 1) * kThreads) {
+        const int c = a.counts[k];
+        const int kp = c < C ? c : C;
         a.kept[k] = kp;
         if (c == 0) continue;
-        int s = k / a.E, e = k - s * a.E, b = e / a.Ed;
+        const int s = k / a.E, e = k - s * a.E, b = e / a.Ed;
         if (b == s) { raw0 += c; kp0 += kp; }
         else if (b / a.Dn == s / a.Dn) { raw1 += c; kp1 += kp; }
         else { raw2 += c; kp2 += kp; }
@@ -176,20 +184,77 @@ __global__ void __launch_bounds__(kScanThreads) route_scan_kernel(const RouteArg
     }
 }
 
+__global__ void __launch_bounds__(kThreads) route_extras_kernel(const RouteArgs a) {
+    route_extras(a, blockIdx.x, gridDim.x);
+}
+
+// One radix pass over one tile per CTA; CTAs beyond ntiles run the extras.
 template <bool FIRST, bool LAST>
-__global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs a, int pass, int shift, int nbins) {
-    extern __shared__ int cnt[];  // [kWarps][nbins]
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    for (int i = threadIdx.x; i < kWarps * nbins; i += blockDim.x) cnt[i] = 0;
+__global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs a, int pass, int shift) {
+    if ((int)blockIdx.x >= a.ntiles) {
+        route_extras(a, blockIdx.x - a.ntiles, gridDim.x - a.ntiles);
+        return;
+    }
+    extern __shared__ int sm[];
+    const int nbins = 1 << a.bits[pass];
+    int* cnt = sm;                       // [kWarps][nbins] per-warp digit counters, then running offsets
+    int* pre = sm + kWarps * nbins;      // [nbins] tokens of the digit in earlier tiles
+    int* tot = pre + nbins;              // [nbins] tokens of the digit in all tiles, then digit bases
+    __shared__ int wsum[kWarps];
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int tileid = blockIdx.x;
+    for (int i = tid; i < kWarps * nbins; i += kThreads) cnt[i] = 0;
+
+    // ---- this tile's offsets from the (digit, tile) histogram matrix: one warp per digit row ----
+    const int32_t* H = a.hist[pass];
+    for (int d = w; d < nbins; d += kWarps) {
+        const int32_t* row = H + (size_t)d * a.ntiles;
+        int before = 0, all = 0;
+        for (int j = lane; j < a.ntiles; j += 32) {
+            const int v = row[j];
+            all += v;
+            if (j < tileid) before += v;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            before += __shfl_xor_sync(0xffffffffu, before, o);
+            all += __shfl_xor_sync(0xffffffffu, all, o);
+        }
+        if (lane == 0) { pre[d] = before; tot[d] = all; }
+    }
+    __syncthreads();
+    // exclusive scan of tot[] over the digits -> digit bases; the grand total is the number of valid items
+    int n_valid;
+    {
+        const int chunk = (nbins + kThreads - 1) / kThreads;
+        const int lo = min(tid * chunk, nbins), hi = min(lo + chunk, nbins);
+        int s = 0;
+        for (int i = lo; i < hi; ++i) s += tot[i];
+        int incl = s;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) wsum[w] = incl;
+        __syncthreads();
+        int wb = 0, total = 0;
+#pragma unroll
+        for (int ww = 0; ww < kWarps; ++ww) { if (ww < w) wb += wsum[ww]; total += wsum[ww]; }
+        n_valid = total;
+        int run = wb + incl - s;
+        for (int i = lo; i < hi; ++i) { int v = tot[i]; tot[i] = run; run += v; }
+    }
     __syncthreads();
 
-    const int n = FIRST ? a.T : *a.n_valid;
+    // ---- stable rank inside the tile ----
+    const int n = FIRST ? a.T : n_valid;
     const uint32_t mask = (uint32_t)nbins - 1u;
     const uint32_t* kin = a.keys[(pass + 1) & 1];
     const int32_t* tin = a.toks[(pass + 1) & 1];
     uint32_t* kout = a.keys[pass & 1];
     int32_t* tout = a.toks[pass & 1];
-    const int wbase = blockIdx.x * a.tile + w * a.rounds * 32;
+    const int wbase = tileid * a.tile + w * a.rounds * 32;
     const uint32_t lt = (1u << lane) - 1u;
     int* mycnt = cnt + w * nbins;
 
@@ -198,18 +263,16 @@ __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs
     for (int r = 0; r < kMaxRounds; ++r) {
         key[r] = -1; tok[r] = -1; rank[r] = 0;
         if (r < a.rounds) {
-            int j = wbase + r * 32 + lane;
+            const int j = wbase + r * 32 + lane;
             if (j < n) {
-                if (FIRST) {
-                    int warn = 0;
-                    tok[r] = j;
-                    key[r] = token_key(a, j, &warn);
-                    if (key[r] < 0) { a.pos[j] = -1; a.slot[j] = -1; a.drop[j] = 1; }
-                } else {
-                    key[r] = (int)kin[j];
-                    tok[r] = tin[j];
-                }
+                if (FIRST) { int warn = 0; tok[r] = j; key[r] = token_key(a, j, &warn); }
+                else { key[r] = (int)kin[j]; tok[r] = tin[j]; }
             }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) {
+        if (r < a.rounds) {
             const bool valid = key[r] >= 0;
             const uint32_t d = valid ? (((uint32_t)key[r] >> shift) & mask) : 0xffffffffu;
             const uint32_t peers = __match_any_sync(0xffffffffu, d);
@@ -224,12 +287,12 @@ __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs
         }
     }
     __syncthreads();
-    // counters -> starting offsets: global (digit, tile) offset plus the earlier warps of this tile
-    for (int d = threadIdx.x; d < nbins; d += blockDim.x) {
-        int run = a.hist[(size_t)d * a.ntiles + blockIdx.x];
+    // counters -> starting offsets: digit base + earlier tiles + earlier warps of this tile
+    for (int d = tid; d < nbins; d += kThreads) {
+        int run = tot[d] + pre[d];
 #pragma unroll
         for (int ww = 0; ww < kWarps; ++ww) {
-            int c = cnt[ww * nbins + d];
+            const int c = cnt[ww * nbins + d];
             cnt[ww * nbins + d] = run;
             run += c;
         }
@@ -238,33 +301,20 @@ __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs
 
     int C = 0;
     if (LAST) { C = a.cap->C_local; if (C > a.C_alloc) C = a.C_alloc; }
+    const int nshift = shift + a.bits[pass];
+    const uint32_t nmask = LAST ? 0u : (uint32_t)(1 << a.bits[LAST ? pass : pass + 1]) - 1u;
+    int32_t* Hn = LAST ? nullptr : a.hist[LAST ? pass : pass + 1];
 #pragma unroll
     for (int r = 0; r < kMaxRounds; ++r) {
         if (r < a.rounds && key[r] >= 0) {
             const uint32_t d = ((uint32_t)key[r] >> shift) & mask;
             const int dest = mycnt[d] + rank[r];
-            if (!LAST) {
+            if (LAST) {
+                route_emit(a, key[r], tok[r], dest, C);
+            } else {
                 kout[dest] = (uint32_t)key[r];
                 tout[dest] = tok[r];
-            } else {
-                const int k = key[r], t = tok[r];
-                const int p = dest - a.keystart[k];
-                const bool dropped = p >= C;
-                a.pos[t] = p;
-                a.drop[t] = dropped ? 1 : 0;
-                int row = -1;
-                if (!dropped) {
-                    const int s = k / a.E, e = k - s * a.E;
-                    const int b = e / a.Ed, el = e - b * a.Ed;
-                    long long rr;
-                    if (a.layout == LOCMOE_LAYOUT_SEND)
-                        rr = (((long long)s * a.D + dest_rank(s, b, a.N, a.Dn)) * a.Ed + el) * a.C_alloc + p;
-                    else
-                        rr = ((long long)e * a.D + dest_rank(b, s, a.N, a.Dn)) * a.C_alloc + p;
-                    row = (int)rr;
-                    a.inv[row] = t;
-                }
-                a.slot[t] = row;
+                atomicAdd(&Hn[(size_t)(((uint32_t)key[r] >> nshift) & nmask) * a.ntiles + dest / a.tile], 1);
             }
         }
     }
@@ -294,15 +344,18 @@ int plan_route(const locmoe_shape_t& s, RoutePlan* p) {
     p->rounds = rounds;
     p->tile = kWarps * rounds * 32;
     p->ntiles = (int)(((long long)s.T + p->tile - 1) / p->tile);
-    int maxbins = 1 << p->bits[0];
     size_t off = 0;
     for (int i = 0; i < 2; ++i) {
         p->off_keys[i] = off; off += p->passes > 1 ? align256((size_t)s.T * 4) : 0;
         p->off_toks[i] = off; off += p->passes > 1 ? align256((size_t)s.T * 4) : 0;
     }
-    p->off_hist = off; off += align256((size_t)maxbins * p->ntiles * 4 + 4);
+    for (int i = 0; i < 4; ++i) {
+        p->off_hist[i] = off;
+        if (i < p->passes) off += align256(((size_t)p->ntiles << p->bits[i]) * 4);
+    }
     p->off_keystart = off; off += align256((size_t)K * 4);
     p->total = off;
+    p->launches = 2 + p->passes + (p->passes == 1 ? 1 : 0);
     return LOCMOE_OK;
 }
 
@@ -322,14 +375,16 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
     a.T = s.T; a.E = s.E; a.N = s.n_nodes; a.Dn = s.dev_per_node; a.D = a.N * a.Dn; a.Ed = a.E / a.D;
     a.K = a.D * a.E; a.layout = s.layout;
     a.rows = (long long)a.K * C_alloc;
-    a.tile = p.tile; a.rounds = p.rounds; a.ntiles = p.ntiles;
+    a.tile = p.tile; a.rounds = p.rounds; a.ntiles = p.ntiles; a.passes = p.passes;
     char* w = static_cast<char*>(ws);
     for (int i = 0; i < 2; ++i) {
         a.keys[i] = reinterpret_cast<uint32_t*>(w + p.off_keys[i]);
         a.toks[i] = reinterpret_cast<int32_t*>(w + p.off_toks[i]);
     }
-    a.hist = reinterpret_cast<int32_t*>(w + p.off_hist);
-    a.n_valid = a.hist + (size_t)(1 << p.bits[0]) * p.ntiles;
+    for (int i = 0; i < kMaxPasses; ++i) {
+        a.bits[i] = p.bits[i];
+        a.hist[i] = reinterpret_cast<int32_t*>(w + p.off_hist[i]);
+    }
     a.keystart = reinterpret_cast<int32_t*>(w + p.off_keystart);
 
     long long init_items = a.rows > a.K ? a.rows : a.K;
@@ -339,22 +394,25 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
     route_init_kernel<<<init_blocks, kThreads, 0, st>>>(a);
     if ((rc = check_launch())) return rc;
 
-    int stats_blocks = (a.K + kScanThreads - 1) / kScanThreads;
-    if (stats_blocks > 64) stats_blocks = 64;
+    route_hist0_kernel<<<p.ntiles, kThreads, sizeof(int) << p.bits[0], st>>>(a);
+    if ((rc = check_launch())) return rc;
+
+    int extras = 1 + (a.K + kThreads * 4 - 1) / (kThreads * 4);
+    if (extras > 33) extras = 33;
+    if (extras < 2) extras = 2;
+    if (p.passes == 1) {
+        route_extras_kernel<<<extras, kThreads, 0, st>>>(a);
+        if ((rc = check_launch())) return rc;
+    }
     int shift = 0;
     for (int pass = 0; pass < p.passes; ++pass) {
-        const int nbins = 1 << p.bits[pass];
         const bool first = pass == 0, last = pass == p.passes - 1;
-        if (first) route_hist_kernel<true><<<p.ntiles, kThreads, nbins * sizeof(int), st>>>(a, pass, shift, nbins);
-        else route_hist_kernel<false><<<p.ntiles, kThreads, nbins * sizeof(int), st>>>(a, pass, shift, nbins);
-        if ((rc = check_launch())) return rc;
-        route_scan_kernel<<<first ? 2 + stats_blocks : 1, kScanThreads, 0, st>>>(a, nbins, first ? 1 : 0);
-        if ((rc = check_launch())) return rc;
-        const size_t sm = (size_t)kWarps * nbins * sizeof(int);
-        if (first && last) route_scatter_kernel<true, true><<<p.ntiles, kThreads, sm, st>>>(a, pass, shift, nbins);
-        else if (first) route_scatter_kernel<true, false><<<p.ntiles, kThreads, sm, st>>>(a, pass, shift, nbins);
-        else if (last) route_scatter_kernel<false, true><<<p.ntiles, kThreads, sm, st>>>(a, pass, shift, nbins);
-        else route_scatter_kernel<false, false><<<p.ntiles, kThreads, sm, st>>>(a, pass, shift, nbins);
+        const size_t smb = ((size_t)(kWarps + 2) * sizeof(int)) << p.bits[pass];
+        const int grid = p.ntiles + ((first && !last) ? extras : 0);
+        if (first && last) route_scatter_kernel<true, true><<<grid, kThreads, smb, st>>>(a, pass, shift);
+        else if (first) route_scatter_kernel<true, false><<<grid, kThreads, smb, st>>>(a, pass, shift);
+        else if (last) route_scatter_kernel<false, true><<<grid, kThreads, smb, st>>>(a, pass, shift);
+        else route_scatter_kernel<false, false><<<grid, kThreads, smb, st>>>(a, pass, shift);
         if ((rc = check_launch())) return rc;
         shift += p.bits[pass];
     }

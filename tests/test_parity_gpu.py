@@ -64,6 +64,28 @@ def test_config4_full_size_sampled(P):
     assert rep["C_local"] == 16 and 0.05 < rep["drop_frac"] < 0.15
 
 
+# ---- the multi-kernel capacity path (default only beyond 2M tokens or 8192 experts) at small sizes ----
+
+@pytest.fixture
+def grid_path(monkeypatch):
+    monkeypatch.setenv("LOCMOE_PATH", "grid")
+
+
+@pytest.mark.parametrize("cfg,T", [(1, 4096), (2, 70001), (3, 8229), (4, 5003), (5, 7001)])
+def test_grid_path_configs(P, grid_path, cfg, T):
+    rep = P.run_staged(P.W.CONFIGS[cfg].scaled(T), 1.0, full=True, y_random=cfg == 4)
+    assert rep["status"] == 0
+
+
+@pytest.mark.parametrize("kw", [
+    dict(T=1, H=64, E=4, n_nodes=1, dev_per_node=2),
+    dict(T=513, H=1024, E=512, n_nodes=4, dev_per_node=8),
+    dict(T=4097, H=2048, E=2048, n_nodes=8, dev_per_node=8),
+])
+def test_grid_path_shapes(P, grid_path, kw):
+    P.run_staged(_wl(P, **kw), 1.0, layout=1, full=True)
+
+
 # ---- edge cases and degenerate inputs ----
 
 @pytest.mark.parametrize("kw", [
