@@ -185,6 +185,12 @@ int locmoe_combine(const locmoe_shape_t *shape, int32_t C_alloc, const void *y, 
  * has no counterpart. */
 int locmoe_launch_counts(const locmoe_shape_t *shape, int32_t counts[5]);
 
+/* Device-side diagnostics of this library on the current device, copied to host
+ * memory after waiting for the stream: bit 0 is set if a kernel gave up a
+ * bounded wait for one of its own asynchronous copies (its output is then
+ * incomplete).  0 in normal operation.  The paper has no counterpart. */
+int locmoe_device_flags(int32_t *flags_host, void *stream);
+
 /* Text for a return code of this library (host string, never NULL). */
 const char *locmoe_status_string(int code);
 

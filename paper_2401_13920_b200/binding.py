@@ -24,7 +24,7 @@ FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
     "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_read", "locmoe_route",
-    "locmoe_dispatch", "locmoe_combine", "locmoe_launch_counts", "locmoe_status_string",
+    "locmoe_dispatch", "locmoe_combine", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
 
@@ -69,6 +69,7 @@ def _load() -> C.CDLL:
     lib.locmoe_dispatch.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, i32, vp]
     lib.locmoe_combine.argtypes = [C.POINTER(Shape), i32, vp, i32, vp, vp, vp, i32, vp]
     lib.locmoe_launch_counts.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32 * 5)]
+    lib.locmoe_device_flags.argtypes = [C.POINTER(C.c_int32), vp]
     lib.locmoe_status_string.argtypes = [C.c_int]
     lib.locmoe_status_string.restype = C.c_char_p
     for name in EXPORTS[:-1]:
@@ -139,6 +140,12 @@ def locmoe_launch_counts(shape: Shape) -> dict:
     out = (C.c_int32 * 5)()
     _check("locmoe_launch_counts", _lib.locmoe_launch_counts(C.byref(shape), C.byref(out)))
     return dict(zip(("gate", "capacity", "route", "dispatch", "combine"), list(out)))
+
+
+def locmoe_device_flags(stream=None) -> int:
+    out = C.c_int32(0)
+    _check("locmoe_device_flags", _lib.locmoe_device_flags(C.byref(out), _stream(stream)))
+    return out.value
 
 
 def locmoe_gate(shape: Shape, x, eps, idx, gate_w, cos_sim, probs=None, stream=None) -> int:

@@ -152,6 +152,14 @@ int locmoe_launch_counts(const locmoe_shape_t* shape, int32_t counts[5]) {
     return LOCMOE_OK;
 }
 
+int locmoe_device_flags(int32_t* flags_host, void* stream) {
+    if (!flags_host) return LOCMOE_ERR_NULL;
+    int v = 0;
+    int rc = read_device_flags(&v, static_cast<cudaStream_t>(stream));
+    *flags_host = v;
+    return rc;
+}
+
 const char* locmoe_status_string(int code) {
     switch (code) {
         case LOCMOE_OK: return "ok";

@@ -205,22 +205,62 @@ __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs
     const int tileid = blockIdx.x;
     for (int i = tid; i < kWarps * nbins; i += kThreads) cnt[i] = 0;
 
+    // ---- this tile's items, loaded first so that their latency overlaps the offset computation ----
+    const uint32_t mask = (uint32_t)nbins - 1u;
+    const uint32_t* kin = a.keys[(pass + 1) & 1];
+    const int32_t* tin = a.toks[(pass + 1) & 1];
+    uint32_t* kout = a.keys[pass & 1];
+    int32_t* tout = a.toks[pass & 1];
+    const int wbase = tileid * a.tile + w * a.rounds * 32;
+    const uint32_t lt = (1u << lane) - 1u;
+    int* mycnt = cnt + w * nbins;
+    int key[kMaxRounds], tok[kMaxRounds], rank[kMaxRounds];
+#pragma unroll
+    for (int r = 0; r < kMaxRounds; ++r) {
+        key[r] = -1; tok[r] = -1; rank[r] = 0;
+        if (r < a.rounds) {
+            const int j = wbase + r * 32 + lane;
+            if (j < a.T) {
+                if (FIRST) { int warn = 0; tok[r] = j; key[r] = token_key(a, j, &warn); }
+                else { key[r] = (int)kin[j]; tok[r] = tin[j]; }
+            }
+        }
+    }
+
     // ---- this tile's offsets from the (digit, tile) histogram matrix: one warp per digit row ----
+    // (kRB rows per batch so that their loads are all in flight together: the matrix lives in L2)
     const int32_t* H = a.hist[pass];
-    for (int d = w; d < nbins; d += kWarps) {
-        const int32_t* row = H + (size_t)d * a.ntiles;
-        int before = 0, all = 0;
+    constexpr int kRB = 8;
+    for (int d0 = w; d0 < nbins; d0 += kWarps * kRB) {
+        int before[kRB], all[kRB];
+#pragma unroll
+        for (int q = 0; q < kRB; ++q) { before[q] = 0; all[q] = 0; }
         for (int j = lane; j < a.ntiles; j += 32) {
-            const int v = row[j];
-            all += v;
-            if (j < tileid) before += v;
+#pragma unroll
+            for (int q = 0; q < kRB; ++q) {
+                const int d = d0 + q * kWarps;
+                if (d < nbins) {
+                    const int v = H[(size_t)d * a.ntiles + j];
+                    all[q] += v;
+                    if (j < tileid) before[q] += v;
+                }
+            }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
-            before += __shfl_xor_sync(0xffffffffu, before, o);
-            all += __shfl_xor_sync(0xffffffffu, all, o);
+#pragma unroll
+            for (int q = 0; q < kRB; ++q) {
+                before[q] += __shfl_xor_sync(0xffffffffu, before[q], o);
+                all[q] += __shfl_xor_sync(0xffffffffu, all[q], o);
+            }
         }
-        if (lane == 0) { pre[d] = before; tot[d] = all; }
+        if (lane == 0) {
+#pragma unroll
+            for (int q = 0; q < kRB; ++q) {
+                const int d = d0 + q * kWarps;
+                if (d < nbins) { pre[d] = before[q]; tot[d] = all[q]; }
+            }
+        }
     }
     __syncthreads();
     // exclusive scan of tot[] over the digits -> digit bases; the grand total is the number of valid items
@@ -248,28 +288,9 @@ __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs
     __syncthreads();
 
     // ---- stable rank inside the tile ----
-    const int n = FIRST ? a.T : n_valid;
-    const uint32_t mask = (uint32_t)nbins - 1u;
-    const uint32_t* kin = a.keys[(pass + 1) & 1];
-    const int32_t* tin = a.toks[(pass + 1) & 1];
-    uint32_t* kout = a.keys[pass & 1];
-    int32_t* tout = a.toks[pass & 1];
-    const int wbase = tileid * a.tile + w * a.rounds * 32;
-    const uint32_t lt = (1u << lane) - 1u;
-    int* mycnt = cnt + w * nbins;
-
-    int key[kMaxRounds], tok[kMaxRounds], rank[kMaxRounds];
 #pragma unroll
-    for (int r = 0; r < kMaxRounds; ++r) {
-        key[r] = -1; tok[r] = -1; rank[r] = 0;
-        if (r < a.rounds) {
-            const int j = wbase + r * 32 + lane;
-            if (j < n) {
-                if (FIRST) { int warn = 0; tok[r] = j; key[r] = token_key(a, j, &warn); }
-                else { key[r] = (int)kin[j]; tok[r] = tin[j]; }
-            }
-        }
-    }
+    for (int r = 0; r < kMaxRounds; ++r)
+        if (!FIRST && wbase + r * 32 + lane >= n_valid) key[r] = -1;   // beyond the valid items: stale buffer contents
 #pragma unroll
     for (int r = 0; r < kMaxRounds; ++r) {
         if (r < a.rounds) {

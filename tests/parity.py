@@ -181,6 +181,7 @@ def run_staged(w: W.Workload, capacity_factor=1.0, min_mult=None, layout=B.LAYOU
         y = W.make_expert_out(w, st.rows, dev, "f32" if w.y_dtype == "f32" else w.dtype)
     B.router_forward(st, x, src, y=y, eps=eps_dev)
     torch.cuda.synchronize()
+    assert B.locmoe_device_flags() == 0, "a kernel reported a failed bounded wait"
 
     rep = {"workload": w.name, "T": w.T, "C_alloc": C_alloc}
     gi = check_gate(x, shape, st, eps_dev)

@@ -86,6 +86,14 @@ def test_grid_path_shapes(P, grid_path, kw):
     P.run_staged(_wl(P, **kw), 1.0, layout=1, full=True)
 
 
+def test_bulk_copy_dispatch_variant(P, monkeypatch):
+    # the TMA (cp.async.bulk) dispatch kernel: whole rows, split rows (> 16 KB), zero rows
+    monkeypatch.setenv("LOCMOE_DISPATCH", "tma")
+    P.run_staged(P.W.CONFIGS[2].scaled(6000), 1.25, full=True)
+    P.run_staged(_wl(P, T=300, H=16384, E=8, n_nodes=2, dev_per_node=2, dtype="f32"), 2.0, full=True)
+    P.run_staged(P.W.CONFIGS[1], 1.0, layout=1, full=True)
+
+
 # ---- edge cases and degenerate inputs ----
 
 @pytest.mark.parametrize("kw", [
