@@ -50,7 +50,8 @@ enum {
     LOCMOE_ERR_DTYPE = -3,     /* unknown dtype / layout / bound form                  */
     LOCMOE_ERR_ALIGN = -4,     /* a pointer lacks the stated alignment                 */
     LOCMOE_ERR_WORKSPACE = -5, /* ws too small or misaligned                           */
-    LOCMOE_ERR_CUDA = -6       /* a CUDA call failed (launch error is cleared)         */
+    LOCMOE_ERR_CUDA = -6,      /* a CUDA call failed (launch error is cleared)         */
+    LOCMOE_ERR_TOO_LARGE = -7  /* size beyond the built-in scratch of a no-allocation call */
 };
 enum {                         /* bits of the device status word                       */
     LOCMOE_WARN_CLAMPED = 1,   /* C_local > C_alloc: capacity clamped to C_alloc       */
@@ -131,6 +132,38 @@ int locmoe_gate(const locmoe_shape_t *shape, const void *x, const float *eps,
 int locmoe_capacity(const locmoe_shape_t *shape, const int32_t *idx, const float *cos_sim,
                     const locmoe_capacity_rule_t *rule, float *delta_e, float *theta_e,
                     locmoe_capacity_t *cap_dev, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * The same computation as locmoe_capacity, for callers that cannot supply a
+ * workspace.  (This entry point has no counterpart in the paper; it exists for
+ * deployment reasons only.)
+ *
+ * Meant for host code that has no device allocator to turn to: a plug-in inside
+ * a serving process that has already claimed the whole HBM for its own pools,
+ * so that a cudaMalloc would fail or eat into them, or a C caller that is handed
+ * nothing but the input and output buffers of an operator.  The scratch that
+ * locmoe_capacity takes from `ws` is here a fixed 256 KiB array inside the
+ * library's device image; the call itself performs no cudaMalloc / cudaFree and
+ * uses no allocating library routine.  Inputs and outputs are the caller's, as
+ * in locmoe_capacity, with the same meaning, layout and results.
+ *
+ * Limits and rules that follow from the built-in array:
+ *   - at most 8192 experts; a larger shape->E returns LOCMOE_ERR_TOO_LARGE
+ *     before anything is launched;
+ *   - every GPU on which the library is used holds the 256 KiB until the
+ *     process exits;
+ *   - all calls on one device share the array and it keeps whatever the last
+ *     call left in it.  Each call rewrites all it reads, so calls that follow
+ *     one another on a stream are independent, but two calls that can overlap
+ *     on the GPU (different streams, no dependency) race on it and must be
+ *     ordered by the caller;
+ *   - the first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current) and caches it; make
+ *     that first call outside of, and before, any stream capture.
+ */
+int locmoe_capacity_noalloc(const locmoe_shape_t *shape, const int32_t *idx, const float *cos_sim,
+                            const locmoe_capacity_rule_t *rule, float *delta_e, float *theta_e,
+                            locmoe_capacity_t *cap_dev, void *stream);
 
 /* Copies the device record to host memory and waits for the stream. */
 int locmoe_capacity_read(const locmoe_capacity_t *cap_dev, locmoe_capacity_t *cap_host, void *stream);

@@ -23,7 +23,7 @@ WARN_CLAMPED, WARN_BAD_SRC, WARN_BAD_IDX = 1, 2, 4
 FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
-    "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_read", "locmoe_route",
+    "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route",
     "locmoe_dispatch", "locmoe_combine", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
@@ -64,6 +64,7 @@ def _load() -> C.CDLL:
     lib.locmoe_workspace_bytes.argtypes = [C.POINTER(Shape), i32, C.POINTER(C.c_size_t)]
     lib.locmoe_gate.argtypes = [C.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp]
     lib.locmoe_capacity.argtypes = [C.POINTER(Shape), vp, vp, C.POINTER(CapacityRule), vp, vp, vp, vp, C.c_size_t, vp]
+    lib.locmoe_capacity_noalloc.argtypes = [C.POINTER(Shape), vp, vp, C.POINTER(CapacityRule), vp, vp, vp, vp]
     lib.locmoe_capacity_read.argtypes = [vp, C.POINTER(Capacity), vp]
     lib.locmoe_route.argtypes = [C.POINTER(Shape), vp, vp, vp, i32] + [vp] * 10 + [vp, C.c_size_t, vp]
     lib.locmoe_dispatch.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, i32, vp]
@@ -170,6 +171,19 @@ def locmoe_capacity(shape: Shape, idx, cos_sim, rule: CapacityRule, delta_e, the
     return _check("locmoe_capacity", _lib.locmoe_capacity(
         C.byref(shape), _ptr(idx), _ptr(cos_sim), C.byref(rule), _ptr(delta_e), _ptr(theta_e), _ptr(cap_dev),
         _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def locmoe_capacity_noalloc(shape: Shape, idx, cos_sim, rule: CapacityRule, delta_e, theta_e, cap_dev, stream=None) -> int:
+    """locmoe_capacity without a workspace argument: for callers that cannot allocate device memory (the
+    scratch is a fixed array inside the library, at most 8192 experts, shared by all calls on a device)."""
+    _want(idx, torch.int32, shape.T, "idx")
+    _want(cos_sim, torch.float32, shape.T, "cos_sim")
+    _want(delta_e, torch.float32, shape.E, "delta_e")
+    _want(theta_e, torch.float32, shape.E, "theta_e")
+    _want(cap_dev, torch.uint8, CAPACITY_BYTES, "cap_dev")
+    return _check("locmoe_capacity_noalloc", _lib.locmoe_capacity_noalloc(
+        C.byref(shape), _ptr(idx), _ptr(cos_sim), C.byref(rule), _ptr(delta_e), _ptr(theta_e), _ptr(cap_dev),
+        _stream(stream)))
 
 
 def locmoe_capacity_read(cap_dev, stream=None) -> Capacity:

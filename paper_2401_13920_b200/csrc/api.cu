@@ -169,6 +169,7 @@ const char* locmoe_status_string(int code) {
         case LOCMOE_ERR_ALIGN: return "pointer alignment";
         case LOCMOE_ERR_WORKSPACE: return "workspace missing, too small or misaligned";
         case LOCMOE_ERR_CUDA: return "a CUDA call failed";
+        case LOCMOE_ERR_TOO_LARGE: return "size exceeds the built-in scratch of the no-allocation entry point";
         default: return code > 0 ? "warning bits set" : "unknown error";
     }
 }
