@@ -294,17 +294,67 @@ def make_router(shape: Shape, C_alloc: int, rule: CapacityRule, device="cuda") -
     )
 
 
-def router_forward(st: RouterState, x, src_dev, y=None, eps=None, stream=None):
+def router_forward(st: RouterState, x, src_dev, y=None, eps=None, stream=None, out=None):
     """gate -> capacity -> route -> dispatch -> combine on one stream.
 
     ``y`` are the expert outputs in slot layout; with ``y=None`` the experts are
-    the identity and the dispatched buffer itself is combined.  Returns ``st.out``.
+    the identity and the dispatched buffer itself is combined.  Returns the
+    combined output (``st.out`` unless ``out`` is given).
     """
     sh, Ca = st.shape, st.C_alloc
+    out = st.out if out is None else out
     locmoe_gate(sh, x, eps, st.idx, st.gate_w, st.cos_sim, None, stream)
     locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
     locmoe_route(sh, st.idx, src_dev, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
                  st.send_counts, st.load, st.locality, st.status, st.ws, stream)
     locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream)
-    locmoe_combine(sh, Ca, st.buf if y is None else y, st.slot, st.gate_w, st.out, False, stream)
-    return st.out
+    locmoe_combine(sh, Ca, st.buf if y is None else y, st.slot, st.gate_w, out, False, stream)
+    return out
+
+
+class HostRouter:
+    """The path for tokens that live in (pinned) host memory: copy in, five C-ABI calls, copy out.
+
+    Successive ``forward`` calls are pipelined over three streams with double buffers: the host-to-device
+    copy of step i+1 and the device-to-host copy of step i-1 run while step i computes, so a stream of
+    batches is bound by one PCIe direction rather than by the sum of both copies and the kernels.
+    Only memory and stream plumbing lives here; all arithmetic is in the library's kernels.
+    """
+
+    def __init__(self, shape: Shape, C_alloc: int, rule: CapacityRule, device="cuda"):
+        dev = torch.device(device)
+        self.st = make_router(shape, C_alloc, rule, dev)
+        xdt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
+        self.x = [torch.empty(shape.T, shape.H, dtype=xdt, device=dev) for _ in range(2)]
+        self.src = [torch.empty(shape.T, dtype=torch.int32, device=dev) for _ in range(2)]
+        self.out = [self.st.out, torch.empty_like(self.st.out)]
+        self.s_in, self.s_comp, self.s_out = (torch.cuda.Stream(dev) for _ in range(3))
+        self.ev_in = [torch.cuda.Event() for _ in range(2)]
+        self.ev_comp = [torch.cuda.Event() for _ in range(2)]
+        self.ev_out = [torch.cuda.Event() for _ in range(2)]
+        self.i = 0
+
+    def forward(self, x_host, src_host, out_host, y=None):
+        """Queues one step; ``out_host`` is valid after ``synchronize()`` (or once a later step has reused its slot)."""
+        k = self.i & 1
+        with torch.cuda.stream(self.s_in):
+            if self.i >= 2:
+                self.s_in.wait_event(self.ev_comp[k])      # step i-2 has finished reading this input buffer
+            self.x[k].copy_(x_host, non_blocking=True)
+            self.src[k].copy_(src_host, non_blocking=True)
+            self.ev_in[k].record(self.s_in)
+        with torch.cuda.stream(self.s_comp):
+            self.s_comp.wait_event(self.ev_in[k])
+            if self.i >= 2:
+                self.s_comp.wait_event(self.ev_out[k])     # step i-2's output has left this output buffer
+            router_forward(self.st, self.x[k], self.src[k], y=y, stream=self.s_comp, out=self.out[k])
+            self.ev_comp[k].record(self.s_comp)
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.ev_comp[k])
+            out_host.copy_(self.out[k], non_blocking=True)
+            self.ev_out[k].record(self.s_out)
+        self.i += 1
+
+    def synchronize(self):
+        for s in (self.s_in, self.s_comp, self.s_out):
+            s.synchronize()

@@ -225,3 +225,28 @@ def test_route_is_deterministic(P):
         torch.cuda.synchronize()
         for u, v in zip(a, (st.pos, st.slot, st.inv, st.counts, st.send_counts, st.locality)):
             assert torch.equal(u, v)
+
+
+def test_host_router_pipeline_matches_device_path(P):
+    # tokens in pinned host memory, three pipelined steps on different batches
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    w = P.W.CONFIGS[5].scaled(5000)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, torch.bfloat16)
+    rule = B.CapacityRule(1.0, 1.0, -1.0, 0, 0)
+    Ca = B.conventional_capacity(w.T, sh.D, w.E, 1.0)
+    hr = B.HostRouter(sh, Ca, rule, dev)
+    st = B.make_router(sh, Ca, rule, dev)
+    src = W.make_src(w, dev)
+    srch = src.cpu().pin_memory()
+    xs, outs = [], []
+    for i in range(3):
+        wi = W.Workload(**{**w.__dict__, "config": 5 + 10 * i})
+        xs.append(W.make_tokens(wi, dev))
+        outs.append(torch.empty(w.T, w.H, dtype=torch.bfloat16).pin_memory())
+        hr.forward(xs[-1].cpu().pin_memory(), srch, outs[-1])
+    hr.synchronize()
+    for x, o in zip(xs, outs):
+        ref = B.router_forward(st, x, src)
+        torch.cuda.synchronize()
+        assert torch.equal(o.view(torch.int16), ref.cpu().view(torch.int16))
