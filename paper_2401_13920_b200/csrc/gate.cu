@@ -81,7 +81,7 @@ __device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gs
     float se = 0.0f;
     for (int i = lane; i < a.E; i += kWarp) {
         float G = fmaxf(gsum[i] * a.inv_g + (a.eps ? a.eps[i] : 0.0f), 0.0f);
-        se += expf(G - best);
+        se += __expf(G - best);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -93,7 +93,7 @@ __device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gs
         float* pr = a.probs + (size_t)row * a.E;
         for (int i = lane; i < a.E; i += kWarp) {
             float G = fmaxf(gsum[i] * a.inv_g + (a.eps ? a.eps[i] : 0.0f), 0.0f);
-            pr[i] = expf(G - best) * R;
+            pr[i] = __expf(G - best) * R;
         }
     }
     if (lane == 0) {

@@ -7,7 +7,7 @@
 // its key class is pos.  Every step is integer and order independent, so the
 // result is a function of the inputs only; no kernel waits on another CTA.
 //
-// Launch sequence for P radix passes (P = 1 up to 1024 keys, 2 up to 65536):
+// Launch sequence for P radix passes of at most 8 bits (P = 1 up to 256 keys, 2 up to 65536):
 //   init      inv = -1, accumulators and later-pass histograms = 0
 //   hist0     per-tile histogram of digit 0, per-key demand counts
 //   scatter_p every CTA derives its own (digit, tile) offsets from the
@@ -18,6 +18,8 @@
 //   extras    key-class starts and count matrices (kept, send_counts, load,
 //             locality tallies): extra CTAs of scatter_0 when P > 1, a launch
 //             of their own before the only scatter when P = 1.
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace locmoe {
@@ -46,6 +48,8 @@ struct RouteArgs {
     int32_t* toks[2];
     int32_t* hist[kMaxPasses];  // [1 << bits[p]][ntiles], digit major
     int32_t* keystart;          // [K]
+    int32_t* rowtot;            // [256] per-digit totals of the pass being scattered (prescan mode)
+    int prescan;                // 1: a prescan launch turned hist[p] into exclusive prefixes along the tiles
 };
 
 __device__ __forceinline__ int dest_rank(int a, int b, int N, int Dn) {
@@ -188,6 +192,30 @@ __global__ void __launch_bounds__(kThreads) route_extras_kernel(const RouteArgs 
     route_extras(a, blockIdx.x, gridDim.x);
 }
 
+// Large batches only: turns every digit row of hist[pass] into its exclusive prefix along the tiles (in place)
+// and stores the row totals, one warp per row, so that a scatter CTA reads one entry per digit instead of a
+// whole row (total work O(bins x tiles) instead of O(bins x tiles^2)).
+__global__ void __launch_bounds__(kThreads) route_prescan_kernel(const RouteArgs a, int pass) {
+    const int nbins = 1 << a.bits[pass];
+    const int lane = threadIdx.x & 31;
+    const int d = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (d >= nbins) return;
+    int32_t* row = a.hist[pass] + (size_t)d * a.ntiles;
+    const int chunk = (a.ntiles + 31) / 32;
+    const int lo = min(lane * chunk, a.ntiles), hi = min(lo + chunk, a.ntiles);
+    int s = 0;
+    for (int j = lo; j < hi; ++j) s += row[j];
+    int incl = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    int run = incl - s;
+    for (int j = lo; j < hi; ++j) { int v = row[j]; row[j] = run; run += v; }
+    if (lane == 31) a.rowtot[d] = incl;
+}
+
 // One radix pass over one tile per CTA; CTAs beyond ntiles run the extras.
 template <bool FIRST, bool LAST>
 __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs a, int pass, int shift) {
@@ -231,6 +259,9 @@ __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs
     // (kRB rows per batch so that their loads are all in flight together: the matrix lives in L2)
     const int32_t* H = a.hist[pass];
     constexpr int kRB = 8;
+    if (a.prescan) {
+        for (int d = tid; d < nbins; d += kThreads) { pre[d] = H[(size_t)d * a.ntiles + tileid]; tot[d] = a.rowtot[d]; }
+    } else
     for (int d0 = w; d0 < nbins; d0 += kWarps * kRB) {
         int before[kRB], all[kRB];
 #pragma unroll
@@ -351,7 +382,7 @@ int plan_route(const locmoe_shape_t& s, RoutePlan* p) {
     int kb = 1;
     while ((1ll << kb) < K) ++kb;
     p->key_bits = kb;
-    p->passes = kb <= 10 ? 1 : (kb + 7) / 8;
+    p->passes = (kb + 7) / 8;
     int left = kb;
     for (int i = 0; i < 4; ++i) p->bits[i] = 0;
     for (int i = 0; i < p->passes; ++i) {
@@ -375,8 +406,14 @@ int plan_route(const locmoe_shape_t& s, RoutePlan* p) {
         if (i < p->passes) off += align256(((size_t)p->ntiles << p->bits[i]) * 4);
     }
     p->off_keystart = off; off += align256((size_t)K * 4);
+    p->off_rowtot = off; off += 1024;
     p->total = off;
-    p->launches = 2 + p->passes + (p->passes == 1 ? 1 : 0);
+    p->prescan = ((long long)p->ntiles << p->bits[0]) > 32768 ? 1 : 0;
+    {   // testing aid: LOCMOE_PATH=grid forces the large-batch variants at any size
+        const char* o = getenv("LOCMOE_PATH");
+        if (o && o[0] == 'g') p->prescan = 1;
+    }
+    p->launches = 2 + p->passes + (p->passes == 1 ? 1 : 0) + (p->prescan ? p->passes : 0);
     return LOCMOE_OK;
 }
 
@@ -407,6 +444,8 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
         a.hist[i] = reinterpret_cast<int32_t*>(w + p.off_hist[i]);
     }
     a.keystart = reinterpret_cast<int32_t*>(w + p.off_keystart);
+    a.rowtot = reinterpret_cast<int32_t*>(w + p.off_rowtot);
+    a.prescan = p.prescan;
 
     long long init_items = a.rows > a.K ? a.rows : a.K;
     int init_blocks = (int)((init_items + kThreads * 4 - 1) / (kThreads * 4));
@@ -428,6 +467,10 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
     int shift = 0;
     for (int pass = 0; pass < p.passes; ++pass) {
         const bool first = pass == 0, last = pass == p.passes - 1;
+        if (p.prescan) {
+            route_prescan_kernel<<<((1 << p.bits[pass]) + kWarps - 1) / kWarps, kThreads, 0, st>>>(a, pass);
+            if ((rc = check_launch())) return rc;
+        }
         const size_t smb = ((size_t)(kWarps + 2) * sizeof(int)) << p.bits[pass];
         const int grid = p.ntiles + ((first && !last) ? extras : 0);
         if (first && last) route_scatter_kernel<true, true><<<grid, kThreads, smb, st>>>(a, pass, shift);

@@ -64,7 +64,7 @@ def test_config4_full_size_sampled(P):
     assert rep["C_local"] == 16 and 0.05 < rep["drop_frac"] < 0.15
 
 
-# ---- the multi-kernel capacity path (default only beyond 2M tokens or 8192 experts) at small sizes ----
+# ---- the large-batch variants (multi-kernel capacity, prescanned route histograms) forced at small sizes ----
 
 @pytest.fixture
 def grid_path(monkeypatch):
