@@ -213,6 +213,45 @@ int locmoe_combine(const locmoe_shape_t *shape, int32_t C_alloc, const void *y, 
                    const int32_t *slot, const float *gate_w, void *out, int32_t accumulate,
                    void *stream);
 
+/*
+ * Expert feed-forward networks (first equation of Sec. 3.2.1):
+ *   y[row] = W_out[e] . GeLU(W_in[e] . buf[row]),  GeLU(v) = v * Phi(v) (erf form),
+ * for every row of the dispatched buffer, e being the expert that owns the row.
+ * Needs shape->layout == LOCMOE_LAYOUT_RECV (the rows of one expert are the
+ * contiguous block [e * D * C_alloc, (e + 1) * D * C_alloc)) and bf16 tokens.
+ * Empty (zero) rows give zero rows.  Two grouped GEMMs on the tensor cores
+ * (tcgen05, fp32 accumulation); the intermediate is rounded to bf16.
+ *   buf   [D*E*C_alloc][H] bf16        w_in  [E][F][H] bf16      w_out [E][H][F] bf16
+ *   h1    [D*E*C_alloc][F] bf16 scratch (caller's)               y [D*E*C_alloc][H] of y_dtype
+ * H and F must be multiples of 8; all five pointers 16-byte aligned.
+ */
+int locmoe_expert_ffn(const locmoe_shape_t *shape, int32_t C_alloc, int32_t F, const void *buf,
+                      const void *w_in, const void *w_out, void *h1, void *y, int32_t y_dtype,
+                      void *stream);
+
+/* Every device array of one MoE layer pass, for locmoe_moe_layer (host struct of device pointers;
+ * sizes as documented at the individual calls). */
+typedef struct {
+    int32_t *idx; float *gate_w; float *cos_sim; float *delta_e; float *theta_e;
+    locmoe_capacity_t *cap_dev;
+    int32_t *pos; int32_t *slot; uint8_t *drop; int32_t *inv;
+    int32_t *counts; int32_t *kept; int32_t *send_counts; int32_t *load; int64_t *locality; int32_t *status;
+    void *ws; size_t ws_bytes;
+    void *buf;   /* [D*E*C_alloc][H] of x_dtype                                   */
+    void *h1;    /* [D*E*C_alloc][F] bf16, only with experts                      */
+    void *y;     /* [D*E*C_alloc][H] bf16, only with experts                      */
+} locmoe_layer_buffers_t;
+
+/*
+ * One whole MoE layer pass on one stream: gate -> capacity -> route -> dispatch ->
+ * expert FFN -> combine (the six calls above, in order, nothing else).  With
+ * w_in == NULL the experts are the identity and the dispatched buffer itself is
+ * combined.  out [T][H] of x_dtype.  eps may be NULL.
+ */
+int locmoe_moe_layer(const locmoe_shape_t *shape, const void *x, const int32_t *src_dev, const float *eps,
+                     const locmoe_capacity_rule_t *rule, int32_t C_alloc, int32_t F, const void *w_in,
+                     const void *w_out, const locmoe_layer_buffers_t *bufs, void *out, void *stream);
+
 /* Kernels launched per call of gate, capacity, route, dispatch, combine on this
  * shape (counts[5], host memory); a bookkeeping aid for benchmarks.  The paper
  * has no counterpart. */
@@ -221,7 +260,8 @@ int locmoe_launch_counts(const locmoe_shape_t *shape, int32_t counts[5]);
 /* Device-side diagnostics of this library on the current device, copied to host
  * memory after waiting for the stream: bit 0 is set if a kernel gave up a
  * bounded wait for one of its own asynchronous copies (its output is then
- * incomplete).  0 in normal operation.  The paper has no counterpart. */
+ * incomplete); bit 1 the same for the expert-FFN kernels.  0 in normal operation.
+ * The paper has no counterpart. */
 int locmoe_device_flags(int32_t *flags_host, void *stream);
 
 /* Text for a return code of this library (host string, never NULL). */

@@ -77,6 +77,9 @@ def lib():
         L.oracle_combine.restype = C.c_int
         L.oracle_combine.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p]
+        L.oracle_ffn_rows.restype = C.c_int
+        L.oracle_ffn_rows.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -244,3 +247,19 @@ def combine(y, y_dtype, slot, R, prev=None) -> np.ndarray:
     if rc != 0:
         raise ValueError("oracle_combine: error %d" % rc)
     return out
+
+
+def ffn_rows(x_bits, w_in_bits, w_out_bits):
+    """Expert FFN of one expert on rows x [n][H]; w_in [F][H], w_out [H][F] (bf16 bits).  Returns (y, spread)."""
+    x = _raw(x_bits, BF16)
+    w_in = _raw(w_in_bits, BF16)
+    w_out = _raw(w_out_bits, BF16)
+    n, H = x.shape
+    F = w_in.shape[0]
+    assert w_in.shape == (F, H) and w_out.shape == (H, F)
+    y = np.empty((n, H), np.float64)
+    sp = np.empty((n, H), np.float64)
+    rc = lib().oracle_ffn_rows(_p(x), n, H, F, _p(w_in), _p(w_out), _p(y), _p(sp))
+    if rc != 0:
+        raise ValueError("oracle_ffn_rows: error %d" % rc)
+    return y, sp

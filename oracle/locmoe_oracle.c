@@ -30,6 +30,10 @@
  *   oracle_combine   y_m = R_m * expert_out (first equation of Sec. 3.2.1,
  *                    top-1 so a single term; a dropped token has no term).
  *
+ *   oracle_ffn_rows  expert network of the same equation:
+ *                    W_out . GeLU(W_in . x), GeLU(v) = v * Phi(v) with Phi the
+ *                    standard Gaussian CDF (Sec. 3.2.1), in double.
+ *
  * Parity pins: every function below is pinned by tests/test_oracle_*.py
  * (dense-weight identity, closed forms, library incomplete beta, brute force,
  * round trip).  The locality loss L_loc is not computed here at all.
@@ -376,5 +380,40 @@ int oracle_combine(const void *y, int y_dtype, int64_t T, int32_t H, const int32
             if (prev) v += prev[t * H + j];
             out[t * H + j] = v;
         }
+    return 0;
+}
+
+/*
+ * Expert FFN on `nrows` rows that all belong to one expert (first equation of Sec. 3.2.1):
+ *   h[f] = sum_j W_in[f][j] x[j],   g[f] = h[f] * Phi(h[f]) = 0.5 h[f] (1 + erf(h[f] / sqrt 2)),
+ *   y[i] = sum_f W_out[i][f] g[f].
+ * x [nrows][H], w_in [F][H], w_out [H][F] are bf16 bit patterns, widened exactly; everything in double.
+ * y [nrows][H].  spread [nrows][H] (may be NULL) receives sqrt(sum_f (W_out[i][f] g[f])^2): the tests derive
+ * from it how far a result whose intermediate g was rounded to bf16 may lie from y.
+ */
+int oracle_ffn_rows(const uint16_t *x, int64_t nrows, int32_t H, int32_t F, const uint16_t *w_in,
+                    const uint16_t *w_out, double *y, double *spread)
+{
+    double *g = (double *)malloc(sizeof(double) * (size_t)F);
+    if (!g) return -6;
+    for (int64_t r = 0; r < nrows; ++r) {
+        for (int32_t f = 0; f < F; ++f) {
+            double h = 0.0;
+            for (int32_t j = 0; j < H; ++j)
+                h += widen(w_in, ORACLE_BF16, (int64_t)f * H + j) * widen(x, ORACLE_BF16, r * H + j);
+            g[f] = 0.5 * h * (1.0 + erf(h / sqrt(2.0)));
+        }
+        for (int32_t i = 0; i < H; ++i) {
+            double acc = 0.0, sq = 0.0;
+            for (int32_t f = 0; f < F; ++f) {
+                double term = widen(w_out, ORACLE_BF16, (int64_t)i * F + f) * g[f];
+                acc += term;
+                sq += term * term;
+            }
+            y[r * H + i] = acc;
+            if (spread) spread[r * H + i] = sqrt(sq);
+        }
+    }
+    free(g);
     return 0;
 }

@@ -24,7 +24,7 @@ FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
     "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route",
-    "locmoe_dispatch", "locmoe_combine", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
+    "locmoe_dispatch", "locmoe_combine", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
 
@@ -48,6 +48,13 @@ class Capacity(C.Structure):
                 ("flags", C.c_int32)]
 
 
+class LayerBuffers(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("idx", "gate_w", "cos_sim", "delta_e", "theta_e", "cap_dev", "pos", "slot",
+                                           "drop", "inv", "counts", "kept", "send_counts", "load", "locality",
+                                           "status", "ws")] + [("ws_bytes", C.c_size_t)] + \
+               [(n, C.c_void_p) for n in ("buf", "h1", "y")]
+
+
 CAPACITY_BYTES = C.sizeof(Capacity)
 
 
@@ -69,6 +76,9 @@ def _load() -> C.CDLL:
     lib.locmoe_route.argtypes = [C.POINTER(Shape), vp, vp, vp, i32] + [vp] * 10 + [vp, C.c_size_t, vp]
     lib.locmoe_dispatch.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, i32, vp]
     lib.locmoe_combine.argtypes = [C.POINTER(Shape), i32, vp, i32, vp, vp, vp, i32, vp]
+    lib.locmoe_expert_ffn.argtypes = [C.POINTER(Shape), i32, i32, vp, vp, vp, vp, vp, i32, vp]
+    lib.locmoe_moe_layer.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(CapacityRule), i32, i32, vp, vp,
+                                     C.POINTER(LayerBuffers), vp, vp]
     lib.locmoe_launch_counts.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32 * 5)]
     lib.locmoe_device_flags.argtypes = [C.POINTER(C.c_int32), vp]
     lib.locmoe_status_string.argtypes = [C.c_int]
@@ -233,6 +243,33 @@ def locmoe_combine(shape: Shape, C_alloc, y, slot, gate_w, out, accumulate=False
     return _check("locmoe_combine", _lib.locmoe_combine(C.byref(shape), int(C_alloc), _ptr(y), dtype_code(y.dtype),
                                                         _ptr(slot), _ptr(gate_w), _ptr(out), 1 if accumulate else 0,
                                                         _stream(stream)))
+
+
+def locmoe_expert_ffn(shape: Shape, C_alloc, F, buf, w_in, w_out, h1, y, stream=None) -> int:
+    rows = shape.D * shape.E * C_alloc
+    _want(buf, torch.bfloat16, rows * shape.H, "buf")
+    _want(w_in, torch.bfloat16, shape.E * F * shape.H, "w_in")
+    _want(w_out, torch.bfloat16, shape.E * shape.H * F, "w_out")
+    _want(h1, torch.bfloat16, rows * F, "h1")
+    _want(y, y.dtype, rows * shape.H, "y")
+    return _check("locmoe_expert_ffn", _lib.locmoe_expert_ffn(C.byref(shape), int(C_alloc), int(F), _ptr(buf), _ptr(w_in),
+                                                              _ptr(w_out), _ptr(h1), _ptr(y), dtype_code(y.dtype),
+                                                              _stream(stream)))
+
+
+def layer_buffers(st: "RouterState", h1=None, y=None) -> LayerBuffers:
+    """Pointer block for locmoe_moe_layer from a RouterState (plus the FFN scratch and output)."""
+    p = lambda t: None if t is None else t.data_ptr()
+    return LayerBuffers(p(st.idx), p(st.gate_w), p(st.cos_sim), p(st.delta_e), p(st.theta_e), p(st.cap_dev), p(st.pos),
+                        p(st.slot), p(st.drop), p(st.inv), p(st.counts), p(st.kept), p(st.send_counts), p(st.load),
+                        p(st.locality), p(st.status), p(st.ws), st.ws.numel(), p(st.buf), p(h1), p(y))
+
+
+def locmoe_moe_layer(shape: Shape, x, src_dev, eps, rule: CapacityRule, C_alloc, F, w_in, w_out, bufs: LayerBuffers,
+                     out, stream=None) -> int:
+    return _check("locmoe_moe_layer", _lib.locmoe_moe_layer(
+        C.byref(shape), _ptr(x), _ptr(src_dev), _ptr(eps), C.byref(rule), int(C_alloc), int(F), _ptr(w_in), _ptr(w_out),
+        C.byref(bufs), _ptr(out), _stream(stream)))
 
 
 def conventional_capacity(T: int, D: int, E: int, capacity_factor: float) -> int:

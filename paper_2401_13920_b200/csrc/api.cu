@@ -138,6 +138,53 @@ int locmoe_combine(const locmoe_shape_t* shape, int32_t C_alloc, const void* y, 
     return launch_combine(*shape, rows, y, y_dtype, slot, gate_w, out, accumulate, static_cast<cudaStream_t>(stream));
 }
 
+int locmoe_expert_ffn(const locmoe_shape_t* shape, int32_t C_alloc, int32_t F, const void* buf, const void* w_in,
+                      const void* w_out, void* h1, void* y, int32_t y_dtype, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!buf || !w_in || !w_out || !h1 || !y) return LOCMOE_ERR_NULL;
+    if (shape->layout != LOCMOE_LAYOUT_RECV || shape->x_dtype != LOCMOE_BF16) return LOCMOE_ERR_DTYPE;
+    if (y_dtype != LOCMOE_F32 && y_dtype != LOCMOE_BF16) return LOCMOE_ERR_DTYPE;
+    if (F < 8 || F % 8 != 0 || shape->H % 8 != 0) return LOCMOE_ERR_SHAPE;
+    const long long rows = buffer_rows(shape, C_alloc);
+    if (rows < 0) return LOCMOE_ERR_SHAPE;
+    if ((uintptr_t)buf % 16 || (uintptr_t)w_in % 16 || (uintptr_t)w_out % 16 || (uintptr_t)h1 % 16 || (uintptr_t)y % 16)
+        return LOCMOE_ERR_ALIGN;
+    return launch_expert_ffn(*shape, rows, F, buf, w_in, w_out, h1, y, y_dtype, static_cast<cudaStream_t>(stream));
+}
+
+int locmoe_moe_layer(const locmoe_shape_t* shape, const void* x, const int32_t* src_dev, const float* eps,
+                     const locmoe_capacity_rule_t* rule, int32_t C_alloc, int32_t F, const void* w_in,
+                     const void* w_out, const locmoe_layer_buffers_t* b, void* out, void* stream) {
+    if (!b) return LOCMOE_ERR_NULL;
+    int warn = 0;
+    int rc = locmoe_gate(shape, x, eps, b->idx, b->gate_w, b->cos_sim, nullptr, stream);
+    if (rc < 0) return rc;
+    warn |= rc;
+    rc = locmoe_capacity(shape, b->idx, b->cos_sim, rule, b->delta_e, b->theta_e, b->cap_dev, b->ws, b->ws_bytes, stream);
+    if (rc < 0) return rc;
+    warn |= rc;
+    rc = locmoe_route(shape, b->idx, src_dev, b->cap_dev, C_alloc, b->pos, b->slot, b->drop, b->inv, b->counts, b->kept,
+                      b->send_counts, b->load, b->locality, b->status, b->ws, b->ws_bytes, stream);
+    if (rc < 0) return rc;
+    warn |= rc;
+    rc = locmoe_dispatch(shape, C_alloc, x, b->inv, b->buf, 1, stream);
+    if (rc < 0) return rc;
+    warn |= rc;
+    const void* ysrc = b->buf;
+    int ydt = shape->x_dtype;
+    if (w_in) {
+        rc = locmoe_expert_ffn(shape, C_alloc, F, b->buf, w_in, w_out, b->h1, b->y, LOCMOE_BF16, stream);
+        if (rc < 0) return rc;
+        warn |= rc;
+        ysrc = b->y;
+        ydt = LOCMOE_BF16;
+    }
+    rc = locmoe_combine(shape, C_alloc, ysrc, ydt, b->slot, b->gate_w, out, 0, stream);
+    if (rc < 0) return rc;
+    return warn | rc;
+}
+
 int locmoe_launch_counts(const locmoe_shape_t* shape, int32_t counts[5]) {
     int rc = check_shape(shape);
     if (rc) return rc;
@@ -154,9 +201,10 @@ int locmoe_launch_counts(const locmoe_shape_t* shape, int32_t counts[5]) {
 
 int locmoe_device_flags(int32_t* flags_host, void* stream) {
     if (!flags_host) return LOCMOE_ERR_NULL;
-    int v = 0;
+    int v = 0, f = 0;
     int rc = read_device_flags(&v, static_cast<cudaStream_t>(stream));
-    *flags_host = v;
+    if (rc == LOCMOE_OK) rc = read_ffn_flags(&f, static_cast<cudaStream_t>(stream));
+    *flags_host = v | (f << 1);
     return rc;
 }
 

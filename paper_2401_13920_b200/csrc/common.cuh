@@ -53,6 +53,10 @@ int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const 
 int launch_combine(const locmoe_shape_t& s, int64_t rows, const void* y, int y_dtype, const int32_t* slot, const float* gate_w,
                    void* out, int accumulate, cudaStream_t st);
 
+int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* buf, const void* w_in,
+                      const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st);
+int read_ffn_flags(int* out, cudaStream_t st);
+
 // Copies the device diagnostics word to host memory (synchronises the stream).
 int read_device_flags(int* out, cudaStream_t st);
 

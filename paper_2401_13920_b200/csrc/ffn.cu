@@ -1,0 +1,325 @@
+// Expert FFN of the MoE layer (first equation of Sec. 3.2.1):
+//   y = W_out . GeLU(W_in . x)   per expert, GeLU(v) = v * Phi(v) (exact erf form),
+// on the dispatched buffer in RECV layout, where the rows of one expert are contiguous.
+//
+// Two grouped GEMMs (all experts in one launch each), both "NT": the activations [rows][K] and the
+// weights [E][N][K] are K-major, so both operands are loaded as 128-byte-swizzled K-major tiles.
+//   - TMA (cp.async.bulk.tensor, no multicast) fills a 4-stage ring of 128x64 (A) and 256x64 (B) bf16 tiles,
+//   - one elected thread issues tcgen05.mma (128 x 256 x 16 per instruction, fp32 accumulators in TMEM),
+//   - two 128x256 accumulators (512 TMEM columns) alternate, so the epilogue of a tile overlaps the MMAs
+//     of the next one,
+//   - four epilogue warps read the accumulator with tcgen05.ld (one row per thread), apply GeLU (first GEMM),
+//     convert and store.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = epilogue.  Persistent CTAs, one per SM.
+// Every barrier wait is bounded; on a timeout the kernel raises the device diagnostics flag, leaves its
+// loops, frees its TMEM and returns.
+#include <cuda.h>
+#include <math.h>
+
+#include <mutex>
+
+#include "common.cuh"
+
+namespace locmoe {
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, NSTAGE = 4;
+constexpr int UMMA_K = 16;
+constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int kFfnThreads = 192;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr size_t kFfnSmem = (size_t)NSTAGE * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+__device__ int g_ffn_flags = 0;  // bit 0: a bounded wait gave up
+
+struct FfnArgs {
+    void* out;            // [E * M][N] bf16 or fp32
+    int out_f32;          // 0: bf16, 1: fp32
+    int gelu;             // apply GeLU in the epilogue
+    int E, M, N, K;       // experts, rows per expert, output columns, reduction length
+    int m_tiles, n_tiles;
+};
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait that also gives up as soon as another role has raised the abort word.
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_word) {
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 63u && *abort_word) return false;
+    }
+    *abort_word = 1;
+    atomicOr(&g_ffn_flags, 1);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile with 128-byte swizzle: rows of 128 bytes, groups of
+// 8 rows 1024 bytes apart (stride byte offset), leading byte offset unused (1), descriptor version 1.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr & 0x3ffffu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate) : "memory");
+}
+// Arrives on the mbarrier once all MMAs issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)); }
+
+__global__ void __launch_bounds__(kFfnThreads, 1)
+ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const FfnArgs a) {
+    extern __shared__ unsigned char smraw[];
+    // 1024-byte alignment: the 128-byte swizzle pattern repeats every 8 rows of 128 bytes
+    unsigned char* base = reinterpret_cast<unsigned char*>(((uintptr_t)smraw + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)NSTAGE * STAGE_BYTES);
+    uint64_t* full = bars;                 // [NSTAGE] tile landed in shared memory
+    uint64_t* empty = bars + NSTAGE;       // [NSTAGE] MMAs that read the stage are done
+    uint64_t* acc_full = bars + 2 * NSTAGE;  // [2] accumulator complete
+    uint64_t* acc_empty = acc_full + 2;      // [2] accumulator drained by the epilogue
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile int* abort_word = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
+        *abort_word = 0;
+        mbar_init_fence();
+    }
+    if (warp == 2) {  // one warp allocates all 512 TMEM columns (one CTA per SM, so this cannot starve)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int tiles_per_expert = a.m_tiles * a.n_tiles;
+    const int total_tiles = a.E * tiles_per_expert;
+    const int kblocks = (a.K + BK - 1) / BK;
+
+    if (warp == 0) {
+        if (lane == 0) {  // ---- TMA producer ----
+            int stage = 0; uint32_t phase = 0;
+            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+                const int e = tile / tiles_per_expert, rem = tile - e * tiles_per_expert;
+                const int nt = rem / a.m_tiles, mt = rem - nt * a.m_tiles;
+                const int row0 = e * a.M + mt * BM, n0 = nt * BN;
+                bool ok = true;
+                for (int kb = 0; kb < kblocks && ok; ++kb) {
+                    if (!wait_or_abort(&empty[stage], phase ^ 1u, abort_word)) { ok = false; break; }
+                    unsigned char* sa = base + (size_t)stage * STAGE_BYTES;
+                    mbar_expect_tx(&full[stage], STAGE_BYTES);
+                    tma_load_2d(sa, &tmA, kb * BK, row0, &full[stage]);
+                    tma_load_3d(sa + A_BYTES, &tmB, kb * BK, n0, e, &full[stage]);
+                    if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {  // ---- MMA issuer ----
+            int stage = 0; uint32_t phase = 0;
+            int acc = 0; uint32_t acc_phase = 0;
+            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+                if (!wait_or_abort(&acc_empty[acc], acc_phase ^ 1u, abort_word)) break;
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)acc * BN;
+                bool ok = true;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!wait_or_abort(&full[stage], phase, abort_word)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(base + (size_t)stage * STAGE_BYTES);
+                    const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        umma_bf16(tmem_d, umma_desc_sw128(sa + k * UMMA_K * 2), umma_desc_sw128(sb + k * UMMA_K * 2),
+                                  (kb > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(&empty[stage]);
+                    if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(&acc_full[acc]);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {  // ---- epilogue warps 2..5: TMEM lane quadrant = warp % 4 ----
+        const int q = warp & 3;
+        int acc = 0; uint32_t acc_phase = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            const int e = tile / tiles_per_expert, rem = tile - e * tiles_per_expert;
+            const int nt = rem / a.m_tiles, mt = rem - nt * a.m_tiles;
+            if (!wait_or_abort(&acc_full[acc], acc_phase, abort_word)) break;
+            tc_fence_after();
+            const int r_in = mt * BM + q * 32 + lane;        // row inside the expert's block
+            const bool row_ok = r_in < a.M;
+            const long long grow = (long long)e * a.M + r_in;
+            const int n0 = nt * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                __syncwarp();  // tcgen05.ld is warp-collective: reconverge after the masked stores
+                uint32_t r[32];
+                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
+                const int col0 = n0 + c * 32;
+                if (!row_ok || col0 >= a.N) continue;
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    v[i] = __uint_as_float(r[i]);
+                    if (a.gelu) v[i] = gelu_erf(v[i]);
+                }
+                if (col0 + 32 <= a.N) {
+                    if (a.out_f32) {
+                        uint4* dst = reinterpret_cast<uint4*>(static_cast<float*>(a.out) + grow * a.N + col0);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            dst[i] = make_uint4(__float_as_uint(v[4 * i]), __float_as_uint(v[4 * i + 1]),
+                                                __float_as_uint(v[4 * i + 2]), __float_as_uint(v[4 * i + 3]));
+                    } else {
+                        uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(a.out) + grow * a.N + col0);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            dst[i] = make_uint4(cvt_bf16x2(make_float2(v[8 * i], v[8 * i + 1])),
+                                                cvt_bf16x2(make_float2(v[8 * i + 2], v[8 * i + 3])),
+                                                cvt_bf16x2(make_float2(v[8 * i + 4], v[8 * i + 5])),
+                                                cvt_bf16x2(make_float2(v[8 * i + 6], v[8 * i + 7])));
+                    }
+                } else {  // ragged last column block
+                    for (int i = 0; i < 32 && col0 + i < a.N; ++i) {
+                        if (a.out_f32) static_cast<float*>(a.out)[grow * a.N + col0 + i] = v[i];
+                        else static_cast<uint16_t*>(a.out)[grow * a.N + col0 + i] = (uint16_t)f32_to_bf16_bits(v[i]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[acc]);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side: tensor maps through the driver entry point (no link-time dependency on libcuda) ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::mutex m;
+    std::lock_guard<std::mutex> lock(m);
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// K-major bf16 matrix [outer...][rows][K] with a box of box_rows x 64 elements, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* ptr, int rank, const uint64_t* dims, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[3] = {dims[0], dims[1], rank == 3 ? dims[2] : 1};
+    cuuint64_t gstr[2] = {dims[0] * 2, dims[0] * dims[1] * 2};
+    cuuint32_t box[3] = {(cuuint32_t)BK, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), gdim, gstr, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int launch_gemm(const void* A, const void* W, void* out, int out_f32, int gelu, int E, int M, int N, int K,
+                cudaStream_t st) {
+    CUtensorMap tmA, tmB;
+    const uint64_t da[2] = {(uint64_t)K, (uint64_t)E * M};
+    const uint64_t db[3] = {(uint64_t)K, (uint64_t)N, (uint64_t)E};
+    if (!make_map(&tmA, A, 2, da, BM) || !make_map(&tmB, W, 3, db, BN)) return LOCMOE_ERR_CUDA;
+    FfnArgs a{};
+    a.out = out; a.out_f32 = out_f32; a.gelu = gelu; a.E = E; a.M = M; a.N = N; a.K = K;
+    a.m_tiles = (M + BM - 1) / BM;
+    a.n_tiles = (N + BN - 1) / BN;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(ffn_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFfnSmem) != cudaSuccess) {
+            cudaGetLastError();
+            return LOCMOE_ERR_CUDA;
+        }
+        attr_done = true;
+    }
+    long long tiles = (long long)E * a.m_tiles * a.n_tiles;
+    int grid = sm_count();
+    if (tiles < grid) grid = (int)tiles;
+    ffn_gemm_kernel<<<grid, kFfnThreads, kFfnSmem, st>>>(tmA, tmB, a);
+    return check_launch();
+}
+
+}  // namespace
+
+int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* buf, const void* w_in,
+                      const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st) {
+    const int E = s.E;
+    const int M = (int)(rows / E);
+    int rc = launch_gemm(buf, w_in, h1, 0, 1, E, M, F, s.H, st);
+    if (rc) return rc;
+    return launch_gemm(h1, w_out, y, y_dtype == LOCMOE_F32 ? 1 : 0, 0, E, M, s.H, F, st);
+}
+
+int read_ffn_flags(int* out, cudaStream_t st) {
+    if (cudaMemcpyFromSymbolAsync(out, g_ffn_flags, sizeof(int), 0, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return LOCMOE_ERR_CUDA;
+    }
+    return LOCMOE_OK;
+}
+
+}  // namespace locmoe

@@ -133,6 +133,18 @@ def make_expert_out(w: Workload, rows: int, device="cpu", dtype: str = "f32") ->
     return out
 
 
+def make_expert_weights(w: Workload, F: int, device="cpu", std: float = 0.02):
+    """Random-init expert weights of config 5: W_in [E][F][H], W_out [E][H][F], bf16, N(0, std)."""
+    dev = torch.device(device)
+    gen = _gen(dev, w.seed + 5)
+    def draw(a, b, c):
+        out = torch.empty(a, b, c, dtype=torch.bfloat16, device=dev)
+        for e in range(a):
+            out[e] = (torch.randn(b, c, generator=gen, device=dev, dtype=torch.float32) * std).to(torch.bfloat16)
+        return out
+    return draw(w.E, F, w.H), draw(w.E, w.H, F)
+
+
 def host_bits(x: torch.Tensor) -> np.ndarray:
     """Raw storage on the host: float32 array, or uint16 array holding bf16 bits."""
     x = x.detach().cpu().contiguous()

@@ -1,0 +1,113 @@
+"""GPU parity of the expert FFN (tcgen05 grouped GEMMs) and of the whole-layer call against the CPU oracle.
+
+Tolerance, from the arithmetic: the kernels take bf16 inputs, accumulate in fp32 and round the intermediate
+g = GeLU(W_in x) to bf16 (8 significant bits: relative error at most 2^-8 per element, independent signs), then accumulate
+y = sum_f W_out[i][f] g[f] in fp32 and round y to bf16.  With s_i = sqrt(sum_f (W_out[i][f] g[f])^2) (returned by
+the oracle) the deviation from the fp64 oracle is bounded, with wide margin, by
+    6 * 2^-8 / sqrt(3) * s_i   (intermediate rounding: six standard deviations of a uniform error)
+  + 2^-8 * |y_i|               (final bf16 rounding, half an ulp is at most |y| / 256)
+  + 1e-6 * sum-scale           (fp32 accumulation).
+"""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import oracle
+    oracle.build()
+    from tests import parity
+    return parity
+
+
+def _tol(y, spread, out_is_bf16):
+    t = 6.0 * 2.0 ** -8 / np.sqrt(3.0) * spread + 1e-5 * spread + 1e-7
+    if out_is_bf16:
+        t = t + 2.0 ** -8 * np.abs(y)
+    return t
+
+
+def _check_rows(P, buf, w_in, w_out, y, E, M, rows, y_is_bf16=True):
+    W = P.W
+    for r in rows:
+        e = r // M
+        want, spread = P.oracle.ffn_rows(W.host_bits(buf[r:r + 1]), W.host_bits(w_in[e]), W.host_bits(w_out[e]))
+        got = y[r].double().cpu().numpy()
+        err = np.abs(got - want[0])
+        assert (err <= _tol(want[0], spread[0], y_is_bf16)).all(), "row %d: max err %.4g" % (r, err.max())
+
+
+@pytest.mark.parametrize("E,N,Dn,C,H,F,ydt", [
+    (2, 1, 2, 32, 64, 256, torch.bfloat16),      # M = 64: less than one tile
+    (4, 2, 2, 70, 264, 520, torch.bfloat16),     # M = 280, K and N with ragged tails
+    (4, 2, 2, 70, 264, 520, torch.float32),
+    (8, 1, 8, 40, 512, 1024, torch.bfloat16),    # M = 320, several k-blocks and n-tiles
+])
+def test_expert_ffn_small_shapes_all_rows(P, E, N, Dn, C, H, F, ydt):
+    B = P.B
+    dev = torch.device("cuda:0")
+    D = N * Dn
+    rows, M = D * E * C, D * C
+    g = torch.Generator(device=dev).manual_seed(5)
+    buf = torch.randn(rows, H, generator=g, device=dev).to(torch.bfloat16)
+    buf[3] = 0                                                    # an empty slot stays empty
+    w_in = (torch.randn(E, F, H, generator=g, device=dev) * 0.08).to(torch.bfloat16)
+    w_out = (torch.randn(E, H, F, generator=g, device=dev) * 0.08).to(torch.bfloat16)
+    sh = B.make_shape(rows, H, E, N, Dn, torch.bfloat16, B.LAYOUT_RECV)
+    h1 = torch.empty(rows, F, dtype=torch.bfloat16, device=dev)
+    y = torch.full((rows, H), 7.0, dtype=ydt, device=dev)
+    B.locmoe_expert_ffn(sh, C, F, buf, w_in, w_out, h1, y)
+    torch.cuda.synchronize()
+    assert B.locmoe_device_flags() == 0
+    assert not y[3].any().item()
+    _check_rows(P, buf, w_in, w_out, y, E, M, range(rows), ydt == torch.bfloat16)
+
+
+def test_expert_ffn_rejects_send_layout_and_bad_sizes(P):
+    B = P.B
+    import ctypes as C
+    one = C.c_void_p(256)
+    sh = B.make_shape(64, 64, 2, 1, 2, B.BF16, B.LAYOUT_SEND)
+    assert B._lib.locmoe_expert_ffn(C.byref(sh), 4, 64, one, one, one, one, one, B.BF16, None) == -3
+    sh = B.make_shape(64, 64, 2, 1, 2, B.BF16, B.LAYOUT_RECV)
+    assert B._lib.locmoe_expert_ffn(C.byref(sh), 4, 60, one, one, one, one, one, B.BF16, None) == -2
+    assert B._lib.locmoe_expert_ffn(C.byref(sh), 4, 64, C.c_void_p(8), one, one, one, one, B.BF16, None) == -4
+
+
+def test_full_layer_config5_scaled(P):
+    # config 5: router + dispatch (RECV layout), expert FFN with random-init weights, combine; one C-ABI call
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    w = W.CONFIGS[5].scaled(8192)
+    F = 10240
+    x = W.make_tokens(w, dev)
+    src = W.make_src(w, dev)
+    w_in, w_out = W.make_expert_weights(w, F, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, B.LAYOUT_RECV)
+    rule = B.CapacityRule(1.0, 1.0, -1.0, 0, 0)
+    Ca = B.conventional_capacity(w.T, sh.D, w.E, 1.0)
+    st = B.make_router(sh, Ca, rule, dev)
+    h1 = torch.empty(st.rows, F, dtype=torch.bfloat16, device=dev)
+    y = torch.empty(st.rows, w.H, dtype=torch.bfloat16, device=dev)
+    B.locmoe_moe_layer(sh, x, src, None, rule, Ca, F, w_in, w_out, B.layer_buffers(st, h1, y), st.out)
+    torch.cuda.synchronize()
+    assert B.locmoe_device_flags() == 0
+    # router stages against the oracle
+    gi = P.check_gate(x, sh, st)
+    cap, _ = P.check_capacity(sh, st, rule, gi)
+    rr = P.check_route(sh, st, src, cap)
+    P.check_dispatch_full(x, sh, st, rr)
+    # expert outputs of sampled occupied and empty rows
+    rng = np.random.default_rng(3)
+    occ = np.nonzero(rr.inv >= 0)[0]
+    emp = np.nonzero(rr.inv < 0)[0]
+    rows = np.concatenate([rng.choice(occ, 12, replace=False), emp[:2]])
+    _check_rows(P, st.buf, w_in, w_out, y, w.E, st.rows // w.E, [int(r) for r in rows])
+    # combine of the FFN output
+    toks = np.unique(np.concatenate([rng.integers(0, w.T, 256), np.nonzero(rr.drop)[0][:16]]))
+    P.check_combine_sampled(y, sh, st, rr, gi, toks)
