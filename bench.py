@@ -41,6 +41,8 @@ def parse_args():
     ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=12)
+    ap.add_argument("--no-ffn", action="store_true", help="config 5 only: identity experts instead of the expert FFN")
+    ap.add_argument("--ffn-inner", type=int, default=10240, help="config 5: inner size F of the expert FFN")
     ap.add_argument("--tokens", type=int, default=0, help="override T (profiling-sized case; not the metric's workload)")
     return ap.parse_args()
 
@@ -51,6 +53,15 @@ def measured_peak():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def measured_tensor_peak():
+    """Sustained cuBLAS bf16 rate of this pool (the FFN runs inside a long step), else the fallback figure."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured (cuBLAS bf16 sustained, MEASURED_PEAKS.json)"
+    except Exception:
+        return 1400.0, "fallback"
 
 
 class ClockSampler(threading.Thread):
@@ -178,6 +189,7 @@ def workload_config(w, args, n_tokens=None):
     return {
         "workload": "config %d (%s): T=%d H=%d E=%d %s tokens, %dx%d logical devices, c_f=%g, %s layout" % (
             w.config, w.name, n_tokens or w.T, w.H, w.E, w.dtype, w.n_nodes, w.dev_per_node, args.cf, args.layout),
+        "expert_ffn": bool((w.config % 10) == 5 and not getattr(args, "no_ffn", False)),
         "T": n_tokens or w.T, "H": w.H, "E": w.E, "token_dtype": w.dtype, "n_nodes": w.n_nodes,
         "dev_per_node": w.dev_per_node, "capacity_factor": args.cf, "layout": args.layout,
         "l2": "inputs exceed the 126 MB L2, no flush" if (n_tokens or w.T) * w.H * (2 if w.dtype == "bf16" else 4) > 126e6
@@ -216,6 +228,9 @@ def main():
     if world > 1:
         # every rank routes its own batch: same shape, its own seed
         w = W.Workload(**{**w.__dict__, "config": w.config + 10 * rank, "name": w.name})
+    use_ffn = (w.config % 10) == 5 and not args.no_ffn
+    if use_ffn:
+        args.layout = "recv"      # the expert FFN works on the per-expert contiguous (receive-side) layout
     layout = B.LAYOUT_SEND if args.layout == "send" else B.LAYOUT_RECV
     x = W.make_tokens(w, dev)
     src = W.make_src(w, dev)
@@ -226,10 +241,16 @@ def main():
     y = None
     if w.y_dtype == "f32":
         y = W.make_expert_out(w, st.rows, dev, "f32")
+    F = args.ffn_inner
+    w_in = w_out = h1 = None
+    if use_ffn:
+        w_in, w_out = W.make_expert_weights(w, F, dev)
+        h1 = torch.empty(st.rows, F, dtype=torch.bfloat16, device=dev)
+        y = torch.empty(st.rows, w.H, dtype=torch.bfloat16, device=dev)
     ysrc = st.buf if y is None else y
 
     stream = torch.cuda.current_stream()
-    stages = ["gate", "capacity", "route", "dispatch", "combine"]
+    stages = ["gate", "capacity", "route", "dispatch", "ffn", "combine"]
 
     def step(ev=None):
         sh, Ca = st.shape, st.C_alloc
@@ -243,8 +264,11 @@ def main():
         if ev: ev[3].record(stream)
         B.locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream)
         if ev: ev[4].record(stream)
-        B.locmoe_combine(sh, Ca, ysrc, st.slot, st.gate_w, st.out, False, stream)
+        if use_ffn:
+            B.locmoe_expert_ffn(sh, Ca, F, st.buf, w_in, w_out, h1, y, stream)
         if ev: ev[5].record(stream)
+        B.locmoe_combine(sh, Ca, ysrc, st.slot, st.gate_w, st.out, False, stream)
+        if ev: ev[6].record(stream)
 
     def barrier():
         if dist is not None:
@@ -257,7 +281,7 @@ def main():
 
     # ---- timed region: exactly K steps, device-timed, per-stage events on the launching stream ----
     K = args.steps
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(K)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(K)]
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
     barrier()
@@ -298,14 +322,24 @@ def main():
                 "path_bytes": sum(bytes_per_launch.values()),
                 "path_frac": sum(bytes_per_launch.values()) / (ms_per_step * 1e-3) / 1e9 / peak,
                 "kernels": kernels, "stage_ms": stage_ms}
+    if use_ffn:
+        # the expert FFN dominates: two grouped GEMMs, 2 * 2 * rows * H * F flops, tensor-core bound
+        flops = 4.0 * rows * w.H * F
+        tf = flops / (stage_ms["ffn"] * 1e-3) / 1e12
+        tpeak, tkind = measured_tensor_peak()
+        roofline.update({"bound": "tensor", "kernel": "ffn_gemm_kernel (two launches)", "achieved": tf, "peak": tpeak,
+                         "peak_kind": tkind, "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None, "flops": flops,
+                         "hbm_kernels": kernels})
 
     launches = B.locmoe_launch_counts(shape)
+    if use_ffn:
+        launches["ffn"] = 2
     launches_per_step = sum(launches.values())
     cap = B.locmoe_capacity_read(st.cap_dev)
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
     e2e = None
-    if args.e2e_steps > 0:
+    if args.e2e_steps > 0 and not use_ffn:
         xh = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
         xh.copy_(x)
         srch = torch.empty(src.shape, dtype=src.dtype, pin_memory=True)
