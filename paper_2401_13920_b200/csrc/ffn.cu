@@ -8,9 +8,9 @@
 //   - one elected thread issues tcgen05.mma (128 x 256 x 16 per instruction, fp32 accumulators in TMEM),
 //   - two 128x256 accumulators (512 TMEM columns) alternate, so the epilogue of a tile overlaps the MMAs
 //     of the next one,
-//   - four epilogue warps read the accumulator with tcgen05.ld (one row per thread), apply GeLU (first GEMM),
-//     convert and store.
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = epilogue.  Persistent CTAs, one per SM.
+//   - eight epilogue warps read the accumulator with tcgen05.ld (one row per thread, half of the columns per
+//     warp), apply GeLU (first GEMM), convert and store.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = epilogue.  Persistent CTAs, one per SM.
 // Every barrier wait is bounded; on a timeout the kernel raises the device diagnostics flag, leaves its
 // loops, frees its TMEM and returns.
 #include <cuda.h>
@@ -27,7 +27,8 @@ namespace {
 constexpr int BM = 128, BN = 256, BK = 64, NSTAGE = 4;
 constexpr int UMMA_K = 16;
 constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int kFfnThreads = 192;
+constexpr int kEpiWarps = 8;                       // two warps per TMEM lane quadrant, each takes half of the columns
+constexpr int kFfnThreads = 64 + 32 * kEpiWarps;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr size_t kFfnSmem = (size_t)NSTAGE * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
@@ -85,6 +86,14 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// 32-byte store: one full sector per lane (rows of the output are far apart, so a warp store touches 32 sectors;
+// writing each of them whole avoids partial-sector writes in L2).  Needs a 32-byte aligned address.
+__device__ __forceinline__ void st_global_v8(void* p, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t a4,
+                                             uint32_t a5, uint32_t a6, uint32_t a7) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(a0), "r"(a1), "r"(a2), "r"(a3),
+                 "r"(a4), "r"(a5), "r"(a6), "r"(a7) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -100,7 +109,21 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)); }
+// GeLU(v) = v * Phi(v) with Phi(v) = 1 - 0.5 erfc(v / sqrt 2).  erfc(x) = P(t) exp(-x^2), t = 1 / (1 + p x), for
+// x >= 0 by the five-term rational approximation of Abramowitz & Stegun 7.1.26 (absolute error below 1.5e-7,
+// far under the bf16 rounding of the result); the negative side uses erfc(-x) = 2 - erfc(x) written so that a
+// small Phi is not formed by cancellation.  About half the instructions of erff().
+__device__ __forceinline__ float gelu_erf(float v) {
+    const float x = fabsf(v) * 0.70710678118654752f;
+    const float t = __frcp_rn(fmaf(0.3275911f, x, 1.0f));
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    const float half_erfc = 0.5f * poly * t * exp2f(-1.4426950408889634f * x * x);   // 0.5 erfc(|v| / sqrt 2)
+    const float phi = v < 0.0f ? half_erfc : 1.0f - half_erfc;
+    return v * phi;
+}
 
 __global__ void __launch_bounds__(kFfnThreads, 1)
 ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const FfnArgs a) {
@@ -118,7 +141,7 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kEpiWarps); }
         *abort_word = 0;
         mbar_init_fence();
     }
@@ -180,8 +203,9 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
         }
-    } else {  // ---- epilogue warps 2..5: TMEM lane quadrant = warp % 4 ----
+    } else {  // ---- epilogue warps 2..9: TMEM lane quadrant = warp % 4, column half = (warp - 2) / 4 ----
         const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
         int acc = 0; uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             const int e = tile / tiles_per_expert, rem = tile - e * tiles_per_expert;
@@ -192,8 +216,9 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const bool row_ok = r_in < a.M;
             const long long grow = (long long)e * a.M + r_in;
             const int n0 = nt * BN;
+            const bool wide_ok = (a.N % 16 == 0) && ((uintptr_t)a.out % 32 == 0);
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
                 __syncwarp();  // tcgen05.ld is warp-collective: reconverge after the masked stores
                 uint32_t r[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
@@ -205,26 +230,35 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     v[i] = __uint_as_float(r[i]);
                     if (a.gelu) v[i] = gelu_erf(v[i]);
                 }
-                if (col0 + 32 <= a.N) {
+                if (col0 + 32 <= a.N && wide_ok) {
                     if (a.out_f32) {
-                        uint4* dst = reinterpret_cast<uint4*>(static_cast<float*>(a.out) + grow * a.N + col0);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            dst[i] = make_uint4(__float_as_uint(v[4 * i]), __float_as_uint(v[4 * i + 1]),
-                                                __float_as_uint(v[4 * i + 2]), __float_as_uint(v[4 * i + 3]));
-                    } else {
-                        uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(a.out) + grow * a.N + col0);
+                        float* dst = static_cast<float*>(a.out) + grow * a.N + col0;
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            dst[i] = make_uint4(cvt_bf16x2(make_float2(v[8 * i], v[8 * i + 1])),
-                                                cvt_bf16x2(make_float2(v[8 * i + 2], v[8 * i + 3])),
-                                                cvt_bf16x2(make_float2(v[8 * i + 4], v[8 * i + 5])),
-                                                cvt_bf16x2(make_float2(v[8 * i + 6], v[8 * i + 7])));
+                            st_global_v8(dst + 8 * i, __float_as_uint(v[8 * i]), __float_as_uint(v[8 * i + 1]),
+                                         __float_as_uint(v[8 * i + 2]), __float_as_uint(v[8 * i + 3]),
+                                         __float_as_uint(v[8 * i + 4]), __float_as_uint(v[8 * i + 5]),
+                                         __float_as_uint(v[8 * i + 6]), __float_as_uint(v[8 * i + 7]));
+                    } else {
+                        uint16_t* dst = static_cast<uint16_t*>(a.out) + grow * a.N + col0;
+#pragma unroll
+                        for (int i = 0; i < 2; ++i)
+                            st_global_v8(dst + 16 * i, cvt_bf16x2(make_float2(v[16 * i], v[16 * i + 1])),
+                                         cvt_bf16x2(make_float2(v[16 * i + 2], v[16 * i + 3])),
+                                         cvt_bf16x2(make_float2(v[16 * i + 4], v[16 * i + 5])),
+                                         cvt_bf16x2(make_float2(v[16 * i + 6], v[16 * i + 7])),
+                                         cvt_bf16x2(make_float2(v[16 * i + 8], v[16 * i + 9])),
+                                         cvt_bf16x2(make_float2(v[16 * i + 10], v[16 * i + 11])),
+                                         cvt_bf16x2(make_float2(v[16 * i + 12], v[16 * i + 13])),
+                                         cvt_bf16x2(make_float2(v[16 * i + 14], v[16 * i + 15])));
                     }
-                } else {  // ragged last column block
-                    for (int i = 0; i < 32 && col0 + i < a.N; ++i) {
-                        if (a.out_f32) static_cast<float*>(a.out)[grow * a.N + col0 + i] = v[i];
-                        else static_cast<uint16_t*>(a.out)[grow * a.N + col0 + i] = (uint16_t)f32_to_bf16_bits(v[i]);
+                } else {  // ragged or unaligned column block (static indexing keeps v[] in registers)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        if (col0 + i < a.N) {
+                            if (a.out_f32) static_cast<float*>(a.out)[grow * a.N + col0 + i] = v[i];
+                            else static_cast<uint16_t*>(a.out)[grow * a.N + col0 + i] = (uint16_t)f32_to_bf16_bits(v[i]);
+                        }
                     }
                 }
             }
