@@ -41,6 +41,8 @@ def parse_args():
     ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=12)
+    ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
+    ap.add_argument("--event-every", type=int, default=8, help="carry per-stage CUDA events on every n-th timed step")
     ap.add_argument("--no-ffn", action="store_true", help="config 5 only: identity experts instead of the expert FFN")
     ap.add_argument("--ffn-inner", type=int, default=10240, help="config 5: inner size F of the expert FFN")
     ap.add_argument("--tokens", type=int, default=0, help="override T (profiling-sized case; not the metric's workload)")
@@ -250,25 +252,31 @@ def main():
     ysrc = st.buf if y is None else y
 
     stream = torch.cuda.current_stream()
-    stages = ["gate", "capacity", "route", "dispatch", "ffn", "combine"]
+    stages = ["gate", "capacity", "route", "dispatch"] + (["ffn"] if use_ffn else []) + ["combine"]
 
     def step(ev=None):
         sh, Ca = st.shape, st.C_alloc
-        if ev: ev[0].record(stream)
+        i = 0
+        def mark():
+            nonlocal i
+            if ev:
+                ev[i].record(stream)
+            i += 1
+        mark()
         B.locmoe_gate(sh, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
-        if ev: ev[1].record(stream)
+        mark()
         B.locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
-        if ev: ev[2].record(stream)
+        mark()
         B.locmoe_route(sh, st.idx, src, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
                        st.send_counts, st.load, st.locality, st.status, st.ws, stream)
-        if ev: ev[3].record(stream)
+        mark()
         B.locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream)
-        if ev: ev[4].record(stream)
+        mark()
         if use_ffn:
             B.locmoe_expert_ffn(sh, Ca, F, st.buf, w_in, w_out, h1, y, stream)
-        if ev: ev[5].record(stream)
+            mark()
         B.locmoe_combine(sh, Ca, ysrc, st.slot, st.gate_w, st.out, False, stream)
-        if ev: ev[6].record(stream)
+        mark()
 
     def barrier():
         if dist is not None:
@@ -279,9 +287,28 @@ def main():
         step()
     barrier()
 
-    # ---- timed region: exactly K steps, device-timed, per-stage events on the launching stream ----
+    # ---- timed region: exactly K steps, device-timed.  The step is captured once in a CUDA graph and replayed;
+    #      every EV-th step is launched eagerly instead, with CUDA events between its stages on the launching
+    #      stream (an event record costs ~2.5 us of stream time, so only a sample of the steps carries them) ----
     K = args.steps
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(K)]
+    EV = max(1, args.event_every)
+    graph = None
+    if not args.no_graph:
+        side = torch.cuda.Stream(dev)
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            stream_backup = stream
+            stream = side
+            step()                     # one eager pass on the capture stream (lazy initialisation outside capture)
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                step()
+            stream = stream_backup
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+    n_ev = (K + EV - 1) // EV
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(n_ev)]
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
     barrier()
@@ -289,7 +316,10 @@ def main():
     t_end = torch.cuda.Event(enable_timing=True)
     t_start.record(stream)
     for k in range(K):
-        step(evs[k])
+        if k % EV == 0 or graph is None:
+            step(evs[k // EV] if k % EV == 0 else None)
+        else:
+            graph.replay()
     t_end.record(stream)
     barrier()
     clocks = sampler.stop()
@@ -297,8 +327,7 @@ def main():
     ms_per_step = total_ms / K
     value = world * w.T * K / (total_ms * 1e-3)
 
-    stage_ms = {s: float(np.mean([evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(K)])) for i, s in enumerate(stages)}
-
+    stage_ms = {s: float(np.mean([evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(n_ev)])) for i, s in enumerate(stages)}
     # ---- algorithmic bytes per launch (per token: see the per-kernel byte model in the design notes) ----
     kept = int((st.slot >= 0).sum().item())
     bx = x.element_size()
@@ -393,6 +422,8 @@ def main():
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic", "config": workload_config(w, args),
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "launches_per_step": launches,
+            "launch_mode": ("CUDA graph replay of the step; every %d-th step eager with per-stage events" % EV)
+                           if graph is not None else "eager",
             "roofline": roofline, "cpu_baseline": cpu_baseline,
             "routing": {"kept_fraction": kept / w.T, "C_local": cap.C_local, "C_expert": cap.C_expert, "delta": cap.delta,
                         "ec_min": cap.ec_min, "rows": rows, "kept_tokens_per_s": value * kept / w.T},

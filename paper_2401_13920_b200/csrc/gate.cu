@@ -9,6 +9,7 @@
 // The next chunk of loads (possibly of the warp's next row) is always in
 // flight while the current one is being reduced.
 #include <math.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -107,7 +108,7 @@ __device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gs
 // DT: token dtype.  U: elements per unit.  CH: vectors per lane per chunk.
 // EXACT: the row is a whole number of chunks (no bounds tests in the loop).
 template <int DT, int U, int CH, bool EXACT>
-__global__ void __launch_bounds__(256) gate_vec_kernel(const GateArgs a) {
+__global__ void __launch_bounds__(256, 4) gate_vec_kernel(const GateArgs a) {
     constexpr int NP = Vec<DT>::NP;
     constexpr int VE = 2 * NP;
     constexpr int UPV = VE / U;  // units per vector
