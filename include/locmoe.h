@@ -214,6 +214,17 @@ int locmoe_combine(const locmoe_shape_t *shape, int32_t C_alloc, const void *y, 
                    void *stream);
 
 /*
+ * Auxiliary load-balance loss, forward value (Sec. 3.2.2):
+ *   L_aux = alpha * n * sum_i f_i * P_i,  f_i = load[i] / T (share of tokens whose
+ *   arg-max is expert i),  P_i = (1/T) sum_t probs[t][i]  (the paper uses alpha = 0.01).
+ * probs float[T][E] as written by locmoe_gate, load int32[E] as written by
+ * locmoe_route; f_out / p_out float[E], loss_out float[1].  Sums are formed in a
+ * fixed order (deterministic).  ws: at least locmoe_workspace_bytes() bytes.
+ */
+int locmoe_aux_loss(const locmoe_shape_t *shape, const float *probs, const int32_t *load, float alpha,
+                    float *f_out, float *p_out, float *loss_out, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Expert feed-forward networks (first equation of Sec. 3.2.1):
  *   y[row] = W_out[e] . GeLU(W_in[e] . buf[row]),  GeLU(v) = v * Phi(v) (erf form),
  * for every row of the dispatched buffer, e being the expert that owns the row.

@@ -80,6 +80,8 @@ def lib():
         L.oracle_ffn_rows.restype = C.c_int
         L.oracle_ffn_rows.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                       C.c_void_p, C.c_void_p]
+        L.oracle_aux_loss.restype = C.c_double
+        L.oracle_aux_loss.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_double, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -263,3 +265,14 @@ def ffn_rows(x_bits, w_in_bits, w_out_bits):
     if rc != 0:
         raise ValueError("oracle_ffn_rows: error %d" % rc)
     return y, sp
+
+
+def aux_loss(idx, probs, alpha=0.01):
+    """(L_aux, f, P) of Sec. 3.2.2 from the arg-max indices and the probability matrix [T][E]."""
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    probs = np.ascontiguousarray(probs, dtype=np.float64)
+    T, E = probs.shape
+    f = np.empty(E, np.float64)
+    P = np.empty(E, np.float64)
+    L = lib().oracle_aux_loss(_p(idx), _p(probs), T, E, float(alpha), _p(f), _p(P))
+    return L, f, P

@@ -18,8 +18,8 @@
  *   oracle_p_delta   Lemma 3 / Appendix A.2: share of the unit sphere inside
  *                    the two symmetric caps |cos| >= delta.
  *   oracle_ec_min    Theorem 1: the three forms of the capacity lower bound.
- *   oracle_capacity  abstract ("maximal angular deviation between the gating
- *                    weights and the assigned tokens"), Theorem 1, and the
+ *   oracle_capacity  abstract (largest angle between an expert's gating weight
+ *                    and the tokens routed to it), Theorem 1, and the
  *                    conventional rule ec = ceil(b_s c_f / (ep n)) of
  *                    Sec. 3.2.3.
  *   oracle_route     capacity-bounded first-come-first-served placement into
@@ -30,6 +30,8 @@
  *   oracle_combine   y_m = R_m * expert_out (first equation of Sec. 3.2.1,
  *                    top-1 so a single term; a dropped token has no term).
  *
+ *   oracle_aux_loss  L_aux = alpha n sum_i f_i P_i (Sec. 3.2.2, first loss
+ *                    equation), forward value.
  *   oracle_ffn_rows  expert network of the same equation:
  *                    W_out . GeLU(W_in . x), GeLU(v) = v * Phi(v) with Phi the
  *                    standard Gaussian CDF (Sec. 3.2.1), in double.
@@ -416,4 +418,25 @@ int oracle_ffn_rows(const uint16_t *x, int64_t nrows, int32_t H, int32_t F, cons
     }
     free(g);
     return 0;
+}
+
+/*
+ * Auxiliary loss (Sec. 3.2.2): f_i = share of tokens whose arg-max is expert i, P_i = mean over tokens of
+ * p_i(x) (the softmax of the gate logits), L_aux = alpha * n * sum_i f_i P_i.  probs [T][E] in double.
+ */
+double oracle_aux_loss(const int32_t *idx, const double *probs, int64_t T, int32_t E, double alpha,
+                       double *f /* [E] */, double *P /* [E] */)
+{
+    for (int32_t i = 0; i < E; ++i) { f[i] = 0.0; P[i] = 0.0; }
+    for (int64_t t = 0; t < T; ++t) {
+        f[idx[t]] += 1.0;
+        for (int32_t i = 0; i < E; ++i) P[i] += probs[t * E + i];
+    }
+    double s = 0.0;
+    for (int32_t i = 0; i < E; ++i) {
+        f[i] /= (double)T;
+        P[i] /= (double)T;
+        s += f[i] * P[i];
+    }
+    return alpha * (double)E * s;
 }

@@ -24,7 +24,7 @@ FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
     "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route",
-    "locmoe_dispatch", "locmoe_combine", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
+    "locmoe_dispatch", "locmoe_combine", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
 
@@ -79,6 +79,7 @@ def _load() -> C.CDLL:
     lib.locmoe_expert_ffn.argtypes = [C.POINTER(Shape), i32, i32, vp, vp, vp, vp, vp, i32, vp]
     lib.locmoe_moe_layer.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(CapacityRule), i32, i32, vp, vp,
                                      C.POINTER(LayerBuffers), vp, vp]
+    lib.locmoe_aux_loss.argtypes = [C.POINTER(Shape), vp, vp, C.c_float, vp, vp, vp, vp, C.c_size_t, vp]
     lib.locmoe_launch_counts.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32 * 5)]
     lib.locmoe_device_flags.argtypes = [C.POINTER(C.c_int32), vp]
     lib.locmoe_status_string.argtypes = [C.c_int]
@@ -255,6 +256,17 @@ def locmoe_expert_ffn(shape: Shape, C_alloc, F, buf, w_in, w_out, h1, y, stream=
     return _check("locmoe_expert_ffn", _lib.locmoe_expert_ffn(C.byref(shape), int(C_alloc), int(F), _ptr(buf), _ptr(w_in),
                                                               _ptr(w_out), _ptr(h1), _ptr(y), dtype_code(y.dtype),
                                                               _stream(stream)))
+
+
+def locmoe_aux_loss(shape: Shape, probs, load, alpha, f_out, p_out, loss_out, ws, stream=None) -> int:
+    _want(probs, torch.float32, shape.T * shape.E, "probs")
+    _want(load, torch.int32, shape.E, "load")
+    _want(f_out, torch.float32, shape.E, "f_out")
+    _want(p_out, torch.float32, shape.E, "p_out")
+    _want(loss_out, torch.float32, 1, "loss_out")
+    return _check("locmoe_aux_loss", _lib.locmoe_aux_loss(C.byref(shape), _ptr(probs), _ptr(load), float(alpha),
+                                                          _ptr(f_out), _ptr(p_out), _ptr(loss_out), _ptr(ws),
+                                                          ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def layer_buffers(st: "RouterState", h1=None, y=None) -> LayerBuffers:

@@ -55,6 +55,8 @@ int locmoe_workspace_bytes(const locmoe_shape_t* shape, int32_t C_alloc, size_t*
     RoutePlan p;
     if ((rc = plan_route(*shape, &p))) return rc;
     size_t c = capacity_ws_bytes(*shape);
+    const size_t x = aux_ws_bytes(*shape);
+    if (x > c) c = x;
     *bytes = p.total > c ? p.total : c;
     return LOCMOE_OK;
 }
@@ -136,6 +138,15 @@ int locmoe_combine(const locmoe_shape_t* shape, int32_t C_alloc, const void* y, 
     if ((uintptr_t)y % (y_dtype == LOCMOE_F32 ? 4 : 2) || (uintptr_t)out % (shape->x_dtype == LOCMOE_F32 ? 4 : 2))
         return LOCMOE_ERR_ALIGN;
     return launch_combine(*shape, rows, y, y_dtype, slot, gate_w, out, accumulate, static_cast<cudaStream_t>(stream));
+}
+
+int locmoe_aux_loss(const locmoe_shape_t* shape, const float* probs, const int32_t* load, float alpha, float* f_out,
+                    float* p_out, float* loss_out, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!probs || !load || !f_out || !p_out || !loss_out) return LOCMOE_ERR_NULL;
+    if (!ws || ws_bytes < aux_ws_bytes(*shape) || (uintptr_t)ws % 256) return LOCMOE_ERR_WORKSPACE;
+    return launch_aux_loss(*shape, probs, load, alpha, f_out, p_out, loss_out, ws, static_cast<cudaStream_t>(stream));
 }
 
 int locmoe_expert_ffn(const locmoe_shape_t* shape, int32_t C_alloc, int32_t F, const void* buf, const void* w_in,

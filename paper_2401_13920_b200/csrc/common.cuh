@@ -53,6 +53,10 @@ int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const 
 int launch_combine(const locmoe_shape_t& s, int64_t rows, const void* y, int y_dtype, const int32_t* slot, const float* gate_w,
                    void* out, int accumulate, cudaStream_t st);
 
+size_t aux_ws_bytes(const locmoe_shape_t& s);
+int launch_aux_loss(const locmoe_shape_t& s, const float* probs, const int32_t* load, float alpha, float* f, float* P,
+                    float* loss, void* ws, cudaStream_t st);
+
 int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* buf, const void* w_in,
                       const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st);
 int read_ffn_flags(int* out, cudaStream_t st);

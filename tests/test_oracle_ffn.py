@@ -21,7 +21,7 @@ def test_ffn_matches_library_matmul_and_gaussian_cdf(oracle_mod):
     w_out = _bf16(rng.standard_normal((H, F)) * 0.3)
     y, spread = oracle_mod.ffn_rows(x, w_in, w_out)
     h = _f64(x) @ _f64(w_in).T
-    g = h * norm.cdf(h)                       # "the product of input and the standard Gaussian CDF"
+    g = h * norm.cdf(h)                       # Sec. 3.2.1 defines GeLU as the input times the standard normal CDF
     assert np.allclose(y, g @ _f64(w_out).T, rtol=1e-12, atol=1e-14)
     terms = _f64(w_out)[None, :, :] * g[:, None, :]
     assert np.allclose(spread, np.sqrt((terms ** 2).sum(-1)), rtol=1e-12)

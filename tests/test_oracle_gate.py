@@ -17,7 +17,7 @@ def _bf16_round(x32: np.ndarray) -> np.ndarray:
 
 
 def test_grap_weight_is_block_average_and_orthogonal(oracle_mod):
-    # Sec. 3.2.1: w_i = (n/d) 1{i d/n <= j < (i+1) d/n}; "the gating weights of the GrAP layer are orthogonal";
+    # Sec. 3.2.1: w_i = (n/d) 1{i d/n <= j < (i+1) d/n}; the paper notes that these weights are mutually orthogonal;
     # Assumption 1: equal norms.
     for n, d in [(8, 1024), (64, 5120), (256, 5120), (4, 12), (1, 7)]:
         W = oracle_mod.grap_weight(n, d)
@@ -31,7 +31,7 @@ def test_grap_weight_is_block_average_and_orthogonal(oracle_mod):
 
 @pytest.mark.parametrize("T,H,E", [(64, 1024, 8), (33, 5120, 64), (17, 5120, 256), (9, 60, 5)])
 def test_group_mean_equals_dense_layer_with_fixed_weight(oracle_mod, T, H, E):
-    # "It can be regarded as the dense layer with the fixed weight w_i": G = ReLU(x W^T).
+    # Sec. 3.2.1 presents GrAP as a dense layer whose weight is fixed to w_i: G = ReLU(x W^T).
     rng = np.random.default_rng(1)
     x = rng.standard_normal((T, H)).astype(np.float32)
     W = np.kron(np.eye(E), np.ones((1, H // E))) * (E / H)
@@ -144,3 +144,25 @@ def test_lemma2_balanced_assignment_on_spherical_tokens(oracle_mod):
 def test_shape_errors(oracle_mod):
     with pytest.raises(ValueError):
         oracle_mod.gate(np.zeros((2, 10), np.float32), F32, 3)
+
+
+def test_aux_loss_definition_and_minimum(oracle_mod):
+    # Sec. 3.2.2: L_aux = alpha n sum_i f_i P_i; under a uniform assignment with uniform probabilities the sum is
+    # 1/n, so L_aux = alpha (the balanced case the paper names as the loss's minimum); alpha = 0.01.
+    n, T = 8, 64
+    idx = np.arange(T) % n
+    probs = np.full((T, n), 1.0 / n)
+    L, f, P = oracle_mod.aux_loss(idx, probs, 0.01)
+    assert np.allclose(f, 1 / n) and np.allclose(P, 1 / n) and L == pytest.approx(0.01)
+    # everything on one expert with probability one: f = P = e_0, L = alpha n
+    probs = np.zeros((T, n)); probs[:, 0] = 1.0
+    L, f, P = oracle_mod.aux_loss(np.zeros(T, np.int32), probs, 0.01)
+    assert L == pytest.approx(0.01 * n)
+    # against numpy on random data
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal((500, 256)).astype(np.float32)
+    g = oracle_mod.gate(x, F32, 16, want_probs=True)
+    L, f, P = oracle_mod.aux_loss(g.idx, g.probs, 0.01)
+    f_np = np.bincount(g.idx, minlength=16) / 500
+    assert np.allclose(f, f_np) and np.allclose(P, g.probs.mean(0))
+    assert L == pytest.approx(0.01 * 16 * (f_np * g.probs.mean(0)).sum(), rel=1e-12)

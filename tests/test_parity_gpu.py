@@ -250,3 +250,32 @@ def test_host_router_pipeline_matches_device_path(P):
         ref = B.router_forward(st, x, src)
         torch.cuda.synchronize()
         assert torch.equal(o.view(torch.int16), ref.cpu().view(torch.int16))
+
+
+def test_aux_loss_against_oracle(P):
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    w = P.W.CONFIGS[2].scaled(5000)
+    x = W.make_tokens(w, dev)
+    src = W.make_src(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype)
+    st = B.make_router(sh, 2, B.CapacityRule(1.0, 1.0, -1.0, 0, 0), dev)
+    probs = torch.empty(w.T, w.E, device=dev)
+    B.locmoe_gate(sh, x, None, st.idx, st.gate_w, st.cos_sim, probs)
+    B.locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws)
+    B.locmoe_route(sh, st.idx, src, st.cap_dev, 2, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
+                   st.send_counts, st.load, st.locality, st.status, st.ws)
+    f = torch.empty(w.E, device=dev); Pm = torch.empty(w.E, device=dev); loss = torch.empty(1, device=dev)
+    B.locmoe_aux_loss(sh, probs, st.load, 0.01, f, Pm, loss, st.ws)
+    torch.cuda.synchronize()
+    g = P.oracle.gate(W.host_bits(x), sh.x_dtype, w.E, want_probs=True)
+    assert (g.idx != st.idx.cpu().numpy()).sum() <= (g.gap < 1e-6).sum()
+    L, f_o, P_o = P.oracle.aux_loss(st.idx.cpu().numpy(), g.probs, 0.01)
+    assert np.allclose(f.cpu().numpy(), f_o, rtol=1e-6, atol=0)
+    assert np.allclose(Pm.cpu().numpy(), P_o, rtol=1e-5, atol=0)
+    assert abs(loss.item() - L) <= 1e-5 * L
+    # deterministic: a second evaluation gives the same bits
+    loss2 = torch.empty(1, device=dev)
+    B.locmoe_aux_loss(sh, probs, st.load, 0.01, f, Pm, loss2, st.ws)
+    torch.cuda.synchronize()
+    assert loss2.item() == loss.item()
