@@ -1,0 +1,74 @@
+"""The All-to-All around the experts (Sec. 3.2.4), as plain collectives: send-side buffer -> receive-side buffer.
+
+`locmoe_route` / `locmoe_dispatch` fill a buffer whose rows are grouped by (source device, destination in
+"self, own node, other nodes" order); the expert FFN wants the receive-side grouping (expert, source).  On one GPU
+both are just layouts.  With one process per GPU, each owning a contiguous block of the logical devices, this module
+moves the rows between the two layouts with ONE equal-split ``all_to_all_single`` per direction (NCCL over
+NVLink/NVSwitch on GPUs, gloo on CPU in the tests).  Only integer permutations of fixed-size cells (C_alloc rows)
+happen here; no router arithmetic.  This is the library-collective baseline for the exchange step, not a fused
+compute+communication kernel.
+"""
+from __future__ import annotations
+
+import torch
+import torch.distributed as dist
+
+
+def dest_rank_order(a: int, b: int, n_nodes: int, dev_per_node: int) -> int:
+    """Position of device b in device a's destination list: a itself, the rest of a's node, then the other nodes."""
+    return ((b // dev_per_node - a // dev_per_node) % n_nodes) * dev_per_node + ((b % dev_per_node - a % dev_per_node) % dev_per_node)
+
+
+class ExchangePlan:
+    """Cell permutations for one rank.  A cell is the block of C_alloc rows of one (source device, expert) pair."""
+
+    def __init__(self, n_nodes: int, dev_per_node: int, E: int, world: int, rank: int):
+        D = n_nodes * dev_per_node
+        if D % world or E % D:
+            raise ValueError("devices must divide over ranks and experts over devices")
+        per, Ed = D // world, E // D
+        a0 = rank * per
+        self.D, self.Ed, self.per, self.world, self.rank = D, Ed, per, world, rank
+        self.cells_local = per * D * Ed            # cells of this rank in either layout
+        r = lambda a, b: dest_rank_order(a, b, n_nodes, dev_per_node)
+        # send order: destination rank q, then source device a (mine), then destination device b (q's), then local expert
+        send = []
+        for q in range(world):
+            for a in range(a0, a0 + per):
+                for b in range(q * per, (q + 1) * per):
+                    for el in range(Ed):
+                        send.append(((a - a0) * D + r(a, b)) * Ed + el)          # SEND cell ((a, r(a,b)), el), local to me
+        # what arrives: source rank p, then source device a (p's), then destination device b (mine), then local expert;
+        # it belongs at RECV cell ((b, el), r(b, a)), local to me
+        recv = []
+        for p in range(world):
+            for a in range(p * per, (p + 1) * per):
+                for b in range(a0, a0 + per):
+                    for el in range(Ed):
+                        recv.append(((b - a0) * Ed + el) * D + r(b, a))
+        self.send_cells = torch.tensor(send, dtype=torch.int64)
+        self.recv_cells = torch.tensor(recv, dtype=torch.int64)
+        assert sorted(send) == list(range(self.cells_local)) and sorted(recv) == list(range(self.cells_local))
+
+    def _cells(self, buf: torch.Tensor, C_alloc: int) -> torch.Tensor:
+        return buf.reshape(self.cells_local, C_alloc * buf.shape[-1])
+
+    def dispatch(self, send_local: torch.Tensor, C_alloc: int, group=None) -> torch.Tensor:
+        """Local slice of the SEND-layout buffer -> local slice of the RECV-layout buffer (rows of my experts)."""
+        cells = self._cells(send_local, C_alloc)
+        out_of_order = cells.index_select(0, self.send_cells.to(cells.device)).contiguous()
+        arrived = torch.empty_like(out_of_order)
+        dist.all_to_all_single(arrived, out_of_order, group=group)
+        recv = torch.empty_like(arrived)
+        recv.index_copy_(0, self.recv_cells.to(cells.device), arrived)
+        return recv.reshape(send_local.shape)
+
+    def combine(self, recv_local: torch.Tensor, C_alloc: int, group=None) -> torch.Tensor:
+        """The way back: expert outputs in RECV layout -> SEND layout on the ranks the tokens came from."""
+        cells = self._cells(recv_local, C_alloc)
+        leaving = cells.index_select(0, self.recv_cells.to(cells.device)).contiguous()
+        arrived = torch.empty_like(leaving)
+        dist.all_to_all_single(arrived, leaving, group=group)
+        send = torch.empty_like(arrived)
+        send.index_copy_(0, self.send_cells.to(cells.device), arrived)
+        return send.reshape(recv_local.shape)
