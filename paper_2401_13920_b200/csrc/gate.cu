@@ -215,6 +215,145 @@ __global__ void __launch_bounds__(256, 4) gate_vec_kernel(const GateArgs a) {
     }
 }
 
+// Specialised bf16 kernel for the common shapes: the row is a whole number of chunks, every lane owns exactly NGK
+// groups (E = 32 * NGK) of PUK units each.  With PUK and NGK known at compile time the strip needs neither padding
+// nor an offset table (a stride of PUK floats between lanes is at worst a 2-way bank conflict for the PUK values
+// instantiated; PUK % 4 == 0 is read with 16-byte loads), the group sums and logits stay in registers, and the
+// winner's raw sum for the cosine comes from a shuffle.  About half the instructions of the general kernel.
+template <int PUK>
+__device__ __forceinline__ float strip_sum(const float* pp) {
+    if constexpr (PUK % 4 == 0) {
+        float s = 0.0f;
+#pragma unroll
+        for (int k = 0; k < PUK / 4; ++k) {
+            const float4 v = reinterpret_cast<const float4*>(pp)[k];
+            s += (v.x + v.y) + (v.z + v.w);
+        }
+        return s;
+    } else if constexpr (PUK % 2 == 0) {
+        float s = 0.0f;
+#pragma unroll
+        for (int k = 0; k < PUK / 2; ++k) {
+            const float2 v = reinterpret_cast<const float2*>(pp)[k];
+            s += v.x + v.y;
+        }
+        return s;
+    } else {
+        float s = 0.0f;
+#pragma unroll
+        for (int k = 0; k < PUK; ++k) s += pp[k];
+        return s;
+    }
+}
+
+template <int U, int CH, int PUK, int NGK>
+__global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
+    constexpr int NP = 4, VE = 8, UPV = VE / U;
+    extern __shared__ float smem[];
+    const unsigned full = 0xffffffffu;
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int wpb = blockDim.x >> 5;
+    float* part = smem + (size_t)wib * a.warp_floats;
+    const int nw = gridDim.x * wpb;
+    const uint4* xv = reinterpret_cast<const uint4*>(a.x);
+    constexpr float kLog2e = 1.4426950408889634f;
+
+    uint4 bufA[CH], bufB[CH];
+    float2 sq2 = make_float2(0.0f, 0.0f);
+
+    auto load = [&](uint4 (&buf)[CH], int r, int c) {
+        const uint4* base = xv + (size_t)r * a.V + c * (CH * kWarp) + lane;
+#pragma unroll
+        for (int k = 0; k < CH; ++k) buf[k] = ld_stream(base + k * kWarp);
+    };
+
+    auto consume = [&](const uint4 (&buf)[CH], int c) {
+        float* dst = part + (c * (CH * kWarp) + lane) * UPV;
+#pragma unroll
+        for (int k = 0; k < CH; ++k) {
+            float2 p[NP];
+            Vec<LOCMOE_BF16>::unpack(buf[k], p);
+#pragma unroll
+            for (int e = 0; e < NP; ++e) sq2 = __ffma2_rn(p[e], p[e], sq2);
+            float* d = dst + k * kWarp * UPV;
+            if constexpr (U == 8) {
+                const float2 s2 = pair_tree<4>(p);
+                d[0] = s2.x + s2.y;
+            } else if constexpr (U == 4) {
+                const float2 lo = __fadd2_rn(p[0], p[1]), hi = __fadd2_rn(p[2], p[3]);
+                *reinterpret_cast<float2*>(d) = make_float2(lo.x + lo.y, hi.x + hi.y);
+            } else {  // U == 2
+                *reinterpret_cast<float4*>(d) = make_float4(p[0].x + p[0].y, p[1].x + p[1].y, p[2].x + p[2].y, p[3].x + p[3].y);
+            }
+        }
+    };
+
+    auto finish_row = [&](int row) {
+        __syncwarp();
+        float gs[NGK];
+#pragma unroll
+        for (int m = 0; m < NGK; ++m) gs[m] = strip_sum<PUK>(part + (size_t)(lane + 32 * m) * PUK);
+        __syncwarp();  // the strip may now be overwritten by the next row
+        // the logits are recomputed in the second pass rather than kept: fewer live registers, no spills
+        auto logit = [&](int m) { return fmaxf(fmaf(gs[m], a.inv_g, a.eps ? a.eps[lane + 32 * m] : 0.0f), 0.0f); };
+        float best = -1.0f;
+        int bi = 0x7fffffff;
+#pragma unroll
+        for (int m = 0; m < NGK; ++m) {
+            const float G = logit(m);
+            if (G > best) { best = G; bi = lane + 32 * m; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(full, best, o);
+            const int oi = __shfl_xor_sync(full, bi, o);
+            if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+        }
+        const float nb = -best * kLog2e;
+        float se = 0.0f;
+#pragma unroll
+        for (int m = 0; m < NGK; ++m) se += exp2f(fmaf(logit(m), kLog2e, nb));
+        float sq = sq2.x + sq2.y;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            se += __shfl_xor_sync(full, se, o);
+            sq += __shfl_xor_sync(full, sq, o);
+        }
+        float cand = gs[0];
+#pragma unroll
+        for (int m = 1; m < NGK; ++m) if ((bi >> 5) == m) cand = gs[m];
+        const float wsum = __shfl_sync(full, cand, bi & 31);
+        if (lane == 0) {
+            const float nrm = sqrtf(sq);
+            a.idx[row] = bi;
+            a.gate_w[row] = 1.0f / se;
+            a.cos_sim[row] = nrm > 0.0f ? wsum / (a.sqrt_g * nrm) : 0.0f;
+        }
+        sq2 = make_float2(0.0f, 0.0f);
+    };
+
+    int row = blockIdx.x * wpb + wib, ch = 0;
+    if (row >= a.T) return;
+    load(bufA, row, 0);
+    while (true) {
+        int ch2 = ch + 1, row2 = row;
+        if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
+        if (row2 < a.T) load(bufB, row2, ch2);
+        consume(bufA, ch);
+        if (ch2 == 0) finish_row(row);
+        if (row2 >= a.T) break;
+        row = row2; ch = ch2;
+
+        ch2 = ch + 1; row2 = row;
+        if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
+        if (row2 < a.T) load(bufA, row2, ch2);
+        consume(bufB, ch);
+        if (ch2 == 0) finish_row(row);
+        if (row2 >= a.T) break;
+        row = row2; ch = ch2;
+    }
+}
+
 // Fallback for rows that are not 16-byte friendly: plain element loads, one warp per row.
 template <int DT>
 __global__ void __launch_bounds__(256) gate_scalar_kernel(const GateArgs a) {
@@ -308,6 +447,25 @@ int launch_gate(const locmoe_shape_t& s, const void* x, const float* eps, int32_
     bool exact = whole && per_lane % 4 == 0;
     if (!exact && whole && per_lane % 5 == 0) { CH = 5; exact = true; }
     a.nch = (a.V + CH * kWarp - 1) / (CH * kWarp);
+    // specialised kernel for the common bf16 shapes (whole chunks, E a multiple of 32 with a known group layout);
+    // LOCMOE_GATE=general keeps the general kernel (testing aid)
+    if (s.x_dtype == LOCMOE_BF16 && exact && probs == nullptr && a.S == 1 && s.E % 32 == 0 &&
+        !(getenv("LOCMOE_GATE") && getenv("LOCMOE_GATE")[0] == 'g')) {
+        const int NG = s.E / 32;
+        GateArgs f = a;
+        f.warp_floats = (s.H / U + 3) & ~3;
+        f.tab_ints = 0;
+#define LOCMOE_FAST_CASE(UU, CC, PP, NN) \
+        if (U == UU && CH == CC && a.PU == PP && NG == NN) return launch_persistent(gate_fast_kernel<UU, CC, PP, NN>, f, 8, st);
+        LOCMOE_FAST_CASE(8, 4, 10, 2)   // H = 5120, E = 64
+        LOCMOE_FAST_CASE(8, 5, 10, 1)   // H = 2560, E = 32
+        LOCMOE_FAST_CASE(8, 4, 4, 4)    // H = 4096, E = 128
+        LOCMOE_FAST_CASE(4, 4, 5, 8)    // H = 5120, E = 256
+        LOCMOE_FAST_CASE(8, 4, 8, 2)    // H = 4096, E = 64
+        LOCMOE_FAST_CASE(4, 4, 7, 8)    // H = 7168, E = 256
+        LOCMOE_FAST_CASE(8, 4, 16, 1)   // H = 4096, E = 32
+#undef LOCMOE_FAST_CASE
+    }
 #define LOCMOE_GATE_CASE(DT, UU)                                                                              \
     if (s.x_dtype == DT && U == UU) {                                                                         \
         if (exact && CH == 4) return launch_persistent(gate_vec_kernel<DT, UU, 4, true>, a, 8, st);           \

@@ -86,6 +86,18 @@ def test_grid_path_shapes(P, grid_path, kw):
     P.run_staged(_wl(P, **kw), 1.0, layout=1, full=True)
 
 
+@pytest.mark.parametrize("cfg,T", [(2, 3001), (4, 2999)])
+def test_general_gate_kernel_on_the_common_shapes(P, monkeypatch, cfg, T):
+    # the common bf16 shapes normally take the specialised gate kernel; LOCMOE_GATE=general forces the general one
+    monkeypatch.setenv("LOCMOE_GATE", "general")
+    P.run_staged(P.W.CONFIGS[cfg].scaled(T), 1.0, full=True)
+
+
+@pytest.mark.parametrize("H,E", [(4096, 64), (7168, 256), (4096, 32)])
+def test_specialised_gate_kernel_other_shapes(P, H, E):
+    P.run_staged(_wl(P, T=1500, H=H, E=E, n_nodes=2, dev_per_node=4), 1.0, full=True)
+
+
 def test_bulk_copy_dispatch_variant(P, monkeypatch):
     # the TMA (cp.async.bulk) dispatch kernel: whole rows, split rows (> 16 KB), zero rows
     monkeypatch.setenv("LOCMOE_DISPATCH", "tma")
