@@ -3,7 +3,7 @@
 // Per-expert minimum of the token cosines (integer min on an order-preserving
 // encoding, so the result does not depend on scheduling), then a finish that
 // decodes the minima and evaluates the closed forms in fp64 on one thread.
-// Moderate batches run as ONE kernel on one thread-block cluster (hardware
+// Batches up to 262144 tokens run as ONE kernel on one thread-block cluster (hardware
 // cluster barrier between the two steps); large ones as memset + grid-wide
 // minimum + single-CTA finish.  Nothing is read back by the host.
 #include <math.h>
@@ -200,7 +200,7 @@ bool capacity_cluster_eligible(const locmoe_shape_t& s) {
     const char* o = getenv("LOCMOE_PATH");
     if (o && o[0] == 'g') return false;
     if (o && o[0] == 'c') return true;
-    return s.T <= (1 << 21);
+    return s.T <= (1 << 18);   // beyond that, eight CTAs take longer to read the tokens than two more launches cost
 }
 
 size_t capacity_ws_bytes(const locmoe_shape_t& s) { return ((size_t)kCapCS * s.E * sizeof(uint32_t) + 255) & ~(size_t)255; }

@@ -124,27 +124,40 @@ __global__ void __launch_bounds__(kThreads) route_hist0_kernel(const RouteArgs a
     for (int d = threadIdx.x; d < nbins; d += blockDim.x) a.hist[0][(size_t)d * a.ntiles + blockIdx.x] = sh[d];
 }
 
-// Exclusive scan of in[0..n) into out[0..n) by one CTA of kThreads threads (in == out allowed).
+// Exclusive scan of in[0..n) into out[0..n) by one CTA of kThreads threads (in == out allowed).  Every warp owns a
+// contiguous eighth of the array and walks it in coalesced 32-element tiles (first to total it, then to write the
+// running prefix), so that the single CTA streams the array instead of chasing per-thread chunks.
 __device__ void block_exclusive_scan(const int32_t* in, int32_t* out, int n) {
     __shared__ int warp_sums[kWarps];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    const int chunk = (n + kThreads - 1) / kThreads;
-    const int lo = min(tid * chunk, n), hi = min(lo + chunk, n);
+    const int per = ((n + kWarps - 1) / kWarps + 31) & ~31;   // multiple of 32 per warp
+    const int lo = min(w * per, n), hi = min(lo + per, n);
     int s = 0;
-    for (int i = lo; i < hi; ++i) s += in[i];
-    int incl = s;
+    for (int i = lo + lane; i < hi; i += 32) s += in[i];
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) warp_sums[w] = incl;
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) warp_sums[w] = s;
     __syncthreads();
-    int wbase = 0;
+    int run = 0;
 #pragma unroll
-    for (int ww = 0; ww < kWarps; ++ww) if (ww < w) wbase += warp_sums[ww];
-    int run = wbase + incl - s;
-    for (int i = lo; i < hi; ++i) { int v = in[i]; out[i] = run; run += v; }
+    for (int ww = 0; ww < kWarps; ++ww) if (ww < w) run += warp_sums[ww];
+    for (int i0 = lo; i0 < hi; i0 += 128) {
+        int v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { const int i = i0 + q * 32 + lane; v[q] = i < hi ? in[i] : 0; }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int incl = v[q];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += u;
+            }
+            const int i = i0 + q * 32 + lane;
+            if (i < hi) out[i] = run + incl - v[q];
+            run += __shfl_sync(0xffffffffu, incl, 31);
+        }
+    }
     __syncthreads();
 }
 
