@@ -1,4 +1,6 @@
 // C-ABI front end: argument validation on the host, then the kernel launchers.
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace locmoe {
@@ -16,6 +18,12 @@ int sm_count() {
         cached[dev] = n;
     }
     return cached[dev];
+}
+
+bool pdl_enabled() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("LOCMOE_PDL"); v = (e && e[0] == '0') ? 0 : 1; }
+    return v != 0;
 }
 
 namespace {

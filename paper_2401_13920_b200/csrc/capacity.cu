@@ -176,6 +176,8 @@ __global__ void __cluster_dims__(kCapCS, 1, 1) __launch_bounds__(kCapThreads, 1)
 capacity_cluster_kernel(const int32_t* __restrict__ idx, const float* __restrict__ cs, uint32_t* __restrict__ part,
                         int T, int E, int H, int D, locmoe_capacity_rule_t rule, float* __restrict__ delta_e,
                         float* __restrict__ theta_e, locmoe_capacity_t* __restrict__ cap) {
+    pdl_wait();
+    pdl_trigger();
     extern __shared__ uint32_t smin[];
     cg::cluster_group cluster = cg::this_cluster();
     const int cta = (int)cluster.block_rank();
@@ -210,9 +212,8 @@ int launch_capacity(const locmoe_shape_t& s, const int32_t* idx, const float* co
                     locmoe_capacity_t* cap_dev, void* ws, cudaStream_t st) {
     uint32_t* gmin = static_cast<uint32_t*>(ws);
     if (capacity_cluster_eligible(s)) {
-        capacity_cluster_kernel<<<kCapCS, kCapThreads, (size_t)s.E * sizeof(uint32_t), st>>>(
-            idx, cos_sim, gmin, s.T, s.E, s.H, s.n_nodes * s.dev_per_node, rule, delta_e, theta_e, cap_dev);
-        return check_launch();
+        return launch_pdl(capacity_cluster_kernel, kCapCS, kCapThreads, (size_t)s.E * sizeof(uint32_t), st, idx, cos_sim, gmin,
+                          s.T, s.E, s.H, s.n_nodes * s.dev_per_node, rule, delta_e, theta_e, cap_dev);
     }
     if (cudaMemsetAsync(gmin, 0xff, (size_t)s.E * sizeof(uint32_t), st) != cudaSuccess) {
         cudaGetLastError();

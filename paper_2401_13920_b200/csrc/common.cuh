@@ -64,6 +64,29 @@ int read_ffn_flags(int* out, cudaStream_t st);
 // Copies the device diagnostics word to host memory (synchronises the stream).
 int read_device_flags(int* out, cudaStream_t st);
 
+// ---- programmatic dependent launch: a kernel launched with launch_pdl() may be scheduled while its predecessor
+// on the stream is still draining; it must call pdl_wait() before it touches anything the predecessor wrote (all
+// kernels here do so first thing), which blocks until the predecessor has completed and flushed.  pdl_trigger()
+// lets the successor start its own launch early.  LOCMOE_PDL=0 in the environment turns the attribute off.
+bool pdl_enabled();
+
+template <typename... P, typename... A>
+inline int launch_pdl(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...) != cudaSuccess) { cudaGetLastError(); return LOCMOE_ERR_CUDA; }
+    return LOCMOE_OK;
+}
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
 // ---- small device helpers ----
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }

@@ -109,6 +109,8 @@ __device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gs
 // EXACT: the row is a whole number of chunks (no bounds tests in the loop).
 template <int DT, int U, int CH, bool EXACT>
 __global__ void __launch_bounds__(256, 4) gate_vec_kernel(const GateArgs a) {
+    pdl_wait();
+    pdl_trigger();
     constexpr int NP = Vec<DT>::NP;
     constexpr int VE = 2 * NP;
     constexpr int UPV = VE / U;  // units per vector
@@ -248,6 +250,8 @@ __device__ __forceinline__ float strip_sum(const float* pp) {
 
 template <int U, int CH, int PUK, int NGK>
 __global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
+    pdl_wait();
+    pdl_trigger();
     constexpr int NP = 4, VE = 8, UPV = VE / U;
     extern __shared__ float smem[];
     const unsigned full = 0xffffffffu;
@@ -357,6 +361,8 @@ __global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
 // Fallback for rows that are not 16-byte friendly: plain element loads, one warp per row.
 template <int DT>
 __global__ void __launch_bounds__(256) gate_scalar_kernel(const GateArgs a) {
+    pdl_wait();
+    pdl_trigger();
     extern __shared__ float smem[];
     const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -409,8 +415,7 @@ int launch_persistent(K kernel, const GateArgs& a, int max_warps, cudaStream_t s
     long long want = ((long long)a.T + wpb - 1) / wpb;
     long long grid = (long long)per_sm * sm_count();
     if (grid > want) grid = want;
-    kernel<<<(unsigned)grid, wpb * 32, smem, st>>>(a);
-    return check_launch();
+    return launch_pdl(kernel, (unsigned)grid, wpb * 32, smem, st, a);
 }
 
 }  // namespace

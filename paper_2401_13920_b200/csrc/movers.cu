@@ -23,6 +23,8 @@ constexpr int kThreads = 256;
 __global__ void __launch_bounds__(kThreads, 6) dispatch_vec_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ inv,
                                                                    uint4* __restrict__ buf, long long rows, int V, int T,
                                                                    int zero_pad) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31;
     const long long nw = (long long)gridDim.x * (blockDim.x >> 5);
     long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -158,6 +160,8 @@ template <int YDT, int ODT, bool ACC>
 __global__ void __launch_bounds__(kThreads, ACC ? 4 : 6) combine_vec_kernel(const void* __restrict__ y, const int32_t* __restrict__ slot,
                                                                const float* __restrict__ gate_w, void* __restrict__ out,
                                                                int T, int O, long long rows) {
+    pdl_wait();
+    pdl_trigger();
     constexpr int CH = 2;
     const int lane = threadIdx.x & 31;
     const int nw = gridDim.x * (blockDim.x >> 5);
@@ -278,8 +282,8 @@ int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const 
         }
     }
     if (vec_ok) {
-        dispatch_vec_kernel<<<grid, kThreads, 0, st>>>(static_cast<const uint4*>(x), inv, static_cast<uint4*>(buf), rows,
-                                                       (int)(rb / 16), s.T, zero_pad);
+        return launch_pdl(dispatch_vec_kernel, grid, kThreads, 0, st, static_cast<const uint4*>(x), inv, static_cast<uint4*>(buf),
+                          (long long)rows, (int)(rb / 16), s.T, zero_pad);
     } else if (esz == 4) {
         dispatch_scalar_kernel<uint32_t><<<grid, kThreads, 0, st>>>(static_cast<const uint32_t*>(x), inv,
                                                                     static_cast<uint32_t*>(buf), rows, s.H, s.T, zero_pad);
@@ -302,8 +306,8 @@ int launch_combine(const locmoe_shape_t& s, int64_t rows, const void* y, int y_d
     const int O = s.H / 8;
 #define LOCMOE_COMBINE_CASE(YD, OD, AC)                                                                              \
     if (y_dtype == YD && s.x_dtype == OD && (accumulate != 0) == AC) {                                               \
-        combine_vec_kernel<YD, OD, AC><<<grid, kThreads, 0, st>>>(y, slot, gate_w, out, s.T, O, rows);               \
-        return check_launch();                                                                                       \
+        return launch_pdl(combine_vec_kernel<YD, OD, AC>, grid, kThreads, 0, st, y, slot, gate_w, out, s.T, O, (long long)rows); \
+                                                                                     \
     }
     LOCMOE_COMBINE_CASE(LOCMOE_F32, LOCMOE_F32, false)
     LOCMOE_COMBINE_CASE(LOCMOE_F32, LOCMOE_F32, true)

@@ -89,6 +89,8 @@ __device__ __forceinline__ void route_emit(const RouteArgs& a, int k, int t, int
 }
 
 __global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a) {
+    pdl_wait();
+    pdl_trigger();
     const long long stride = (long long)gridDim.x * blockDim.x;
     const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     for (long long i = i0; i < a.rows; i += stride) a.inv[i] = -1;
@@ -104,6 +106,8 @@ __global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a)
 }
 
 __global__ void __launch_bounds__(kThreads) route_hist0_kernel(const RouteArgs a) {
+    pdl_wait();
+    pdl_trigger();
     extern __shared__ int sh[];
     const int nbins = 1 << a.bits[0];
     for (int d = threadIdx.x; d < nbins; d += blockDim.x) sh[d] = 0;
@@ -202,6 +206,8 @@ __device__ void route_extras(const RouteArgs& a, int x, int nx) {
 }
 
 __global__ void __launch_bounds__(kThreads) route_extras_kernel(const RouteArgs a) {
+    pdl_wait();
+    pdl_trigger();
     route_extras(a, blockIdx.x, gridDim.x);
 }
 
@@ -209,6 +215,8 @@ __global__ void __launch_bounds__(kThreads) route_extras_kernel(const RouteArgs 
 // and stores the row totals, one warp per row, so that a scatter CTA reads one entry per digit instead of a
 // whole row (total work O(bins x tiles) instead of O(bins x tiles^2)).
 __global__ void __launch_bounds__(kThreads) route_prescan_kernel(const RouteArgs a, int pass) {
+    pdl_wait();
+    pdl_trigger();
     const int nbins = 1 << a.bits[pass];
     const int lane = threadIdx.x & 31;
     const int d = blockIdx.x * kWarps + (threadIdx.x >> 5);
@@ -232,6 +240,8 @@ __global__ void __launch_bounds__(kThreads) route_prescan_kernel(const RouteArgs
 // One radix pass over one tile per CTA; CTAs beyond ntiles run the extras.
 template <bool FIRST, bool LAST>
 __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs a, int pass, int shift) {
+    pdl_wait();
+    pdl_trigger();
     if ((int)blockIdx.x >= a.ntiles) {
         route_extras(a, blockIdx.x - a.ntiles, gridDim.x - a.ntiles);
         return;
@@ -464,33 +474,29 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
     int init_blocks = (int)((init_items + kThreads * 4 - 1) / (kThreads * 4));
     if (init_blocks > 4 * sm_count()) init_blocks = 4 * sm_count();
     if (init_blocks < 1) init_blocks = 1;
-    route_init_kernel<<<init_blocks, kThreads, 0, st>>>(a);
-    if ((rc = check_launch())) return rc;
+    if ((rc = launch_pdl(route_init_kernel, init_blocks, kThreads, 0, st, a))) return rc;
 
-    route_hist0_kernel<<<p.ntiles, kThreads, sizeof(int) << p.bits[0], st>>>(a);
-    if ((rc = check_launch())) return rc;
+    if ((rc = launch_pdl(route_hist0_kernel, p.ntiles, kThreads, sizeof(int) << p.bits[0], st, a))) return rc;
 
     int extras = 1 + (a.K + kThreads * 4 - 1) / (kThreads * 4);
     if (extras > 33) extras = 33;
     if (extras < 2) extras = 2;
     if (p.passes == 1) {
-        route_extras_kernel<<<extras, kThreads, 0, st>>>(a);
-        if ((rc = check_launch())) return rc;
+        if ((rc = launch_pdl(route_extras_kernel, extras, kThreads, 0, st, a))) return rc;
     }
     int shift = 0;
     for (int pass = 0; pass < p.passes; ++pass) {
         const bool first = pass == 0, last = pass == p.passes - 1;
         if (p.prescan) {
-            route_prescan_kernel<<<((1 << p.bits[pass]) + kWarps - 1) / kWarps, kThreads, 0, st>>>(a, pass);
-            if ((rc = check_launch())) return rc;
+            if ((rc = launch_pdl(route_prescan_kernel, ((1 << p.bits[pass]) + kWarps - 1) / kWarps, kThreads, 0, st, a, pass))) return rc;
         }
         const size_t smb = ((size_t)(kWarps + 2) * sizeof(int)) << p.bits[pass];
         const int grid = p.ntiles + ((first && !last) ? extras : 0);
-        if (first && last) route_scatter_kernel<true, true><<<grid, kThreads, smb, st>>>(a, pass, shift);
-        else if (first) route_scatter_kernel<true, false><<<grid, kThreads, smb, st>>>(a, pass, shift);
-        else if (last) route_scatter_kernel<false, true><<<grid, kThreads, smb, st>>>(a, pass, shift);
-        else route_scatter_kernel<false, false><<<grid, kThreads, smb, st>>>(a, pass, shift);
-        if ((rc = check_launch())) return rc;
+        if (first && last) rc = launch_pdl(route_scatter_kernel<true, true>, grid, kThreads, smb, st, a, pass, shift);
+        else if (first) rc = launch_pdl(route_scatter_kernel<true, false>, grid, kThreads, smb, st, a, pass, shift);
+        else if (last) rc = launch_pdl(route_scatter_kernel<false, true>, grid, kThreads, smb, st, a, pass, shift);
+        else rc = launch_pdl(route_scatter_kernel<false, false>, grid, kThreads, smb, st, a, pass, shift);
+        if (rc) return rc;
         shift += p.bits[pass];
     }
     return LOCMOE_OK;
