@@ -113,16 +113,23 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 // x >= 0 by the five-term rational approximation of Abramowitz & Stegun 7.1.26 (absolute error below 1.5e-7,
 // far under the bf16 rounding of the result); the negative side uses erfc(-x) = 2 - erfc(x) written so that a
 // small Phi is not formed by cancellation.  About half the instructions of erff().
-__device__ __forceinline__ float gelu_erf(float v) {
-    const float x = fabsf(v) * 0.70710678118654752f;
-    const float t = __frcp_rn(fmaf(0.3275911f, x, 1.0f));
-    float poly = fmaf(1.061405429f, t, -1.453152027f);
-    poly = fmaf(poly, t, 1.421413741f);
-    poly = fmaf(poly, t, -0.284496736f);
-    poly = fmaf(poly, t, 0.254829592f);
-    const float half_erfc = 0.5f * poly * t * exp2f(-1.4426950408889634f * x * x);   // 0.5 erfc(|v| / sqrt 2)
-    const float phi = v < 0.0f ? half_erfc : 1.0f - half_erfc;
-    return v * phi;
+// Two elements at a time with the two-wide fp32 instructions: the epilogue warps share their schedulers with
+// the TMA and MMA warps, so fewer epilogue instructions directly mean fewer bubbles in the MMA stream.
+__device__ __forceinline__ float2 gelu_erf2(float2 v) {
+    const float2 x = __fmul2_rn(make_float2(fabsf(v.x), fabsf(v.y)), make_float2(0.70710678118654752f, 0.70710678118654752f));
+    const float2 den = __ffma2_rn(make_float2(0.3275911f, 0.3275911f), x, make_float2(1.0f, 1.0f));
+    const float2 t = make_float2(__frcp_rn(den.x), __frcp_rn(den.y));
+    // coefficients already halved: the polynomial gives 0.5 erfc / exp(-x^2)
+    float2 poly = __ffma2_rn(make_float2(0.5307027145f, 0.5307027145f), t, make_float2(-0.7265760135f, -0.7265760135f));
+    poly = __ffma2_rn(poly, t, make_float2(0.7107068705f, 0.7107068705f));
+    poly = __ffma2_rn(poly, t, make_float2(-0.142248368f, -0.142248368f));
+    poly = __ffma2_rn(poly, t, make_float2(0.127414796f, 0.127414796f));
+    const float2 arg = __fmul2_rn(__fmul2_rn(x, x), make_float2(-1.4426950408889634f, -1.4426950408889634f));
+    const float2 ex = make_float2(exp2f(arg.x), exp2f(arg.y));
+    const float2 h = __fmul2_rn(__fmul2_rn(poly, t), ex);                    // 0.5 erfc(|v| / sqrt 2)
+    const float2 om = __ffma2_rn(h, make_float2(-1.0f, -1.0f), make_float2(1.0f, 1.0f));
+    const float2 phi = make_float2(v.x < 0.0f ? h.x : om.x, v.y < 0.0f ? h.y : om.y);
+    return __fmul2_rn(v, phi);
 }
 
 __global__ void __launch_bounds__(kFfnThreads, 1)
@@ -226,9 +233,10 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 if (!row_ok || col0 >= a.N) continue;
                 float v[32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    v[i] = __uint_as_float(r[i]);
-                    if (a.gelu) v[i] = gelu_erf(v[i]);
+                for (int i = 0; i < 32; i += 2) {
+                    float2 pr = make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                    if (a.gelu) pr = gelu_erf2(pr);
+                    v[i] = pr.x; v[i + 1] = pr.y;
                 }
                 if (col0 + 32 <= a.N && wide_ok) {
                     if (a.out_f32) {
@@ -321,7 +329,10 @@ int launch_gemm(const void* A, const void* W, void* out, int out_f32, int gelu, 
     a.out = out; a.out_f32 = out_f32; a.gelu = gelu; a.E = E; a.M = M; a.N = N; a.K = K;
     a.m_tiles = (M + BM - 1) / BM;
     a.n_tiles = (N + BN - 1) / BN;
-    static bool attr_done = false;
+    static bool attr_done_dev[64] = {false};   // the attribute is per device
+    int attr_dev = 0;
+    cudaGetDevice(&attr_dev);
+    bool& attr_done = attr_done_dev[attr_dev & 63];
     if (!attr_done) {
         if (cudaFuncSetAttribute(ffn_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFfnSmem) != cudaSuccess) {
             cudaGetLastError();

@@ -263,7 +263,10 @@ int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const 
             if (nw > 24) nw = 24;
             if (nw >= 4) {
                 const size_t smem = (size_t)seg * (nw + 1) + (size_t)nw * 8;
-                static bool attr_done = false;
+                static bool attr_done_dev[64] = {false};   // the attribute is per device
+    int attr_dev = 0;
+    cudaGetDevice(&attr_dev);
+    bool& attr_done = attr_done_dev[attr_dev & 63];
                 if (!attr_done) {
                     if (cudaFuncSetAttribute(dispatch_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
                         cudaGetLastError();
