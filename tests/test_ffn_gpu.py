@@ -111,3 +111,24 @@ def test_full_layer_config5_scaled(P):
     # combine of the FFN output
     toks = np.unique(np.concatenate([rng.integers(0, w.T, 256), np.nonzero(rr.drop)[0][:16]]))
     P.check_combine_sampled(y, sh, st, rr, gi, toks)
+
+
+def test_layer_call_with_identity_experts_equals_the_five_calls(P):
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    w = W.CONFIGS[2].scaled(5000)
+    x = W.make_tokens(w, dev)
+    src = W.make_src(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype)
+    rule = B.CapacityRule(1.25, 1.25, -1.0, 0, 0)
+    Ca = B.conventional_capacity(w.T, sh.D, w.E, 1.25)
+    a = B.make_router(sh, Ca, rule, dev)
+    b = B.make_router(sh, Ca, rule, dev)
+    B.router_forward(a, x, src)
+    B.locmoe_moe_layer(sh, x, src, None, rule, Ca, 0, None, None, B.layer_buffers(b), b.out)
+    torch.cuda.synchronize()
+    for name in ("idx", "gate_w", "cos_sim", "pos", "slot", "drop", "inv", "counts", "kept", "send_counts", "load",
+                 "locality", "status"):
+        assert torch.equal(getattr(a, name), getattr(b, name)), name
+    assert torch.equal(a.buf.view(torch.int16), b.buf.view(torch.int16))
+    assert torch.equal(a.out.view(torch.int16), b.out.view(torch.int16))
