@@ -106,6 +106,14 @@ def test_bulk_copy_dispatch_variant(P, monkeypatch):
     P.run_staged(P.W.CONFIGS[1], 1.0, layout=1, full=True)
 
 
+def test_warp_per_row_dispatch_variant(P, monkeypatch):
+    # the warp-per-row dispatch kernel (the default is the flat (row, vector) mapping)
+    monkeypatch.setenv("LOCMOE_DISPATCH", "vec")
+    P.run_staged(P.W.CONFIGS[2].scaled(6000), 1.25, full=True)
+    P.run_staged(_wl(P, T=1500, H=1000, E=8, n_nodes=2, dev_per_node=2, dtype="f32"), 0.5, full=True)
+    P.run_staged(P.W.CONFIGS[1], 1.0, layout=1, full=True)
+
+
 # ---- edge cases and degenerate inputs ----
 
 @pytest.mark.parametrize("kw", [
