@@ -439,7 +439,7 @@ def main():
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
 # profiles/dram_traffic_config2.md, taken at the bench's full size.
 NCU_TRAFFIC = {
-    (2, 1.0): {"gate": 671147776 + 3150336, "dispatch": 606027776 + 621532672, "combine": 606182656 + 618204928},
+    (2, 1.0): {"gate": 671118080 + 3236352, "dispatch": 605918208 + 615610624, "combine": 606182656 + 618102272},
 }
 
 
