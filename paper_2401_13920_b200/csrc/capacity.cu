@@ -51,54 +51,64 @@ __global__ void __launch_bounds__(256) mincos_kernel(const int32_t* __restrict__
     }
 }
 
-// Continued fraction of the regularised incomplete beta function (Lentz's
-// method on the classical even/odd coefficient pair); valid for
-// x < (a + 1) / (a + b + 2).  Returns I_x(a, b) given ln x and ln(1 - x).
-__device__ double beta_cf(double a, double b, double x, double lnx, double ln1mx) {
-    const double tiny = 1e-300, eps = 1e-15;
-    double c = 1.0, d = 1.0 - (a + b) * x / (a + 1.0);
-    if (fabs(d) < tiny) d = tiny;
-    d = 1.0 / d;
-    double h = d;
-    for (int m = 1; m <= 20000; ++m) {
-        double m2 = 2.0 * m;
-        double num = m * (b - m) * x / ((a + m2 - 1.0) * (a + m2));
-        d = 1.0 + num * d; if (fabs(d) < tiny) d = tiny;
-        c = 1.0 + num / c; if (fabs(c) < tiny) c = tiny;
-        d = 1.0 / d;
-        h *= d * c;
-        num = -(a + m) * (a + b + m) * x / ((a + m2) * (a + m2 + 1.0));
-        d = 1.0 + num * d; if (fabs(d) < tiny) d = tiny;
-        c = 1.0 + num / c; if (fabs(c) < tiny) c = tiny;
-        d = 1.0 / d;
-        double del = d * c;
-        h *= del;
-        if (fabs(del - 1.0) < eps) break;
+// Continued fraction of the regularised incomplete beta function, valid for x < (a + 1) / (a + b + 2):
+//   I_x(a, b) = x^a (1 - x)^b / (a B(a, b)) * h,   h = 1 / (1 + d_1 / (1 + d_2 / (1 + ...)))
+// with the classical even/odd coefficients d_n.  Returns h, evaluated by the forward three-term recurrence of
+// the convergents A_n / B_n, four coefficients per trip: their divisions do not depend on one another, and the
+// only division on the dependent chain is the renormalisation (B_n = 1) once per trip, which also yields the
+// convergent for the stopping test.
+__device__ double beta_cf_h(double a, double b, double x) {
+    const double eps = 1e-15;
+    double Ap = 0.0, Bp = 1.0, A = 1.0, B = 1.0;   // convergents n = 0 and n = 1
+    double h = 1.0;
+    for (int m0 = 0; m0 < 40000; m0 += 2) {
+        double c[4];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const double m = (double)(m0 + q), e = m + 1.0;
+            c[2 * q] = -(a + m) * (a + b + m) * x / ((a + 2.0 * m) * (a + 2.0 * m + 1.0));     // d_{2m+1}
+            c[2 * q + 1] = e * (b - e) * x / ((a + 2.0 * e - 1.0) * (a + 2.0 * e));            // d_{2m+2}
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const double An = A + c[k] * Ap, Bn = B + c[k] * Bp;
+            Ap = A; Bp = B; A = An; B = Bn;
+        }
+        const double inv = 1.0 / B;
+        A *= inv; Ap *= inv; Bp *= inv; B = 1.0;
+        const bool done = fabs(A - h) <= eps * fabs(A);
+        h = A;
+        if (done) break;
     }
-    double lnfront = a * lnx + b * ln1mx - (lgamma(a) + lgamma(b) - lgamma(a + b));
-    return exp(lnfront) * h / a;
+    return h;
 }
 
-// Lemma 3: p_delta = 1 - I_{delta^2}(1/2, (d-1)/2) = I_{1-delta^2}((d-1)/2, 1/2),
-// evaluated on whichever side the continued fraction converges, never as a
-// difference of nearly equal numbers when p_delta is small.
-__device__ double p_delta_device(double delta, int d) {
-    if (delta <= 0.0) return 1.0;
-    if (delta >= 1.0) return 0.0;
-    const double b = 0.5 * (double)(d - 1);
-    const double x = delta * delta, y = 1.0 - x;
-    const double lnx = 2.0 * log(delta), lny = log1p(-x);
-    if (y < (b + 1.0) / (b + 2.5)) return beta_cf(b, 0.5, y, lny, lnx);
-    return 1.0 - beta_cf(0.5, b, x, lnx, lny);
+// Scratch of the finish in shared memory.  lg[] does not depend on the data and is filled by finish_begin().
+struct FinishShared {
+    float min[32];
+    int empty[32];
+    double lg[2];      // ln Gamma((d-1)/2), ln Gamma(d/2)
+    double part[4];    // h of the continued fraction, ln delta^2, ln(1 - delta^2), Theorem 1's erfc / exp form
+};
+
+// The last two warps of the CTA carry the data-independent log-gamma evaluations.
+__device__ __forceinline__ void finish_begin(FinishShared& fs, int H) {
+    const int first = (blockDim.x >> 5) - 2;
+    const double bb = 0.5 * (double)(H - 1);
+    if (threadIdx.x == first * 32) fs.lg[0] = lgamma(bb);
+    if (threadIdx.x == (first + 1) * 32) fs.lg[1] = lgamma(bb + 0.5);
 }
 
 // Decodes the per-expert minima (nsets partial arrays of E codes each, combined by min), writes delta_e /
-// theta_e, and lets thread 0 evaluate the closed forms and the integer rule.  One CTA, any block size <= 1024.
-__device__ void capacity_finish(const uint32_t* __restrict__ gmin, int nsets, int T, int E, int H, int D,
-                                const locmoe_capacity_rule_t& rule, float* __restrict__ delta_e,
+// theta_e, and evaluates the closed forms and the integer rule.  Lemma 3:
+//   p_delta = 1 - I_{delta^2}(1/2, (d-1)/2) = I_{1-delta^2}((d-1)/2, 1/2),
+// on whichever side the continued fraction converges, never as a difference of nearly equal numbers when
+// p_delta is small.  The independent pieces (continued fraction, the two logarithms, Theorem 1's other forms)
+// run on four different warps at once; thread 0 puts them together.  One CTA of 128 to 1024 threads, a multiple
+// of 32, that has called finish_begin() before.
+__device__ void capacity_finish(FinishShared& fs, const uint32_t* __restrict__ gmin, int nsets, int T, int E, int H,
+                                int D, const locmoe_capacity_rule_t& rule, float* __restrict__ delta_e,
                                 float* __restrict__ theta_e, locmoe_capacity_t* __restrict__ cap) {
-    __shared__ float s_min[32];
-    __shared__ int s_empty[32];
     float lmin = INFINITY;
     int lempty = 0;
     for (int e = threadIdx.x; e < E; e += blockDim.x) {
@@ -115,12 +125,13 @@ __device__ void capacity_finish(const uint32_t* __restrict__ gmin, int nsets, in
         lmin = fminf(lmin, __shfl_xor_sync(0xffffffffu, lmin, o));
         lempty += __shfl_xor_sync(0xffffffffu, lempty, o);
     }
-    if ((threadIdx.x & 31) == 0) { s_min[threadIdx.x >> 5] = lmin; s_empty[threadIdx.x >> 5] = lempty; }
+    if ((threadIdx.x & 31) == 0) { fs.min[threadIdx.x >> 5] = lmin; fs.empty[threadIdx.x >> 5] = lempty; }
     __syncthreads();
-    if (threadIdx.x != 0) return;
-    const int nwarps = (blockDim.x + 31) >> 5;
-    for (int w = 1; w < nwarps; ++w) { lmin = fminf(lmin, s_min[w]); lempty += s_empty[w]; }
+    const int role = (threadIdx.x & 31) == 0 ? (int)(threadIdx.x >> 5) : -1;   // lane 0 of warps 0..3 work on
 
+    const int nwarps = (blockDim.x + 31) >> 5;
+    lmin = fs.min[0]; lempty = fs.empty[0];
+    for (int w = 1; w < nwarps; ++w) { lmin = fminf(lmin, fs.min[w]); lempty += fs.empty[w]; }
     int flags = 0;
     double delta = (double)lmin;
     delta = delta < 0.0 ? 0.0 : (delta > 1.0 ? 1.0 : delta);
@@ -128,12 +139,32 @@ __device__ void capacity_finish(const uint32_t* __restrict__ gmin, int nsets, in
         delta = rule.delta_override > 1.0 ? 1.0 : rule.delta_override;
         flags |= LOCMOE_FLAG_DELTA_OVERRIDE;
     }
+    const double bb = 0.5 * (double)(H - 1);
+    const double x = delta * delta, y = 1.0 - x;
+    const bool interior = delta > 0.0 && delta < 1.0;
+    const bool upper = y < (bb + 1.0) / (bb + 2.5);   // the fraction converges for I_y(bb, 1/2)
+    const double arg = x * (double)H / (2.0 - x);
+    if (role == 0) fs.part[0] = interior ? (upper ? beta_cf_h(bb, 0.5, y) : beta_cf_h(0.5, bb, x)) : 0.0;
+    if (role == 1) fs.part[1] = interior ? 2.0 * log(delta) : 0.0;
+    if (role == 2) fs.part[2] = interior ? log1p(-x) : 0.0;
+    if (role == 3) fs.part[3] = rule.bound_form == LOCMOE_BOUND_ERFC ? erfc(sqrt(arg))
+                              : (rule.bound_form == LOCMOE_BOUND_EXP ? exp(arg) : 0.0);
+    __syncthreads();
+    if (role != 0) return;
+
     const double n = (double)E, dT = (double)T, dD = (double)D;
-    const double p = p_delta_device(delta, H);
-    const double arg = delta * delta * (double)H / (2.0 - delta * delta);
+    double p;
+    if (delta <= 0.0) p = 1.0;
+    else if (delta >= 1.0) p = 0.0;
+    else {
+        const double lnbeta = 0.57236494292470008707 + fs.lg[0] - fs.lg[1];   // ln Gamma(1/2) = ln(pi) / 2
+        const double lnx = fs.part[1], lny = fs.part[2], h = fs.part[0];
+        p = upper ? exp(bb * lny + 0.5 * lnx - lnbeta) * h / bb
+                  : 1.0 - exp(0.5 * lnx + bb * lny - lnbeta) * h / 0.5;
+    }
     double ec;
-    if (rule.bound_form == LOCMOE_BOUND_ERFC) ec = 1.0 / (n * erfc(sqrt(arg)));
-    else if (rule.bound_form == LOCMOE_BOUND_EXP) ec = exp(arg) / n;
+    if (rule.bound_form == LOCMOE_BOUND_ERFC) ec = 1.0 / (n * fs.part[3]);
+    else if (rule.bound_form == LOCMOE_BOUND_EXP) ec = fs.part[3] / n;
     else ec = 1.0 / (n * p);
 
     // integer rule: each product / quotient rounded once (no fused multiply-add)
@@ -163,7 +194,9 @@ __global__ void __launch_bounds__(256) capacity_finish_kernel(const uint32_t* __
                                                               int D, locmoe_capacity_rule_t rule,
                                                               float* __restrict__ delta_e, float* __restrict__ theta_e,
                                                               locmoe_capacity_t* __restrict__ cap) {
-    capacity_finish(gmin, 1, T, E, H, D, rule, delta_e, theta_e, cap);
+    __shared__ FinishShared fs;
+    finish_begin(fs, H);
+    capacity_finish(fs, gmin, 1, T, E, H, D, rule, delta_e, theta_e, cap);
 }
 
 // Whole stage in one kernel on one cluster: every CTA reduces its share of the tokens into per-expert minima in
@@ -179,18 +212,27 @@ capacity_cluster_kernel(const int32_t* __restrict__ idx, const float* __restrict
     pdl_wait();
     pdl_trigger();
     extern __shared__ uint32_t smin[];
+    __shared__ FinishShared fs;
     cg::cluster_group cluster = cg::this_cluster();
     const int cta = (int)cluster.block_rank();
     for (int e = threadIdx.x; e < E; e += blockDim.x) smin[e] = 0xffffffffu;
     __syncthreads();
-    for (int t = cta * kCapThreads + threadIdx.x; t < T; t += kCapCS * kCapThreads) {
-        const int e = idx[t];
-        if (e >= 0 && e < E) atomicMin(&smin[e], order_code(cs[t]));
+    // CTA 0's last two warps evaluate the log-gammas instead of reading tokens; the other threads share the tokens
+    constexpr int kMath = 64, kWorkers = kCapCS * kCapThreads - kMath;
+    const bool math = cta == 0 && threadIdx.x >= kCapThreads - kMath;
+    if (math) {
+        finish_begin(fs, H);
+    } else {
+        const int wid = cta == 0 ? (int)threadIdx.x : cta * kCapThreads - kMath + (int)threadIdx.x;
+        for (int t = wid; t < T; t += kWorkers) {
+            const int e = idx[t];
+            if (e >= 0 && e < E) atomicMin(&smin[e], order_code(cs[t]));
+        }
     }
     __syncthreads();
     for (int e = threadIdx.x; e < E; e += blockDim.x) part[(size_t)cta * E + e] = smin[e];
     cluster.sync();
-    if (cta == 0) capacity_finish(part, kCapCS, T, E, H, D, rule, delta_e, theta_e, cap);
+    if (cta == 0) capacity_finish(fs, part, kCapCS, T, E, H, D, rule, delta_e, theta_e, cap);
 }
 
 }  // namespace

@@ -46,8 +46,10 @@ struct RouteArgs {
     int bits[kMaxPasses];
     uint32_t* keys[2];
     int32_t* toks[2];
-    int32_t* hist[kMaxPasses];  // [1 << bits[p]][ntiles], digit major
+    int32_t* hist[kMaxPasses];  // [1 << bits[p]][hstride], digit major
     int32_t* keystart;          // [K]
+    int32_t* rowbase;           // [K] first buffer row of the key's class
+    int hstride, tile_shift;    // row stride of the histogram matrices (a multiple of 4 >= ntiles); log2(tile)
     int32_t* rowtot;            // [256] per-digit totals of the pass being scattered (prescan mode)
     int prescan;                // 1: a prescan launch turned hist[p] into exclusive prefixes along the tiles
 };
@@ -74,20 +76,6 @@ __device__ __forceinline__ long long route_row_base(const RouteArgs& a, int k) {
     return (long long)e * a.D + dest_rank(b, s, a.N, a.Dn);
 }
 
-// Final outputs of one token: `dest` is its position in the stable sort by key.
-__device__ __forceinline__ void route_emit(const RouteArgs& a, int k, int t, int dest, int C) {
-    const int p = dest - a.keystart[k];
-    const bool dropped = p >= C;
-    a.pos[t] = p;
-    a.drop[t] = dropped ? 1 : 0;
-    int row = -1;
-    if (!dropped) {
-        row = (int)(route_row_base(a, k) * a.C_alloc + p);
-        a.inv[row] = t;
-    }
-    a.slot[t] = row;
-}
-
 __global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a) {
     pdl_wait();
     pdl_trigger();
@@ -98,7 +86,7 @@ __global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a)
     for (long long i = i0; i < (long long)a.D * a.D; i += stride) a.send_counts[i] = 0;
     for (long long i = i0; i < a.E; i += stride) a.load[i] = 0;
     for (int p = 1; p < a.passes; ++p) {
-        const long long n = ((long long)a.ntiles) << a.bits[p];
+        const long long n = ((long long)a.hstride) << a.bits[p];
         for (long long i = i0; i < n; i += stride) a.hist[p][i] = 0;
     }
     if (i0 < 6) a.locality[i0] = 0ull;
@@ -125,7 +113,7 @@ __global__ void __launch_bounds__(kThreads) route_hist0_kernel(const RouteArgs a
     }
     if (warn) atomicOr(a.status, warn);
     __syncthreads();
-    for (int d = threadIdx.x; d < nbins; d += blockDim.x) a.hist[0][(size_t)d * a.ntiles + blockIdx.x] = sh[d];
+    for (int d = threadIdx.x; d < nbins; d += blockDim.x) a.hist[0][(size_t)d * a.hstride + blockIdx.x] = sh[d];
 }
 
 // Exclusive scan of in[0..n) into out[0..n) by one CTA of kThreads threads (in == out allowed).  Every warp owns a
@@ -181,6 +169,7 @@ __device__ void route_extras(const RouteArgs& a, int x, int nx) {
         const int c = a.counts[k];
         const int kp = c < C ? c : C;
         a.kept[k] = kp;
+        a.rowbase[k] = (int)(route_row_base(a, k) * a.C_alloc);
         if (c == 0) continue;
         const int s = k / a.E, e = k - s * a.E, b = e / a.Ed;
         if (b == s) { raw0 += c; kp0 += kp; }
@@ -221,7 +210,7 @@ __global__ void __launch_bounds__(kThreads) route_prescan_kernel(const RouteArgs
     const int lane = threadIdx.x & 31;
     const int d = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (d >= nbins) return;
-    int32_t* row = a.hist[pass] + (size_t)d * a.ntiles;
+    int32_t* row = a.hist[pass] + (size_t)d * a.hstride;
     const int chunk = (a.ntiles + 31) / 32;
     const int lo = min(lane * chunk, a.ntiles), hi = min(lo + chunk, a.ntiles);
     int s = 0;
@@ -237,8 +226,9 @@ __global__ void __launch_bounds__(kThreads) route_prescan_kernel(const RouteArgs
     if (lane == 31) a.rowtot[d] = incl;
 }
 
-// One radix pass over one tile per CTA; CTAs beyond ntiles run the extras.
-template <bool FIRST, bool LAST>
+// One radix pass over one tile per CTA; CTAs beyond ntiles run the extras.  R = 32-token rounds per warp
+// (compile time, so that a small batch does not carry the code of a large one).
+template <bool FIRST, bool LAST, int R>
 __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs a, int pass, int shift) {
     pdl_wait();
     pdl_trigger();
@@ -262,57 +252,78 @@ __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs
     const int32_t* tin = a.toks[(pass + 1) & 1];
     uint32_t* kout = a.keys[pass & 1];
     int32_t* tout = a.toks[pass & 1];
-    const int wbase = tileid * a.tile + w * a.rounds * 32;
+    const int wbase = tileid * a.tile + w * R * 32;
     const uint32_t lt = (1u << lane) - 1u;
     int* mycnt = cnt + w * nbins;
-    int key[kMaxRounds], tok[kMaxRounds], rank[kMaxRounds];
+    int key[R], tok[R], rank[R];
+    int kstart[LAST ? R : 1], rbase[LAST ? R : 1];   // last pass: class start and first buffer row of the item's key
+    int C = 0;
+    if (LAST) { C = a.cap->C_local; if (C > a.C_alloc) C = a.C_alloc; }
 #pragma unroll
-    for (int r = 0; r < kMaxRounds; ++r) {
+    for (int r = 0; r < R; ++r) {
         key[r] = -1; tok[r] = -1; rank[r] = 0;
-        if (r < a.rounds) {
-            const int j = wbase + r * 32 + lane;
-            if (j < a.T) {
-                if (FIRST) { int warn = 0; tok[r] = j; key[r] = token_key(a, j, &warn); }
-                else { key[r] = (int)kin[j]; tok[r] = tin[j]; }
+        const int j = wbase + r * 32 + lane;
+        if (j < a.T) {
+            if (FIRST) {
+                const int e = a.idx[j], sd = a.src[j];
+                tok[r] = j;
+                key[r] = ((unsigned)sd < (unsigned)a.D && (unsigned)e < (unsigned)a.E) ? sd * a.E + e : -1;
+            } else {
+                key[r] = (int)kin[j]; tok[r] = tin[j];
             }
         }
     }
+    if (LAST) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            kstart[r] = 0; rbase[r] = 0;
+            if ((unsigned)key[r] < (unsigned)a.K) { kstart[r] = a.keystart[key[r]]; rbase[r] = a.rowbase[key[r]]; }
+        }
+    }
 
-    // ---- this tile's offsets from the (digit, tile) histogram matrix: one warp per digit row ----
-    // (kRB rows per batch so that their loads are all in flight together: the matrix lives in L2)
+    // ---- this tile's offsets from the (digit, tile) histogram matrix: one warp per digit row, kRB rows per
+    // batch, a row read as 16-byte pieces so that all of a batch's loads are in flight together (L2 resident) ----
     const int32_t* H = a.hist[pass];
     constexpr int kRB = 8;
     if (a.prescan) {
-        for (int d = tid; d < nbins; d += kThreads) { pre[d] = H[(size_t)d * a.ntiles + tileid]; tot[d] = a.rowtot[d]; }
-    } else
-    for (int d0 = w; d0 < nbins; d0 += kWarps * kRB) {
-        int before[kRB], all[kRB];
+        for (int d = tid; d < nbins; d += kThreads) { pre[d] = H[(size_t)d * a.hstride + tileid]; tot[d] = a.rowtot[d]; }
+    } else {
+        const int npieces = a.hstride >> 2;
+        for (int d0 = w; d0 < nbins; d0 += kWarps * kRB) {
+            int before[kRB], all[kRB];
 #pragma unroll
-        for (int q = 0; q < kRB; ++q) { before[q] = 0; all[q] = 0; }
-        for (int j = lane; j < a.ntiles; j += 32) {
+            for (int q = 0; q < kRB; ++q) { before[q] = 0; all[q] = 0; }
+            for (int c = lane; c < npieces; c += 32) {
+                int4 v[kRB];
 #pragma unroll
-            for (int q = 0; q < kRB; ++q) {
-                const int d = d0 + q * kWarps;
-                if (d < nbins) {
-                    const int v = H[(size_t)d * a.ntiles + j];
-                    all[q] += v;
-                    if (j < tileid) before[q] += v;
+                for (int q = 0; q < kRB; ++q) {
+                    const int d = d0 + q * kWarps;
+                    v[q] = make_int4(0, 0, 0, 0);
+                    if (d < nbins) v[q] = *reinterpret_cast<const int4*>(H + (size_t)d * a.hstride + 4 * c);
+                }
+                const int j = 4 * c;
+                const bool in0 = j < a.ntiles, in1 = j + 1 < a.ntiles, in2 = j + 2 < a.ntiles, in3 = j + 3 < a.ntiles;
+                const bool b0 = j < tileid, b1 = j + 1 < tileid, b2 = j + 2 < tileid, b3 = j + 3 < tileid;
+#pragma unroll
+                for (int q = 0; q < kRB; ++q) {
+                    all[q] += (in0 ? v[q].x : 0) + (in1 ? v[q].y : 0) + (in2 ? v[q].z : 0) + (in3 ? v[q].w : 0);
+                    before[q] += (b0 ? v[q].x : 0) + (b1 ? v[q].y : 0) + (b2 ? v[q].z : 0) + (b3 ? v[q].w : 0);
                 }
             }
-        }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
+            for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-            for (int q = 0; q < kRB; ++q) {
-                before[q] += __shfl_xor_sync(0xffffffffu, before[q], o);
-                all[q] += __shfl_xor_sync(0xffffffffu, all[q], o);
+                for (int q = 0; q < kRB; ++q) {
+                    before[q] += __shfl_xor_sync(0xffffffffu, before[q], o);
+                    all[q] += __shfl_xor_sync(0xffffffffu, all[q], o);
+                }
             }
-        }
-        if (lane == 0) {
+            if (lane == 0) {
 #pragma unroll
-            for (int q = 0; q < kRB; ++q) {
-                const int d = d0 + q * kWarps;
-                if (d < nbins) { pre[d] = before[q]; tot[d] = all[q]; }
+                for (int q = 0; q < kRB; ++q) {
+                    const int d = d0 + q * kWarps;
+                    if (d < nbins) { pre[d] = before[q]; tot[d] = all[q]; }
+                }
             }
         }
     }
@@ -343,23 +354,21 @@ __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs
 
     // ---- stable rank inside the tile ----
 #pragma unroll
-    for (int r = 0; r < kMaxRounds; ++r)
+    for (int r = 0; r < R; ++r)
         if (!FIRST && wbase + r * 32 + lane >= n_valid) key[r] = -1;   // beyond the valid items: stale buffer contents
 #pragma unroll
-    for (int r = 0; r < kMaxRounds; ++r) {
-        if (r < a.rounds) {
-            const bool valid = key[r] >= 0;
-            const uint32_t d = valid ? (((uint32_t)key[r] >> shift) & mask) : 0xffffffffu;
-            const uint32_t peers = __match_any_sync(0xffffffffu, d);
-            int before = 0;
-            if (valid) before = mycnt[d];
-            __syncwarp();
-            if (valid) {
-                rank[r] = before + __popc(peers & lt);
-                if ((peers & lt) == 0) mycnt[d] = before + __popc(peers);
-            }
-            __syncwarp();
+    for (int r = 0; r < R; ++r) {
+        const bool valid = key[r] >= 0;
+        const uint32_t d = valid ? (((uint32_t)key[r] >> shift) & mask) : 0xffffffffu;
+        const uint32_t peers = __match_any_sync(0xffffffffu, d);
+        int before = 0;
+        if (valid) before = mycnt[d];
+        __syncwarp();
+        if (valid) {
+            rank[r] = before + __popc(peers & lt);
+            if ((peers & lt) == 0) mycnt[d] = before + __popc(peers);
         }
+        __syncwarp();
     }
     __syncthreads();
     // counters -> starting offsets: digit base + earlier tiles + earlier warps of this tile
@@ -374,24 +383,48 @@ __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs
     }
     __syncthreads();
 
-    int C = 0;
-    if (LAST) { C = a.cap->C_local; if (C > a.C_alloc) C = a.C_alloc; }
     const int nshift = shift + a.bits[pass];
     const uint32_t nmask = LAST ? 0u : (uint32_t)(1 << a.bits[LAST ? pass : pass + 1]) - 1u;
     int32_t* Hn = LAST ? nullptr : a.hist[LAST ? pass : pass + 1];
 #pragma unroll
-    for (int r = 0; r < kMaxRounds; ++r) {
-        if (r < a.rounds && key[r] >= 0) {
+    for (int r = 0; r < R; ++r) {
+        if (key[r] >= 0) {
             const uint32_t d = ((uint32_t)key[r] >> shift) & mask;
             const int dest = mycnt[d] + rank[r];
             if (LAST) {
-                route_emit(a, key[r], tok[r], dest, C);
+                // final outputs of the token: dest is its position in the stable sort by key
+                const int t = tok[r];
+                const int p = dest - kstart[r];
+                const bool dropped = p >= C;
+                const int row = dropped ? -1 : rbase[r] + p;
+                a.pos[t] = p;
+                a.drop[t] = dropped ? 1 : 0;
+                if (!dropped) a.inv[row] = t;
+                a.slot[t] = row;
             } else {
                 kout[dest] = (uint32_t)key[r];
                 tout[dest] = tok[r];
-                atomicAdd(&Hn[(size_t)(((uint32_t)key[r] >> nshift) & nmask) * a.ntiles + dest / a.tile], 1);
+                atomicAdd(&Hn[(size_t)(((uint32_t)key[r] >> nshift) & nmask) * a.hstride + (dest >> a.tile_shift)], 1);
             }
         }
+    }
+}
+
+template <int R>
+int launch_scatter_r(bool first, bool last, int grid, size_t smb, cudaStream_t st, const RouteArgs& a, int pass, int shift) {
+    if (first && last) return launch_pdl(route_scatter_kernel<true, true, R>, grid, kThreads, smb, st, a, pass, shift);
+    if (first) return launch_pdl(route_scatter_kernel<true, false, R>, grid, kThreads, smb, st, a, pass, shift);
+    if (last) return launch_pdl(route_scatter_kernel<false, true, R>, grid, kThreads, smb, st, a, pass, shift);
+    return launch_pdl(route_scatter_kernel<false, false, R>, grid, kThreads, smb, st, a, pass, shift);
+}
+
+int launch_scatter(int rounds, bool first, bool last, int grid, size_t smb, cudaStream_t st, const RouteArgs& a, int pass,
+                   int shift) {
+    switch (rounds) {
+        case 2: return launch_scatter_r<2>(first, last, grid, smb, st, a, pass, shift);
+        case 4: return launch_scatter_r<4>(first, last, grid, smb, st, a, pass, shift);
+        case 8: return launch_scatter_r<8>(first, last, grid, smb, st, a, pass, shift);
+        default: return launch_scatter_r<16>(first, last, grid, smb, st, a, pass, shift);
     }
 }
 
@@ -416,9 +449,11 @@ int plan_route(const locmoe_shape_t& s, RoutePlan* p) {
     int rounds = (int)(((long long)s.T + 65535) / 65536);
     if (rounds < 2) rounds = 2;
     if (rounds > kMaxRounds) rounds = kMaxRounds;
+    while (rounds & (rounds - 1)) ++rounds;   // 2, 4, 8 or 16: the scatter kernel is compiled per value
     p->rounds = rounds;
     p->tile = kWarps * rounds * 32;
     p->ntiles = (int)(((long long)s.T + p->tile - 1) / p->tile);
+    p->hstride = (p->ntiles + 3) & ~3;
     size_t off = 0;
     for (int i = 0; i < 2; ++i) {
         p->off_keys[i] = off; off += p->passes > 1 ? align256((size_t)s.T * 4) : 0;
@@ -426,9 +461,10 @@ int plan_route(const locmoe_shape_t& s, RoutePlan* p) {
     }
     for (int i = 0; i < 4; ++i) {
         p->off_hist[i] = off;
-        if (i < p->passes) off += align256(((size_t)p->ntiles << p->bits[i]) * 4);
+        if (i < p->passes) off += align256(((size_t)p->hstride << p->bits[i]) * 4);
     }
     p->off_keystart = off; off += align256((size_t)K * 4);
+    p->off_rowbase = off; off += align256((size_t)K * 4);
     p->off_rowtot = off; off += 1024;
     p->total = off;
     p->prescan = ((long long)p->ntiles << p->bits[0]) > 32768 ? 1 : 0;
@@ -467,6 +503,10 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
         a.hist[i] = reinterpret_cast<int32_t*>(w + p.off_hist[i]);
     }
     a.keystart = reinterpret_cast<int32_t*>(w + p.off_keystart);
+    a.rowbase = reinterpret_cast<int32_t*>(w + p.off_rowbase);
+    a.hstride = p.hstride;
+    a.tile_shift = 0;
+    while ((1 << a.tile_shift) < p.tile) ++a.tile_shift;
     a.rowtot = reinterpret_cast<int32_t*>(w + p.off_rowtot);
     a.prescan = p.prescan;
 
@@ -492,10 +532,7 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
         }
         const size_t smb = ((size_t)(kWarps + 2) * sizeof(int)) << p.bits[pass];
         const int grid = p.ntiles + ((first && !last) ? extras : 0);
-        if (first && last) rc = launch_pdl(route_scatter_kernel<true, true>, grid, kThreads, smb, st, a, pass, shift);
-        else if (first) rc = launch_pdl(route_scatter_kernel<true, false>, grid, kThreads, smb, st, a, pass, shift);
-        else if (last) rc = launch_pdl(route_scatter_kernel<false, true>, grid, kThreads, smb, st, a, pass, shift);
-        else rc = launch_pdl(route_scatter_kernel<false, false>, grid, kThreads, smb, st, a, pass, shift);
+        rc = launch_scatter(p.rounds, first, last, grid, smb, st, a, pass, shift);
         if (rc) return rc;
         shift += p.bits[pass];
     }
