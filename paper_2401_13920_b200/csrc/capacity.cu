@@ -224,9 +224,19 @@ capacity_cluster_kernel(const int32_t* __restrict__ idx, const float* __restrict
         finish_begin(fs, H);
     } else {
         const int wid = cta == 0 ? (int)threadIdx.x : cta * kCapThreads - kMath + (int)threadIdx.x;
-        for (int t = wid; t < T; t += kWorkers) {
-            const int e = idx[t];
-            if (e >= 0 && e < E) atomicMin(&smin[e], order_code(cs[t]));
+        constexpr int kU = 8;   // tokens in flight per thread
+        for (int t0 = wid; t0 < T; t0 += kU * kWorkers) {
+            int e[kU];
+            float c[kU];
+#pragma unroll
+            for (int u = 0; u < kU; ++u) {
+                const int t = t0 + u * kWorkers;
+                e[u] = -1; c[u] = 0.0f;
+                if (t < T) { e[u] = idx[t]; c[u] = cs[t]; }
+            }
+#pragma unroll
+            for (int u = 0; u < kU; ++u)
+                if (e[u] >= 0 && e[u] < E) atomicMin(&smin[e[u]], order_code(c[u]));
         }
     }
     __syncthreads();

@@ -60,14 +60,6 @@ __device__ __forceinline__ int dest_rank(int a, int b, int N, int Dn) {
     return dn * Dn + dl;
 }
 
-// Key of token t, or -1 with a warning bit when the token cannot be routed.
-__device__ __forceinline__ int token_key(const RouteArgs& a, int t, int* warn) {
-    int e = a.idx[t], s = a.src[t];
-    if (s < 0 || s >= a.D) { *warn |= LOCMOE_WARN_BAD_SRC; return -1; }
-    if (e < 0 || e >= a.E) { *warn |= LOCMOE_WARN_BAD_IDX; return -1; }
-    return s * a.E + e;
-}
-
 // Row base (in units of C_alloc rows) of key k = s * E + e in the chosen layout.
 __device__ __forceinline__ long long route_row_base(const RouteArgs& a, int k) {
     const int s = k / a.E, e = k - s * a.E;
@@ -103,13 +95,29 @@ __global__ void __launch_bounds__(kThreads) route_hist0_kernel(const RouteArgs a
     const int base = blockIdx.x * a.tile;
     const uint32_t mask = (uint32_t)nbins - 1u;
     int warn = 0;
-    for (int o = threadIdx.x; o < a.tile; o += blockDim.x) {
-        const int t = base + o;
-        if (t >= a.T) break;
-        const int key = token_key(a, t, &warn);
-        if (key < 0) { a.pos[t] = -1; a.slot[t] = -1; a.drop[t] = 1; continue; }
-        atomicAdd(&a.counts[key], 1);
-        atomicAdd(&sh[(uint32_t)key & mask], 1);
+    constexpr int kU = 4;   // tokens in flight per thread
+    for (int o0 = threadIdx.x; o0 < a.tile; o0 += kU * kThreads) {
+        int e[kU], sd[kU];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int o = o0 + u * kThreads, t = base + o;
+            e[u] = 0; sd[u] = 0;
+            if (o < a.tile && t < a.T) { e[u] = a.idx[t]; sd[u] = a.src[t]; }
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int o = o0 + u * kThreads, t = base + o;
+            if (o >= a.tile || t >= a.T) continue;
+            const bool bad_s = (unsigned)sd[u] >= (unsigned)a.D, bad_e = (unsigned)e[u] >= (unsigned)a.E;
+            if (bad_s || bad_e) {
+                warn |= bad_s ? LOCMOE_WARN_BAD_SRC : LOCMOE_WARN_BAD_IDX;
+                a.pos[t] = -1; a.slot[t] = -1; a.drop[t] = 1;
+                continue;
+            }
+            const int key = sd[u] * a.E + e[u];
+            atomicAdd(&a.counts[key], 1);
+            atomicAdd(&sh[(uint32_t)key & mask], 1);
+        }
     }
     if (warn) atomicOr(a.status, warn);
     __syncthreads();
