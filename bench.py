@@ -270,7 +270,7 @@ def main():
         B.locmoe_route(sh, st.idx, src, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
                        st.send_counts, st.load, st.locality, st.status, st.ws, stream)
         mark()
-        B.locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream)
+        B.locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream, slot=st.slot)
         mark()
         if use_ffn:
             B.locmoe_expert_ffn(sh, Ca, F, st.buf, w_in, w_out, h1, y, stream)

@@ -198,9 +198,18 @@ int locmoe_route(const locmoe_shape_t *shape, const int32_t *idx, const int32_t 
  * Dispatch: buf[row][:] = x[inv[row]][:] bit for bit for occupied rows; rows
  * with inv < 0 are zero-filled when zero_pad != 0 and left untouched otherwise.
  * x [T][H], buf [D * E * C_alloc][H], both of shape->x_dtype.
+ * slot is optional (NULL allowed): int32[T] as written by locmoe_route for the
+ * same routing, i.e. inv[slot[t]] == t for every kept token.  The result is the
+ * same with or without it; with it the rows are copied token by token in
+ * descending token order, so that the tokens the gate read last, which are
+ * still in L2, are read first, and the rows written last are those a combine in
+ * ascending token order reads first.  A slot array that does not belong to inv
+ * gives an unspecified buffer (no out-of-range access: entries outside
+ * [0, rows) are skipped).
  */
 int locmoe_dispatch(const locmoe_shape_t *shape, int32_t C_alloc, const void *x,
-                    const int32_t *inv, void *buf, int32_t zero_pad, void *stream);
+                    const int32_t *inv, const int32_t *slot, void *buf, int32_t zero_pad,
+                    void *stream);
 
 /*
  * Combine: out[t][:] = gate_w[t] * y[slot[t]][:] for a kept token and 0 for a

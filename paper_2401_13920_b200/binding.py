@@ -74,7 +74,7 @@ def _load() -> C.CDLL:
     lib.locmoe_capacity_noalloc.argtypes = [C.POINTER(Shape), vp, vp, C.POINTER(CapacityRule), vp, vp, vp, vp]
     lib.locmoe_capacity_read.argtypes = [vp, C.POINTER(Capacity), vp]
     lib.locmoe_route.argtypes = [C.POINTER(Shape), vp, vp, vp, i32] + [vp] * 10 + [vp, C.c_size_t, vp]
-    lib.locmoe_dispatch.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, i32, vp]
+    lib.locmoe_dispatch.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, vp, i32, vp]
     lib.locmoe_combine.argtypes = [C.POINTER(Shape), i32, vp, i32, vp, vp, vp, i32, vp]
     lib.locmoe_expert_ffn.argtypes = [C.POINTER(Shape), i32, i32, vp, vp, vp, vp, vp, i32, vp]
     lib.locmoe_moe_layer.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(CapacityRule), i32, i32, vp, vp,
@@ -225,14 +225,16 @@ def locmoe_route(shape: Shape, idx, src_dev, cap_dev, C_alloc, pos, slot, drop, 
         _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
 
 
-def locmoe_dispatch(shape: Shape, C_alloc, x, inv, buf, zero_pad=True, stream=None) -> int:
+def locmoe_dispatch(shape: Shape, C_alloc, x, inv, buf, zero_pad=True, stream=None, slot=None) -> int:
     rows = shape.D * shape.E * C_alloc
     dt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
     _want(x, dt, shape.T * shape.H, "x")
     _want(inv, torch.int32, rows, "inv")
     _want(buf, dt, rows * shape.H, "buf")
-    return _check("locmoe_dispatch", _lib.locmoe_dispatch(C.byref(shape), int(C_alloc), _ptr(x), _ptr(inv), _ptr(buf),
-                                                          1 if zero_pad else 0, _stream(stream)))
+    if slot is not None:
+        _want(slot, torch.int32, shape.T, "slot")
+    return _check("locmoe_dispatch", _lib.locmoe_dispatch(C.byref(shape), int(C_alloc), _ptr(x), _ptr(inv), _ptr(slot),
+                                                          _ptr(buf), 1 if zero_pad else 0, _stream(stream)))
 
 
 def locmoe_combine(shape: Shape, C_alloc, y, slot, gate_w, out, accumulate=False, stream=None) -> int:
@@ -356,7 +358,7 @@ def router_forward(st: RouterState, x, src_dev, y=None, eps=None, stream=None, o
     locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
     locmoe_route(sh, st.idx, src_dev, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
                  st.send_counts, st.load, st.locality, st.status, st.ws, stream)
-    locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream)
+    locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream, slot=st.slot)
     locmoe_combine(sh, Ca, st.buf if y is None else y, st.slot, st.gate_w, out, False, stream)
     return out
 

@@ -123,8 +123,8 @@ int locmoe_route(const locmoe_shape_t* shape, const int32_t* idx, const int32_t*
                         locality, status, ws, static_cast<cudaStream_t>(stream));
 }
 
-int locmoe_dispatch(const locmoe_shape_t* shape, int32_t C_alloc, const void* x, const int32_t* inv, void* buf,
-                    int32_t zero_pad, void* stream) {
+int locmoe_dispatch(const locmoe_shape_t* shape, int32_t C_alloc, const void* x, const int32_t* inv,
+                    const int32_t* slot, void* buf, int32_t zero_pad, void* stream) {
     int rc = check_shape(shape);
     if (rc) return rc;
     if (!x || !inv || !buf) return LOCMOE_ERR_NULL;
@@ -132,7 +132,7 @@ int locmoe_dispatch(const locmoe_shape_t* shape, int32_t C_alloc, const void* x,
     if (rows < 0) return LOCMOE_ERR_SHAPE;
     const int esz = shape->x_dtype == LOCMOE_F32 ? 4 : 2;
     if ((uintptr_t)x % esz || (uintptr_t)buf % esz) return LOCMOE_ERR_ALIGN;
-    return launch_dispatch(*shape, rows, x, inv, buf, zero_pad, static_cast<cudaStream_t>(stream));
+    return launch_dispatch(*shape, rows, x, inv, slot, buf, zero_pad, static_cast<cudaStream_t>(stream));
 }
 
 int locmoe_combine(const locmoe_shape_t* shape, int32_t C_alloc, const void* y, int32_t y_dtype, const int32_t* slot,
@@ -187,7 +187,7 @@ int locmoe_moe_layer(const locmoe_shape_t* shape, const void* x, const int32_t* 
                       b->send_counts, b->load, b->locality, b->status, b->ws, b->ws_bytes, stream);
     if (rc < 0) return rc;
     warn |= rc;
-    rc = locmoe_dispatch(shape, C_alloc, x, b->inv, b->buf, 1, stream);
+    rc = locmoe_dispatch(shape, C_alloc, x, b->inv, b->slot, b->buf, 1, stream);
     if (rc < 0) return rc;
     warn |= rc;
     const void* ysrc = b->buf;

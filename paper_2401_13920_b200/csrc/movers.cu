@@ -80,6 +80,55 @@ __global__ void __launch_bounds__(kThreads) dispatch_flat_kernel(const uint4* __
     }
 }
 
+// Token-major dispatch (used when the caller supplies slot[]): the (token, vector) items are walked in descending
+// token order, every CTA a contiguous run of 8 items per thread, so that the copy starts with the tokens the gate
+// read last (still in L2) and ends with the lowest tokens, whose rows a combine in ascending token order reads
+// first.  Rows without a token are zero-filled by the same CTAs: CTA b looks at rows [b * zrows, (b + 1) * zrows).
+constexpr int kTokIters = 2;
+__global__ void __launch_bounds__(kThreads) dispatch_token_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ slot,
+                                                                  const int32_t* __restrict__ inv, uint4* __restrict__ buf,
+                                                                  unsigned total, unsigned V, int T, long long rows,
+                                                                  int zero_pad, int zrows) {
+    pdl_wait();
+    pdl_trigger();
+    const unsigned base = blockIdx.x * (unsigned)(kThreads * 4 * kTokIters);
+#pragma unroll
+    for (int it = 0; it < kTokIters; ++it) {
+        uint4 r[4];
+        size_t dst[4];
+        bool st[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const unsigned jj = base + (unsigned)((it * 4 + k) * kThreads) + threadIdx.x;
+            st[k] = false;
+            if (jj < total && jj >= base) {
+                const unsigned tt = jj / V, v = jj - tt * V;
+                const int t = T - 1 - (int)tt;
+                const int row = __ldg(slot + t);
+                if (row >= 0 && row < rows) {
+                    r[k] = ld_stream(x + (size_t)t * V + v);
+                    dst[k] = (size_t)row * V + v;
+                    st[k] = true;
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (st[k]) st_stream(buf + dst[k], r[k]);
+    }
+    if (zero_pad) {
+        const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+        for (int i = w; i < zrows; i += kThreads / 32) {
+            const long long row = (long long)blockIdx.x * zrows + i;
+            if (row >= rows) break;
+            const int t = __ldg(inv + row);
+            if (t >= 0 && t < T) continue;
+            uint4* d = buf + row * V;
+            for (unsigned v = lane; v < V; v += kWarp) st_stream(d + v, make_uint4(0, 0, 0, 0));
+        }
+    }
+}
+
 // Device-side diagnostics word (bit 0: a bounded barrier wait gave up).  Read with locmoe_device_flags().
 __device__ int g_device_flags = 0;
 
@@ -188,14 +237,16 @@ template <> struct Oct<LOCMOE_BF16> {
 template <int YDT, int ODT, bool ACC>
 __global__ void __launch_bounds__(kThreads, ACC ? 4 : 6) combine_vec_kernel(const void* __restrict__ y, const int32_t* __restrict__ slot,
                                                                const float* __restrict__ gate_w, void* __restrict__ out,
-                                                               int T, int O, long long rows) {
+                                                               int T, int O, long long rows, int tpc) {
     pdl_wait();
     pdl_trigger();
     constexpr int CH = 2;
     const int lane = threadIdx.x & 31;
-    const int nw = gridDim.x * (blockDim.x >> 5);
     const int nch = (O + CH * kWarp - 1) / (CH * kWarp);
-    for (int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); t < T; t += nw) {
+    // every CTA owns a contiguous run of tpc tokens, so that the grid walks the tokens in ascending order
+    const long long t_lo = (long long)blockIdx.x * tpc;
+    const int t_hi = (int)min((long long)T, t_lo + tpc);
+    for (int t = (int)t_lo + (threadIdx.x >> 5); t < t_hi; t += blockDim.x >> 5) {
         const int s = slot[t];
         const long long obase = (long long)t * O;
         if (s < 0 || s >= rows) {
@@ -282,8 +333,8 @@ int grid_for(long long units, int warps_per_block, int blocks_per_sm) {
 
 }  // namespace
 
-int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const int32_t* inv, void* buf,
-                    int zero_pad, cudaStream_t st) {
+int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const int32_t* inv, const int32_t* slot,
+                    void* buf, int zero_pad, cudaStream_t st) {
     const int esz = s.x_dtype == LOCMOE_F32 ? 4 : 2;
     const size_t rb = (size_t)s.H * esz;
     const bool vec_ok = rb % 16 == 0 && (uintptr_t)x % 16 == 0 && (uintptr_t)buf % 16 == 0;
@@ -323,6 +374,14 @@ int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const 
             }
         }
     }
+    if (vec_ok && slot && !mode && (unsigned long long)s.T * (rb / 16) < 0xf0000000ull) {
+        const unsigned total = (unsigned)((unsigned long long)s.T * (rb / 16));
+        const unsigned per = (unsigned)(kThreads * 4 * kTokIters);
+        const int g = (int)((total + per - 1) / per);
+        const int zrows = (int)((rows + g - 1) / g);
+        return launch_pdl(dispatch_token_kernel, g, kThreads, 0, st, static_cast<const uint4*>(x), slot, inv,
+                          static_cast<uint4*>(buf), total, (unsigned)(rb / 16), s.T, (long long)rows, zero_pad, zrows);
+    }
     if (vec_ok && !(mode && mode[0] == 'v') && (unsigned long long)rows * (rb / 16) < 0xffffffffull) {
         const int fg = flat_grid((unsigned long long)rows * (rb / 16), 4);
         return launch_pdl(dispatch_flat_kernel, fg, kThreads, 0, st, static_cast<const uint4*>(x), inv, static_cast<uint4*>(buf),
@@ -347,6 +406,9 @@ int launch_combine(const locmoe_shape_t& s, int64_t rows, const void* y, int y_d
     // several waves of short CTAs measured fastest (~6 %); a flat (token, octet) mapping like dispatch's measured
     // 202-204 us against 197 us for this warp-per-token kernel on the 65536 x 5120 bf16 case and was dropped
     const int grid = grid_for(s.T, kThreads / 32, 32);
+    // vector kernel: one token per warp in ascending order while the grid stays below 1024 CTAs per SM
+    const int cgrid = grid_for(s.T, kThreads / 32, 1024);
+    const int tpc = (s.T + cgrid - 1) / cgrid;
     if (!vec_ok) {
         combine_scalar_kernel<<<grid, kThreads, 0, st>>>(y, y_dtype, slot, gate_w, out, s.x_dtype, s.T, s.H, rows,
                                                          accumulate);
@@ -355,7 +417,7 @@ int launch_combine(const locmoe_shape_t& s, int64_t rows, const void* y, int y_d
     const int O = s.H / 8;
 #define LOCMOE_COMBINE_CASE(YD, OD, AC)                                                                              \
     if (y_dtype == YD && s.x_dtype == OD && (accumulate != 0) == AC) {                                               \
-        return launch_pdl(combine_vec_kernel<YD, OD, AC>, grid, kThreads, 0, st, y, slot, gate_w, out, s.T, O, (long long)rows); \
+        return launch_pdl(combine_vec_kernel<YD, OD, AC>, cgrid, kThreads, 0, st, y, slot, gate_w, out, s.T, O, (long long)rows, tpc); \
                                                                                      \
     }
     LOCMOE_COMBINE_CASE(LOCMOE_F32, LOCMOE_F32, false)

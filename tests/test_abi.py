@@ -65,7 +65,7 @@ def test_null_pointers_are_rejected_before_any_launch(B):
     lib = B._lib
     sh = B.make_shape(16, 64, 8, 2, 4, B.F32)
     assert lib.locmoe_gate(C.byref(sh), None, None, None, None, None, None, None) == -1
-    assert lib.locmoe_dispatch(C.byref(sh), 4, None, None, None, 1, None) == -1
+    assert lib.locmoe_dispatch(C.byref(sh), 4, None, None, None, None, 1, None) == -1
     assert lib.locmoe_combine(C.byref(sh), 4, None, 0, None, None, None, 0, None) == -1
     rule = B.CapacityRule(1.0, 1.0, -1.0, 0, 0)
     assert lib.locmoe_capacity(C.byref(sh), None, None, C.byref(rule), None, None, None, None, 0, None) == -1

@@ -299,3 +299,30 @@ def test_aux_loss_against_oracle(P):
     B.locmoe_aux_loss(sh, probs, st.load, 0.01, f, Pm, loss2, st.ws)
     torch.cuda.synchronize()
     assert loss2.item() == loss.item()
+
+
+def test_row_major_dispatch_without_slot(P):
+    # locmoe_dispatch with slot = NULL (row-major kernels) writes the same buffer as the token-major call
+    import torch
+    B, W = P.B, P.W
+    w = W.CONFIGS[2].scaled(3000)
+    dev = torch.device("cuda:0")
+    x, src = W.make_tokens(w, dev), W.make_src(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype)
+    Ca = B.conventional_capacity(w.T, sh.D, w.E, 1.0)
+    st = B.make_router(sh, Ca, B.CapacityRule(1.0, 1.0, -1.0, 0, 0), dev)
+    B.router_forward(st, x, src)
+    torch.cuda.synchronize()
+    want = st.buf.clone()
+    assert int((st.inv < 0).sum()) > 0 and int((st.slot < 0).sum()) > 0   # empty rows and dropped tokens both occur
+    st.buf.fill_(7.0)
+    B.locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, None)
+    torch.cuda.synchronize()
+    assert torch.equal(st.buf.view(torch.int16), want.view(torch.int16))
+
+
+def test_flat_dispatch_variant(P, monkeypatch):
+    # the flat (row, vector) row-major kernel, forced although slot[] is supplied
+    monkeypatch.setenv("LOCMOE_DISPATCH", "flat")
+    P.run_staged(P.W.CONFIGS[2].scaled(6000), 1.25, full=True)
+    P.run_staged(P.W.CONFIGS[1], 1.0, layout=1, full=True)
