@@ -82,6 +82,9 @@ def lib():
                                       C.c_void_p, C.c_void_p]
         L.oracle_aux_loss.restype = C.c_double
         L.oracle_aux_loss.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_double, C.c_void_p, C.c_void_p]
+        L.oracle_loc_loss.restype = C.c_double
+        L.oracle_loc_loss.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_double, C.c_double,
+                                      C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -276,3 +279,13 @@ def aux_loss(idx, probs, alpha=0.01):
     P = np.empty(E, np.float64)
     L = lib().oracle_aux_loss(_p(idx), _p(probs), T, E, float(alpha), _p(f), _p(P))
     return L, f, P
+
+
+def loc_loss(counts, E, n_nodes, dev_per_node, level=1, mu=1.0, smooth=1e-3):
+    """(L_loc, D_c rows [G][E], KL per group [G]) of Sec. 3.2.2 under the reading stated in the C source."""
+    counts = np.ascontiguousarray(counts, dtype=np.int32).reshape(n_nodes * dev_per_node, E)
+    G = n_nodes if level else n_nodes * dev_per_node
+    dc = np.empty((G, E), np.float64)
+    kl = np.empty(G, np.float64)
+    L = lib().oracle_loc_loss(_p(counts), E, n_nodes, dev_per_node, int(level), float(mu), float(smooth), _p(dc), _p(kl))
+    return L, dc, kl

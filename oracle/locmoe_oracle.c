@@ -32,13 +32,20 @@
  *
  *   oracle_aux_loss  L_aux = alpha n sum_i f_i P_i (Sec. 3.2.2, first loss
  *                    equation), forward value.
+ *   oracle_loc_loss  L_loc = mu KL(D_c || D_l) (Sec. 3.2.2, second loss
+ *                    equation), forward value, under the reading stated at
+ *                    the function (the paper gives neither mu nor the
+ *                    treatment of experts D_l gives no mass): the arithmetic
+ *                    is pinned, the reading is not -- parity unpinned.
  *   oracle_ffn_rows  expert network of the same equation:
  *                    W_out . GeLU(W_in . x), GeLU(v) = v * Phi(v) with Phi the
  *                    standard Gaussian CDF (Sec. 3.2.1), in double.
  *
  * Parity pins: every function below is pinned by tests/test_oracle_*.py
  * (dense-weight identity, closed forms, library incomplete beta, brute force,
- * round trip).  The locality loss L_loc is not computed here at all.
+ * round trip).  oracle_loc_loss: its KL arithmetic is pinned (closed forms, a
+ * library relative entropy), its reading of the paper's D_c / D_l is a choice:
+ * PARITY UNPINNED for that function.
  */
 #include <math.h>
 #include <stdint.h>
@@ -439,4 +446,48 @@ double oracle_aux_loss(const int32_t *idx, const double *probs, int64_t T, int32
         s += f[i] * P[i];
     }
     return alpha * (double)E * s;
+}
+
+/*
+ * Locality loss (Sec. 3.2.2, second loss equation): L_loc = mu * KL(D_c || D_l), D_c the current assignment
+ * distribution, D_l the fully localised one.  The paper defines neither distribution in symbols; the reading here:
+ * both are joint distributions over (source group s, expert e) pairs, a group being a logical device (level 0) or
+ * a logical node (level 1) and G their number;
+ *   D_c(s, e) = counts[s][e] / T_routed                       (what the batch did),
+ *   D_l(s, e) = (n_s / T_routed) * q_s(e)                     (same sources, every token on a local expert),
+ *   q_s(e)    = (1 - smooth) / (E / G) on the E / G experts group s hosts, + smooth / E on every expert
+ * (smooth > 0 keeps the divergence finite when a token leaves its group).  Then
+ *   KL(D_c || D_l) = sum_s (n_s / T_routed) * KL_s,   KL_s = sum_e c_s(e) ln(c_s(e) / q_s(e)),  c_s = counts[s] / n_s,
+ * with 0 ln 0 = 0 and a group without tokens contributing nothing.
+ * counts [D][E] demanded tokens per (source device, expert); experts are laid out in blocks of E / D per device,
+ * devices in blocks of Dn per node.  dc [G][E] receives c_s, kl [G] receives KL_s.  Returns L_loc.
+ */
+double oracle_loc_loss(const int32_t *counts, int32_t E, int32_t N, int32_t Dn, int32_t level, double mu,
+                       double smooth, double *dc /* [G][E] */, double *kl /* [G] */)
+{
+    const int32_t D = N * Dn, G = level ? N : D, per = D / G, Eg = E / G;
+    double total = 0.0, acc = 0.0;
+    for (int32_t s = 0; s < G; ++s)
+        for (int32_t m = 0; m < per; ++m)
+            for (int32_t e = 0; e < E; ++e) total += (double)counts[(s * per + m) * E + e];
+    for (int32_t s = 0; s < G; ++s) {
+        double ns = 0.0;
+        for (int32_t e = 0; e < E; ++e) {
+            double c = 0.0;
+            for (int32_t m = 0; m < per; ++m) c += (double)counts[(s * per + m) * E + e];
+            dc[s * E + e] = c;
+            ns += c;
+        }
+        double k = 0.0;
+        for (int32_t e = 0; e < E; ++e) {
+            const double c = ns > 0.0 ? dc[s * E + e] / ns : 0.0;
+            const int local = e / Eg == s;
+            const double q = (local ? (1.0 - smooth) / (double)Eg : 0.0) + smooth / (double)E;
+            dc[s * E + e] = c;
+            if (c > 0.0) k += c * log(c / q);
+        }
+        kl[s] = k;
+        if (total > 0.0) acc += ns / total * k;
+    }
+    return mu * acc;
 }
