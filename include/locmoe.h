@@ -234,6 +234,31 @@ int locmoe_aux_loss(const locmoe_shape_t *shape, const float *probs, const int32
                     float *f_out, float *p_out, float *loss_out, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Locality loss, forward value (Sec. 3.2.2, second loss equation):
+ *   L_loc = mu * KL(D_c || D_l),
+ * D_c the current assignment distribution of the batch, D_l the fully localised
+ * one.  The paper gives no symbols for the two, no value of mu and no rule for
+ * experts to which D_l gives no mass; this call fixes the following reading.
+ * A source group s is a logical device (level = 0) or a logical node
+ * (level = 1), G their number (D or N); group s hosts the E / G experts
+ * [s * E / G, (s + 1) * E / G).  With n_s the tokens that group s routed and
+ * T_r their sum,
+ *   D_c(s, e) = counts[s][e] / T_r,
+ *   D_l(s, e) = (n_s / T_r) * q_s(e),
+ *   q_s(e) = (1 - smooth) / (E / G) for the experts s hosts, plus smooth / E for every e,
+ *   KL(D_c || D_l) = sum_s (n_s / T_r) * KL_s,  KL_s = sum_e c_s(e) ln(c_s(e) / q_s(e)),
+ *   c_s(e) = counts[s][e] / n_s, 0 ln 0 = 0, a group without tokens adds nothing.
+ * smooth in [0, 1]; with smooth = 0 a single token outside its group makes the
+ * value +inf.  counts int32[D][E] as written by locmoe_route (summed over the
+ * devices of a node for level 1).  Outputs, all on the device: dc_out
+ * float[G][E] = c_s(e); kl_out double[G] = KL_s; group_tokens int64[G] = n_s;
+ * loss_out double[1].  Arithmetic in fp64, sums in a fixed order.
+ */
+int locmoe_loc_loss(const locmoe_shape_t *shape, const int32_t *counts, int32_t level, double mu,
+                    double smooth, float *dc_out, double *kl_out, int64_t *group_tokens,
+                    double *loss_out, void *stream);
+
+/*
  * Expert feed-forward networks (first equation of Sec. 3.2.1):
  *   y[row] = W_out[e] . GeLU(W_in[e] . buf[row]),  GeLU(v) = v * Phi(v) (erf form),
  * for every row of the dispatched buffer, e being the expert that owns the row.

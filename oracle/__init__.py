@@ -85,6 +85,9 @@ def lib():
         L.oracle_loc_loss.restype = C.c_double
         L.oracle_loc_loss.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_double, C.c_double,
                                       C.c_void_p, C.c_void_p]
+        L.oracle_cos_hist.restype = C.c_int64
+        L.oracle_cos_hist.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_int32,
+                                      C.c_int32, C.c_double, C.c_double, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -289,3 +292,19 @@ def loc_loss(counts, E, n_nodes, dev_per_node, level=1, mu=1.0, smooth=1e-3):
     kl = np.empty(G, np.float64)
     L = lib().oracle_loc_loss(_p(counts), E, n_nodes, dev_per_node, int(level), float(mu), float(smooth), _p(dc), _p(kl))
     return L, dc, kl
+
+
+def cos_hist(x, dtype, E, idx, e, j, nbins, lo=-1.0, hi=1.0):
+    """(n routed to e, hist of cos(x, w_e), hist of cos(x, w_j), per-token cos_e, cos_j) -- Sec. 4.1 diagnostic."""
+    x = _raw(x, dtype)
+    T, H = x.shape
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    he = np.empty(nbins, np.int64)
+    hj = np.empty(nbins, np.int64)
+    ce = np.empty(T, np.float64)
+    cj = np.empty(T, np.float64)
+    n = lib().oracle_cos_hist(_p(x), dtype, T, H, E, _p(idx), int(e), int(j), int(nbins), float(lo), float(hi),
+                              _p(he), _p(hj), _p(ce), _p(cj))
+    if n < 0:
+        raise ValueError("oracle_cos_hist: bad argument")
+    return n, he, hj, ce, cj

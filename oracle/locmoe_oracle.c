@@ -32,6 +32,9 @@
  *
  *   oracle_aux_loss  L_aux = alpha n sum_i f_i P_i (Sec. 3.2.2, first loss
  *                    equation), forward value.
+ *   oracle_cos_hist  the two histograms of the second cosine-frequency figure of
+ *                    Sec. 4.1: tokens routed to one expert, their cosine to that
+ *                    expert's gating weight and to another expert's.
  *   oracle_loc_loss  L_loc = mu KL(D_c || D_l) (Sec. 3.2.2, second loss
  *                    equation), forward value, under the reading stated at
  *                    the function (the paper gives neither mu nor the
@@ -490,4 +493,48 @@ double oracle_loc_loss(const int32_t *counts, int32_t E, int32_t N, int32_t Dn, 
         if (total > 0.0) acc += ns / total * k;
     }
     return mu * acc;
+}
+
+/*
+ * Cosine-frequency diagnostic (Sec. 4.1, second cosine-histogram figure): over the tokens routed to expert e,
+ * the histogram of cos(x, w_e) (the expert the token went to) and the histogram of cos(x, w_j) for another
+ * expert j, with w_i the i-th gating weight (1 on the i-th group of d/n entries, scaled; the scale cancels):
+ *   cos(x, w_i) = (sum of the i-th group of x) / (sqrt(d/n) * |x|),   0 when |x| = 0.
+ * nbins equal bins on [lo, hi); a value below lo counts in the first bin, a value >= hi in the last.
+ * Optional per-token outputs cos_e[T], cos_j[T] (NaN for tokens not routed to e) may be NULL.
+ * Returns the number of tokens routed to e, or -2 on a bad argument.
+ */
+int64_t oracle_cos_hist(const void *x, int dtype, int64_t T, int32_t H, int32_t E, const int32_t *idx, int32_t e,
+                        int32_t j, int32_t nbins, double lo, double hi, int64_t *hist_e, int64_t *hist_j,
+                        double *cos_e, double *cos_j)
+{
+    if (H <= 0 || E <= 0 || H % E != 0 || e < 0 || e >= E || j < 0 || j >= E || nbins < 1 || !(hi > lo)) return -2;
+    const int32_t g = H / E;
+    int64_t n = 0;
+    for (int32_t b = 0; b < nbins; ++b) { hist_e[b] = 0; hist_j[b] = 0; }
+    for (int64_t t = 0; t < T; ++t) {
+        if (cos_e) cos_e[t] = NAN;
+        if (cos_j) cos_j[t] = NAN;
+        if (idx[t] != e) continue;
+        double sq = 0.0, se = 0.0, sj = 0.0;
+        for (int32_t k = 0; k < H; ++k) {
+            const double v = widen(x, dtype, t * H + k);
+            sq += v * v;
+            if (k / g == e) se += v;
+            if (k / g == j) sj += v;
+        }
+        const double den = sqrt((double)g) * sqrt(sq);
+        const double c[2] = { den > 0.0 ? se / den : 0.0, den > 0.0 ? sj / den : 0.0 };
+        int64_t *h[2] = { hist_e, hist_j };
+        for (int q = 0; q < 2; ++q) {
+            double pos = floor((c[q] - lo) / (hi - lo) * (double)nbins);
+            if (pos < 0.0) pos = 0.0;
+            if (pos > (double)(nbins - 1)) pos = (double)(nbins - 1);
+            h[q][(int32_t)pos] += 1;
+        }
+        if (cos_e) cos_e[t] = c[0];
+        if (cos_j) cos_j[t] = c[1];
+        ++n;
+    }
+    return n;
 }

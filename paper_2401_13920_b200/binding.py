@@ -24,7 +24,7 @@ FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
     "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route",
-    "locmoe_dispatch", "locmoe_combine", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
+    "locmoe_dispatch", "locmoe_combine", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
 
@@ -80,6 +80,7 @@ def _load() -> C.CDLL:
     lib.locmoe_moe_layer.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(CapacityRule), i32, i32, vp, vp,
                                      C.POINTER(LayerBuffers), vp, vp]
     lib.locmoe_aux_loss.argtypes = [C.POINTER(Shape), vp, vp, C.c_float, vp, vp, vp, vp, C.c_size_t, vp]
+    lib.locmoe_loc_loss.argtypes = [C.POINTER(Shape), vp, i32, C.c_double, C.c_double, vp, vp, vp, vp, vp]
     lib.locmoe_launch_counts.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32 * 5)]
     lib.locmoe_device_flags.argtypes = [C.POINTER(C.c_int32), vp]
     lib.locmoe_status_string.argtypes = [C.c_int]
@@ -269,6 +270,18 @@ def locmoe_aux_loss(shape: Shape, probs, load, alpha, f_out, p_out, loss_out, ws
     return _check("locmoe_aux_loss", _lib.locmoe_aux_loss(C.byref(shape), _ptr(probs), _ptr(load), float(alpha),
                                                           _ptr(f_out), _ptr(p_out), _ptr(loss_out), _ptr(ws),
                                                           ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def locmoe_loc_loss(shape: Shape, counts, level, mu, smooth, dc_out, kl_out, group_tokens, loss_out, stream=None) -> int:
+    G = shape.n_nodes if level else shape.D
+    _want(counts, torch.int32, shape.D * shape.E, "counts")
+    _want(dc_out, torch.float32, G * shape.E, "dc_out")
+    _want(kl_out, torch.float64, G, "kl_out")
+    _want(group_tokens, torch.int64, G, "group_tokens")
+    _want(loss_out, torch.float64, 1, "loss_out")
+    return _check("locmoe_loc_loss", _lib.locmoe_loc_loss(C.byref(shape), _ptr(counts), int(level), float(mu), float(smooth),
+                                                          _ptr(dc_out), _ptr(kl_out), _ptr(group_tokens), _ptr(loss_out),
+                                                          _stream(stream)))
 
 
 def layer_buffers(st: "RouterState", h1=None, y=None) -> LayerBuffers:

@@ -157,6 +157,18 @@ int locmoe_aux_loss(const locmoe_shape_t* shape, const float* probs, const int32
     return launch_aux_loss(*shape, probs, load, alpha, f_out, p_out, loss_out, ws, static_cast<cudaStream_t>(stream));
 }
 
+int locmoe_loc_loss(const locmoe_shape_t* shape, const int32_t* counts, int32_t level, double mu, double smooth,
+                    float* dc_out, double* kl_out, int64_t* group_tokens, double* loss_out, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!counts || !dc_out || !kl_out || !group_tokens || !loss_out) return LOCMOE_ERR_NULL;
+    if (level != 0 && level != 1) return LOCMOE_ERR_DTYPE;
+    if (!(smooth >= 0.0 && smooth <= 1.0)) return LOCMOE_ERR_SHAPE;
+    if ((uintptr_t)kl_out % 8 || (uintptr_t)group_tokens % 8 || (uintptr_t)loss_out % 8) return LOCMOE_ERR_ALIGN;
+    return launch_loc_loss(*shape, counts, level, mu, smooth, dc_out, kl_out, reinterpret_cast<long long*>(group_tokens),
+                           loss_out, static_cast<cudaStream_t>(stream));
+}
+
 int locmoe_expert_ffn(const locmoe_shape_t* shape, int32_t C_alloc, int32_t F, const void* buf, const void* w_in,
                       const void* w_out, void* h1, void* y, int32_t y_dtype, void* stream) {
     int rc = check_shape(shape);

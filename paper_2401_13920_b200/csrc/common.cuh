@@ -58,6 +58,9 @@ size_t aux_ws_bytes(const locmoe_shape_t& s);
 int launch_aux_loss(const locmoe_shape_t& s, const float* probs, const int32_t* load, float alpha, float* f, float* P,
                     float* loss, void* ws, cudaStream_t st);
 
+int launch_loc_loss(const locmoe_shape_t& s, const int32_t* counts, int level, double mu, double smooth, float* dc,
+                    double* kl, long long* group_tokens, double* loss, cudaStream_t st);
+
 int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* buf, const void* w_in,
                       const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st);
 int read_ffn_flags(int* out, cudaStream_t st);

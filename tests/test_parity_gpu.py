@@ -301,6 +301,36 @@ def test_aux_loss_against_oracle(P):
     assert loss2.item() == loss.item()
 
 
+@pytest.mark.parametrize("cfg,T,level", [(2, 5000, 0), (2, 5000, 1), (3, 8229, 1), (1, 4096, 0)])
+def test_locality_loss_against_oracle(P, cfg, T, level):
+    # counts from the CUDA route stage (bit-exact against the oracle elsewhere) -> L_loc in fp64 on both sides
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    w = P.W.CONFIGS[cfg].scaled(T)
+    x, src = W.make_tokens(w, dev), W.make_src(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype)
+    Ca = B.conventional_capacity(w.T, sh.D, w.E, 1.0)
+    st = B.make_router(sh, Ca, B.CapacityRule(1.0, 1.0, -1.0, 0, 0), dev)
+    B.router_forward(st, x, src)
+    G = w.n_nodes if level else sh.D
+    dc = torch.empty(G, w.E, device=dev)
+    kl = torch.empty(G, dtype=torch.float64, device=dev)
+    nt = torch.empty(G, dtype=torch.int64, device=dev)
+    loss = torch.empty(1, dtype=torch.float64, device=dev)
+    B.locmoe_loc_loss(sh, st.counts, level, 0.5, 1e-3, dc, kl, nt, loss)
+    torch.cuda.synchronize()
+    counts = st.counts.cpu().numpy()
+    L, dc_o, kl_o = P.oracle.loc_loss(counts, w.E, w.n_nodes, w.dev_per_node, level=level, mu=0.5, smooth=1e-3)
+    assert np.array_equal(nt.cpu().numpy(), counts.reshape(G, -1).sum(1))
+    assert np.allclose(kl.cpu().numpy(), kl_o, rtol=1e-12, atol=1e-15)
+    assert np.allclose(dc.cpu().numpy(), dc_o, rtol=1e-6, atol=0)
+    assert abs(loss.item() - L) <= 1e-12 * abs(L) and L > 0
+    loss2 = torch.empty(1, dtype=torch.float64, device=dev)
+    B.locmoe_loc_loss(sh, st.counts, level, 0.5, 1e-3, dc, kl, nt, loss2)
+    torch.cuda.synchronize()
+    assert loss2.item() == loss.item()
+
+
 def test_row_major_dispatch_without_slot(P):
     # locmoe_dispatch with slot = NULL (row-major kernels) writes the same buffer as the token-major call
     import torch
