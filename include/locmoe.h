@@ -259,6 +259,22 @@ int locmoe_loc_loss(const locmoe_shape_t *shape, const int32_t *counts, int32_t 
                     double *loss_out, void *stream);
 
 /*
+ * Cosine-frequency diagnostic (Sec. 4.1, the second cosine-histogram figure):
+ * over the tokens t with idx[t] == expert, the histogram of cos(x_t, w_expert)
+ * (the gating weight of the expert the token was routed to) and the histogram
+ * of cos(x_t, w_other), where cos(x, w_i) = (sum of the i-th group of d/n
+ * entries of x) / (sqrt(d/n) * |x|), 0 for a zero token.  nbins equal bins on
+ * [lo, hi); a value below lo counts in the first bin, a value >= hi in the
+ * last.  x [T][H] of shape->x_dtype, idx int32[T] as written by locmoe_gate.
+ * Outputs on the device: hist_routed / hist_other int32[nbins], n_routed
+ * int32[1] (tokens routed to `expert`); they are zeroed first.  Cosines and the
+ * bin index are computed in fp32.
+ */
+int locmoe_cos_hist(const locmoe_shape_t *shape, const void *x, const int32_t *idx, int32_t expert,
+                    int32_t other, int32_t nbins, float lo, float hi, int32_t *hist_routed,
+                    int32_t *hist_other, int32_t *n_routed, void *stream);
+
+/*
  * Expert feed-forward networks (first equation of Sec. 3.2.1):
  *   y[row] = W_out[e] . GeLU(W_in[e] . buf[row]),  GeLU(v) = v * Phi(v) (erf form),
  * for every row of the dispatched buffer, e being the expert that owns the row.

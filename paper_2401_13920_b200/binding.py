@@ -24,7 +24,7 @@ FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
     "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route",
-    "locmoe_dispatch", "locmoe_combine", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
+    "locmoe_dispatch", "locmoe_combine", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
 
@@ -81,6 +81,7 @@ def _load() -> C.CDLL:
                                      C.POINTER(LayerBuffers), vp, vp]
     lib.locmoe_aux_loss.argtypes = [C.POINTER(Shape), vp, vp, C.c_float, vp, vp, vp, vp, C.c_size_t, vp]
     lib.locmoe_loc_loss.argtypes = [C.POINTER(Shape), vp, i32, C.c_double, C.c_double, vp, vp, vp, vp, vp]
+    lib.locmoe_cos_hist.argtypes = [C.POINTER(Shape), vp, vp, i32, i32, i32, C.c_float, C.c_float, vp, vp, vp, vp]
     lib.locmoe_launch_counts.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32 * 5)]
     lib.locmoe_device_flags.argtypes = [C.POINTER(C.c_int32), vp]
     lib.locmoe_status_string.argtypes = [C.c_int]
@@ -282,6 +283,18 @@ def locmoe_loc_loss(shape: Shape, counts, level, mu, smooth, dc_out, kl_out, gro
     return _check("locmoe_loc_loss", _lib.locmoe_loc_loss(C.byref(shape), _ptr(counts), int(level), float(mu), float(smooth),
                                                           _ptr(dc_out), _ptr(kl_out), _ptr(group_tokens), _ptr(loss_out),
                                                           _stream(stream)))
+
+
+def locmoe_cos_hist(shape: Shape, x, idx, expert, other, nbins, lo, hi, hist_routed, hist_other, n_routed, stream=None) -> int:
+    dt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
+    _want(x, dt, shape.T * shape.H, "x")
+    _want(idx, torch.int32, shape.T, "idx")
+    _want(hist_routed, torch.int32, nbins, "hist_routed")
+    _want(hist_other, torch.int32, nbins, "hist_other")
+    _want(n_routed, torch.int32, 1, "n_routed")
+    return _check("locmoe_cos_hist", _lib.locmoe_cos_hist(C.byref(shape), _ptr(x), _ptr(idx), int(expert), int(other),
+                                                          int(nbins), float(lo), float(hi), _ptr(hist_routed),
+                                                          _ptr(hist_other), _ptr(n_routed), _stream(stream)))
 
 
 def layer_buffers(st: "RouterState", h1=None, y=None) -> LayerBuffers:

@@ -169,6 +169,19 @@ int locmoe_loc_loss(const locmoe_shape_t* shape, const int32_t* counts, int32_t 
                            loss_out, static_cast<cudaStream_t>(stream));
 }
 
+int locmoe_cos_hist(const locmoe_shape_t* shape, const void* x, const int32_t* idx, int32_t expert, int32_t other,
+                    int32_t nbins, float lo, float hi, int32_t* hist_routed, int32_t* hist_other, int32_t* n_routed,
+                    void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!x || !idx || !hist_routed || !hist_other || !n_routed) return LOCMOE_ERR_NULL;
+    if (expert < 0 || expert >= shape->E || other < 0 || other >= shape->E || nbins < 1 || !(hi > lo)) return LOCMOE_ERR_SHAPE;
+    const int esz = shape->x_dtype == LOCMOE_F32 ? 4 : 2;
+    if ((uintptr_t)x % esz) return LOCMOE_ERR_ALIGN;
+    return launch_cos_hist(*shape, x, idx, expert, other, nbins, lo, hi, hist_routed, hist_other, n_routed,
+                           static_cast<cudaStream_t>(stream));
+}
+
 int locmoe_expert_ffn(const locmoe_shape_t* shape, int32_t C_alloc, int32_t F, const void* buf, const void* w_in,
                       const void* w_out, void* h1, void* y, int32_t y_dtype, void* stream) {
     int rc = check_shape(shape);

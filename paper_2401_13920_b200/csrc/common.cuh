@@ -61,6 +61,9 @@ int launch_aux_loss(const locmoe_shape_t& s, const float* probs, const int32_t* 
 int launch_loc_loss(const locmoe_shape_t& s, const int32_t* counts, int level, double mu, double smooth, float* dc,
                     double* kl, long long* group_tokens, double* loss, cudaStream_t st);
 
+int launch_cos_hist(const locmoe_shape_t& s, const void* x, const int32_t* idx, int e, int j, int nbins, float lo, float hi,
+                    int32_t* hist_e, int32_t* hist_j, int32_t* n_routed, cudaStream_t st);
+
 int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* buf, const void* w_in,
                       const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st);
 int read_ffn_flags(int* out, cudaStream_t st);

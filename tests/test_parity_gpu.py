@@ -331,6 +331,39 @@ def test_locality_loss_against_oracle(P, cfg, T, level):
     assert loss2.item() == loss.item()
 
 
+@pytest.mark.parametrize("cfg,T,dtype_name", [(2, 20000, "bf16"), (1, 4096, "f32"), (3, 8229, "bf16")])
+def test_cosine_histograms_against_oracle(P, cfg, T, dtype_name):
+    # bins are decided in fp32 by the kernel and in fp64 by the oracle: a token whose cosine lies within 1e-6 of a
+    # bin edge may fall on either side; everything else must agree exactly
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    w = P.W.CONFIGS[cfg].scaled(T)
+    x = W.make_tokens(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype)
+    idx = torch.empty(w.T, dtype=torch.int32, device=dev)
+    gw = torch.empty(w.T, device=dev); cs = torch.empty(w.T, device=dev)
+    B.locmoe_gate(sh, x, None, idx, gw, cs, None)
+    nb, lo, hi = 64, -0.125, 0.25
+    he = torch.empty(nb, dtype=torch.int32, device=dev); hj = torch.empty(nb, dtype=torch.int32, device=dev)
+    n = torch.empty(1, dtype=torch.int32, device=dev)
+    e = int(torch.bincount(idx.long(), minlength=w.E).argmax())
+    j = (e + 1) % w.E
+    B.locmoe_cos_hist(sh, x, idx, e, j, nb, lo, hi, he, hj, n)
+    torch.cuda.synchronize()
+    idx_h = idx.cpu().numpy()
+    n_o, he_o, hj_o, ce, cj = P.oracle.cos_hist(W.host_bits(x), sh.x_dtype, w.E, idx_h, e, j, nb, lo, hi)
+    assert n.item() == n_o == int((idx_h == e).sum()) and n_o > 0
+    edges = lo + (hi - lo) * np.arange(nb + 1) / nb
+    sel = idx_h == e
+    for got, want, c in ((he, he_o, ce[sel]), (hj, hj_o, cj[sel])):
+        got = got.cpu().numpy().astype(np.int64)
+        assert got.sum() == n_o
+        near = int((np.abs(c[:, None] - edges[None, :]).min(1) < 1e-6).sum())
+        assert np.abs(got - want).sum() <= 2 * near
+    # the routed cosines are the gate's own cos_sim output
+    assert np.allclose(cs.cpu().numpy()[sel], ce[sel], rtol=1e-5, atol=1e-7)
+
+
 def test_row_major_dispatch_without_slot(P):
     # locmoe_dispatch with slot = NULL (row-major kernels) writes the same buffer as the token-major call
     import torch
