@@ -82,7 +82,9 @@ typedef struct {
     double capacity_factor; /* c_f of Sec. 3.2.3; 0 = use the minimum alone            */
     double delta_override;  /* < 0: measure delta from the batch; else use this value  */
     int32_t bound_form;     /* LOCMOE_BOUND_*: which form of Theorem 1                 */
-    int32_t reserved;       /* must be 0                                               */
+    int32_t T_global;       /* 0: the batch is shape->T; > 0: tokens of the whole batch
+                             * when this call sees one rank's share (with the whole
+                             * batch's delta passed as delta_override)                  */
 } locmoe_capacity_rule_t;
 
 /* Capacity record (written on the device by locmoe_capacity). */
@@ -221,6 +223,38 @@ int locmoe_dispatch(const locmoe_shape_t *shape, int32_t C_alloc, const void *x,
 int locmoe_combine(const locmoe_shape_t *shape, int32_t C_alloc, const void *y, int32_t y_dtype,
                    const int32_t *slot, const float *gate_w, void *out, int32_t accumulate,
                    void *stream);
+
+/*
+ * Dispatch and combine fused with the exchange around the experts (Sec. 3.2.4:
+ * the All-to-All before and after the expert networks), for one process per
+ * GPU.  Every rank routes the tokens of its own logical source devices
+ * [src_lo, src_hi) with the shape of the WHOLE logical map (n_nodes,
+ * dev_per_node, E; shape->T = this rank's tokens; layout must be
+ * LOCMOE_LAYOUT_RECV), so slot / inv index the global receive-side buffer of
+ * D * E * C_alloc rows.  That buffer is spread over n_peers GPUs, expert-major:
+ * peer q holds the rows [q * R, (q + 1) * R), R = D * E * C_alloc / n_peers
+ * (n_peers divides D, at most 64).
+ *
+ * locmoe_dispatch_peer stores each kept token's row directly into the buffer of
+ * the peer that hosts its expert (peer_bufs[q], base of peer q's R rows, a
+ * pointer valid on this GPU: its own allocation or a peer mapping) and, with
+ * zero_pad, zero-fills the empty rows whose source device is its own; rows of
+ * other ranks' sources are left alone.  locmoe_combine_peer reads the expert
+ * output row of each kept token from peer_y[q] and writes
+ * out[t] = gate_w[t] * y[slot[t]] (0 for a dropped token), as locmoe_combine.
+ * peer_bufs / peer_y are HOST arrays of n_peers device pointers, 16-byte
+ * aligned; rows must be a multiple of 16 bytes.  Plain loads and stores only
+ * (no bulk copies, no multicast).  Nothing here waits for another GPU: the
+ * caller orders dispatch -> experts -> combine across ranks (a barrier after
+ * the stream has been synchronised).
+ */
+int locmoe_dispatch_peer(const locmoe_shape_t *shape, int32_t C_alloc, const void *x,
+                         const int32_t *inv, const int32_t *slot, void *const *peer_bufs,
+                         int32_t n_peers, int32_t src_lo, int32_t src_hi, int32_t zero_pad,
+                         void *stream);
+int locmoe_combine_peer(const locmoe_shape_t *shape, int32_t C_alloc, void *const *peer_y,
+                        int32_t n_peers, int32_t y_dtype, const int32_t *slot, const float *gate_w,
+                        void *out, void *stream);
 
 /*
  * Auxiliary load-balance loss, forward value (Sec. 3.2.2):

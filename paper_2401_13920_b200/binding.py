@@ -24,7 +24,7 @@ FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
     "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route",
-    "locmoe_dispatch", "locmoe_combine", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
+    "locmoe_dispatch", "locmoe_combine", "locmoe_dispatch_peer", "locmoe_combine_peer", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
 
@@ -39,7 +39,7 @@ class Shape(C.Structure):
 
 class CapacityRule(C.Structure):
     _fields_ = [("min_mult", C.c_double), ("capacity_factor", C.c_double), ("delta_override", C.c_double),
-                ("bound_form", C.c_int32), ("reserved", C.c_int32)]
+                ("bound_form", C.c_int32), ("T_global", C.c_int32)]
 
 
 class Capacity(C.Structure):
@@ -82,6 +82,8 @@ def _load() -> C.CDLL:
     lib.locmoe_aux_loss.argtypes = [C.POINTER(Shape), vp, vp, C.c_float, vp, vp, vp, vp, C.c_size_t, vp]
     lib.locmoe_loc_loss.argtypes = [C.POINTER(Shape), vp, i32, C.c_double, C.c_double, vp, vp, vp, vp, vp]
     lib.locmoe_cos_hist.argtypes = [C.POINTER(Shape), vp, vp, i32, i32, i32, C.c_float, C.c_float, vp, vp, vp, vp]
+    lib.locmoe_dispatch_peer.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, C.POINTER(vp), i32, i32, i32, i32, vp]
+    lib.locmoe_combine_peer.argtypes = [C.POINTER(Shape), i32, C.POINTER(vp), i32, i32, vp, vp, vp, vp]
     lib.locmoe_launch_counts.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32 * 5)]
     lib.locmoe_device_flags.argtypes = [C.POINTER(C.c_int32), vp]
     lib.locmoe_status_string.argtypes = [C.c_int]
@@ -271,6 +273,34 @@ def locmoe_aux_loss(shape: Shape, probs, load, alpha, f_out, p_out, loss_out, ws
     return _check("locmoe_aux_loss", _lib.locmoe_aux_loss(C.byref(shape), _ptr(probs), _ptr(load), float(alpha),
                                                           _ptr(f_out), _ptr(p_out), _ptr(loss_out), _ptr(ws),
                                                           ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def _ptr_table(ptrs):
+    """Host array of device pointers (ints or CUDA tensors) for the peer calls."""
+    vals = [p.data_ptr() if hasattr(p, "data_ptr") else int(p) for p in ptrs]
+    return (C.c_void_p * len(vals))(*vals), len(vals)
+
+
+def locmoe_dispatch_peer(shape: Shape, C_alloc, x, inv, slot, peer_bufs, src_lo, src_hi, zero_pad=True, stream=None) -> int:
+    rows = shape.D * shape.E * C_alloc
+    dt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
+    _want(x, dt, shape.T * shape.H, "x")
+    _want(inv, torch.int32, rows, "inv")
+    _want(slot, torch.int32, shape.T, "slot")
+    table, n = _ptr_table(peer_bufs)
+    return _check("locmoe_dispatch_peer", _lib.locmoe_dispatch_peer(C.byref(shape), int(C_alloc), _ptr(x), _ptr(inv), _ptr(slot),
+                                                                    table, n, int(src_lo), int(src_hi), 1 if zero_pad else 0,
+                                                                    _stream(stream)))
+
+
+def locmoe_combine_peer(shape: Shape, C_alloc, peer_y, y_dtype, slot, gate_w, out, stream=None) -> int:
+    dt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
+    _want(slot, torch.int32, shape.T, "slot")
+    _want(gate_w, torch.float32, shape.T, "gate_w")
+    _want(out, dt, shape.T * shape.H, "out")
+    table, n = _ptr_table(peer_y)
+    return _check("locmoe_combine_peer", _lib.locmoe_combine_peer(C.byref(shape), int(C_alloc), table, n, int(y_dtype), _ptr(slot),
+                                                                  _ptr(gate_w), _ptr(out), _stream(stream)))
 
 
 def locmoe_loc_loss(shape: Shape, counts, level, mu, smooth, dc_out, kl_out, group_tokens, loss_out, stream=None) -> int:

@@ -87,6 +87,7 @@ int locmoe_capacity(const locmoe_shape_t* shape, const int32_t* idx, const float
     if (!idx || !cos_sim || !rule || !delta_e || !theta_e || !cap_dev) return LOCMOE_ERR_NULL;
     if (shape->H < 2) return LOCMOE_ERR_SHAPE;
     if (rule->bound_form < LOCMOE_BOUND_BETA || rule->bound_form > LOCMOE_BOUND_EXP) return LOCMOE_ERR_DTYPE;
+    if (rule->T_global < 0) return LOCMOE_ERR_SHAPE;
     if (!(rule->min_mult >= 0.0) || !(rule->capacity_factor >= 0.0) || rule->delta_override != rule->delta_override)
         return LOCMOE_ERR_SHAPE;
     if (!ws || ws_bytes < capacity_ws_bytes(*shape) || (uintptr_t)ws % 256) return LOCMOE_ERR_WORKSPACE;
@@ -180,6 +181,52 @@ int locmoe_cos_hist(const locmoe_shape_t* shape, const void* x, const int32_t* i
     if ((uintptr_t)x % esz) return LOCMOE_ERR_ALIGN;
     return launch_cos_hist(*shape, x, idx, expert, other, nbins, lo, hi, hist_routed, hist_other, n_routed,
                            static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+// Shared checks of the two peer calls: receive-side layout, experts split evenly over at most 64 peers.
+int check_peers(const locmoe_shape_t* shape, void* const* peers, int32_t n_peers) {
+    if (!peers) return LOCMOE_ERR_NULL;
+    if (shape->layout != LOCMOE_LAYOUT_RECV) return LOCMOE_ERR_DTYPE;
+    const int D = shape->n_nodes * shape->dev_per_node;
+    if (n_peers < 1 || n_peers > 64 || D % n_peers != 0) return LOCMOE_ERR_SHAPE;
+    for (int q = 0; q < n_peers; ++q) {
+        if (!peers[q]) return LOCMOE_ERR_NULL;
+        if ((uintptr_t)peers[q] % 16) return LOCMOE_ERR_ALIGN;
+    }
+    return LOCMOE_OK;
+}
+}  // namespace
+
+int locmoe_dispatch_peer(const locmoe_shape_t* shape, int32_t C_alloc, const void* x, const int32_t* inv,
+                         const int32_t* slot, void* const* peer_bufs, int32_t n_peers, int32_t src_lo, int32_t src_hi,
+                         int32_t zero_pad, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!x || !inv || !slot) return LOCMOE_ERR_NULL;
+    if ((rc = check_peers(shape, peer_bufs, n_peers))) return rc;
+    const long long rows = buffer_rows(shape, C_alloc);
+    if (rows < 0) return LOCMOE_ERR_SHAPE;
+    const int D = shape->n_nodes * shape->dev_per_node;
+    if (src_lo < 0 || src_hi > D || src_lo > src_hi) return LOCMOE_ERR_SHAPE;
+    const size_t rb = (size_t)shape->H * (shape->x_dtype == LOCMOE_F32 ? 4 : 2);
+    if (rb % 16 || (uintptr_t)x % 16) return LOCMOE_ERR_ALIGN;
+    if ((unsigned long long)shape->T * (rb / 16) >= 0xf0000000ull) return LOCMOE_ERR_SHAPE;
+    return launch_dispatch_peer(*shape, C_alloc, rows, x, inv, slot, peer_bufs, n_peers, src_lo, src_hi, zero_pad,
+                                static_cast<cudaStream_t>(stream));
+}
+
+int locmoe_combine_peer(const locmoe_shape_t* shape, int32_t C_alloc, void* const* peer_y, int32_t n_peers, int32_t y_dtype,
+                        const int32_t* slot, const float* gate_w, void* out, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!slot || !gate_w || !out) return LOCMOE_ERR_NULL;
+    if (y_dtype != LOCMOE_F32 && y_dtype != LOCMOE_BF16) return LOCMOE_ERR_DTYPE;
+    if ((rc = check_peers(shape, peer_y, n_peers))) return rc;
+    const long long rows = buffer_rows(shape, C_alloc);
+    if (rows < 0) return LOCMOE_ERR_SHAPE;
+    if (shape->H % 8 || (uintptr_t)out % 16) return LOCMOE_ERR_ALIGN;
+    return launch_combine_peer(*shape, rows, peer_y, n_peers, y_dtype, slot, gate_w, out, static_cast<cudaStream_t>(stream));
 }
 
 int locmoe_expert_ffn(const locmoe_shape_t* shape, int32_t C_alloc, int32_t F, const void* buf, const void* w_in,

@@ -152,7 +152,8 @@ __device__ void capacity_finish(FinishShared& fs, const uint32_t* __restrict__ g
     __syncthreads();
     if (role != 0) return;
 
-    const double n = (double)E, dT = (double)T, dD = (double)D;
+    // the batch the rule counts: the caller's whole batch when this call sees one rank's share of it
+    const double n = (double)E, dT = (double)(rule.T_global > 0 ? rule.T_global : T), dD = (double)D;
     double p;
     if (delta <= 0.0) p = 1.0;
     else if (delta >= 1.0) p = 0.0;

@@ -64,6 +64,12 @@ int launch_loc_loss(const locmoe_shape_t& s, const int32_t* counts, int level, d
 int launch_cos_hist(const locmoe_shape_t& s, const void* x, const int32_t* idx, int e, int j, int nbins, float lo, float hi,
                     int32_t* hist_e, int32_t* hist_j, int32_t* n_routed, cudaStream_t st);
 
+int launch_dispatch_peer(const locmoe_shape_t& s, int C_alloc, int64_t rows, const void* x, const int32_t* inv,
+                         const int32_t* slot, void* const* peer_bufs, int n_peers, int src_lo, int src_hi, int zero_pad,
+                         cudaStream_t st);
+int launch_combine_peer(const locmoe_shape_t& s, int64_t rows, void* const* peer_y, int n_peers, int y_dtype,
+                        const int32_t* slot, const float* gate_w, void* out, cudaStream_t st);
+
 int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* buf, const void* w_in,
                       const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st);
 int read_ffn_flags(int* out, cudaStream_t st);

@@ -72,3 +72,34 @@ class ExchangePlan:
         send = torch.empty_like(arrived)
         send.index_copy_(0, self.send_cells.to(cells.device), arrived)
         return send.reshape(recv_local.shape)
+
+
+class PeerBuffers:
+    """Receive buffers of all ranks, addressable from every rank, for the fused dispatch / combine calls.
+
+    Rank q holds the rows [q * R, (q + 1) * R) of the global receive-side buffer (R = rows_per_rank).  With one rank
+    the buffer is an ordinary tensor.  With several, it is allocated as torch symmetric memory, whose rendezvous
+    hands every rank a pointer to every peer's buffer (a peer mapping over NVLink); ``pointers`` is the table the
+    C-ABI calls take.  ``barrier()`` orders the steps across ranks: call it (after synchronising the stream that ran
+    the kernels) between dispatch, the experts and combine.  No multicast mapping is created or used.
+    """
+
+    def __init__(self, rows_per_rank: int, H: int, dtype: torch.dtype, device, group=None):
+        self.group = group
+        world = dist.get_world_size(group) if dist.is_available() and dist.is_initialized() else 1
+        self.world = world
+        if world == 1:
+            self.local = torch.empty(rows_per_rank, H, dtype=dtype, device=device)
+            self.pointers = [self.local.data_ptr()]
+            self._handle = None
+        else:
+            import torch.distributed._symmetric_memory as symm
+            self.local = symm.empty(rows_per_rank, H, dtype=dtype, device=device)
+            self._handle = symm.rendezvous(self.local, group=group if group is not None else dist.group.WORLD)
+            self.pointers = [int(p) for p in self._handle.buffer_ptrs]
+
+    def barrier(self, stream=None):
+        if self.world == 1:
+            return
+        (stream or torch.cuda.current_stream()).synchronize()
+        dist.barrier(group=self.group)

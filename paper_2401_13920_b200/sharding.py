@@ -51,3 +51,20 @@ def aggregate_throughput(units_per_rank: int, steps: int, elapsed_ms_local: floa
     """Whole-job units per second: all ranks' units over the slowest rank's time."""
     ms = max_over_ranks(elapsed_ms_local, device)
     return world * units_per_rank * steps / (ms * 1e-3)
+
+
+def global_capacity_inputs(delta_e_local: torch.Tensor, T_local: int, group=None):
+    """What every rank needs to evaluate the capacity rule of the WHOLE batch from its own share.
+
+    delta_e_local: float32[E], the per-expert minimum cosines of this rank's tokens as written by the capacity
+    call (1.0 for an expert without tokens).  Returns (delta, T_global): the batch-wide minimum over experts and
+    ranks, clamped to [0, 1] exactly as the single-GPU call clamps it, and the total token count.  Pass them to
+    the capacity rule as ``delta_override`` and ``T_global``; every rank then derives the same capacities.
+    """
+    d = delta_e_local.detach().to(torch.float32).clone()
+    n = torch.tensor([int(T_local)], dtype=torch.int64, device=d.device)
+    if dist.is_available() and dist.is_initialized():
+        dist.all_reduce(d, op=dist.ReduceOp.MIN, group=group)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM, group=group)
+    delta = float(d.min().item())
+    return min(max(delta, 0.0), 1.0), int(n.item())

@@ -1,0 +1,135 @@
+"""Dispatch / combine fused with the exchange (peer stores and loads), with the ranks emulated on one GPU.
+
+Every emulated rank is a separate set of calls on its own tokens (those of its logical source devices) and writes
+through the same pointer table the multi-GPU run would use; here all "peer" buffers live on the one GPU.  No kernel
+waits on another, so running the ranks one after the other is the same computation.  The concatenated receive
+buffers must equal the oracle's receive-side buffer of the whole batch bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    import oracle
+    oracle.build()
+    from tests import parity
+    return parity
+
+
+CASES = [
+    dict(T=3000, H=512, E=16, n_nodes=2, dev_per_node=4, dtype="bf16", world=2),
+    dict(T=3000, H=512, E=16, n_nodes=2, dev_per_node=4, dtype="f32", world=4),
+    dict(T=2500, H=1024, E=32, n_nodes=4, dev_per_node=2, dtype="bf16", world=8),
+    dict(T=1500, H=5120, E=64, n_nodes=8, dev_per_node=8, dtype="bf16", world=4, src="mod"),
+    dict(T=700, H=256, E=8, n_nodes=2, dev_per_node=2, dtype="f32", world=1),
+]
+
+
+@pytest.mark.parametrize("case", CASES)
+def test_emulated_ranks_match_the_oracles_receive_buffer(P, case):
+    from paper_2401_13920_b200 import sharding
+    W, B, oracle = P.W, P.B, P.oracle
+    case = dict(case)
+    world = case.pop("world")
+    dev = torch.device("cuda:0")
+    w = W.Workload(name="peer", config=7, tokens="normal", **{"src": "uniform", **case})
+    x, src = W.make_tokens(w, dev), W.make_src(w, dev)
+    D = w.n_nodes * w.dev_per_node
+    cf = 1.0
+    Ca = B.conventional_capacity(w.T, D, w.E, cf)
+    rule = B.CapacityRule(1.0, cf, -1.0, 0, 0)
+
+    # the whole batch on one GPU gives the capacity record every rank uses (a multi-GPU run all-reduces the minima)
+    sh_g = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, B.LAYOUT_RECV)
+    st_g = B.make_router(sh_g, Ca, rule, dev)
+    B.router_forward(st_g, x, src)
+    torch.cuda.synchronize()
+    cap = B.locmoe_capacity_read(st_g.cap_dev)
+    idx_h, src_h = st_g.idx.cpu().numpy(), src.cpu().numpy()
+    ref = oracle.route(idx_h, src_h, w.E, w.n_nodes, w.dev_per_node, cap.C_local, Ca, B.LAYOUT_RECV)
+    rows = D * w.E * Ca
+    want = oracle.dispatch(W.host_bits(x), sh_g.x_dtype, ref.slot, rows)
+    assert (ref.inv < 0).any() and (ref.slot < 0).any()
+
+    rpp = rows // world
+    sentinel = 1.5
+    bufs = [torch.full((rpp, w.H), sentinel, dtype=x.dtype, device=dev) for _ in range(world)]
+    ranks = []
+    # phase 1 on every rank: gate and the per-expert minima of its own tokens; the minimum over the ranks (an
+    # All-Reduce MIN in a multi-GPU run, sharding.global_capacity_inputs) gives the batch-wide delta
+    pre = []
+    for q in range(world):
+        sel = sharding.shard_by_source(src_h, D, world, q)
+        sel_d = torch.as_tensor(sel, device=dev)
+        x_q, src_q = x[sel_d].contiguous(), src[sel_d].contiguous()
+        sh_q = B.make_shape(len(sel), w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, B.LAYOUT_RECV)
+        st_q = B.make_router(sh_q, Ca, rule, dev)
+        B.locmoe_gate(sh_q, x_q, None, st_q.idx, st_q.gate_w, st_q.cos_sim, None)
+        B.locmoe_capacity(sh_q, st_q.idx, st_q.cos_sim, rule, st_q.delta_e, st_q.theta_e, st_q.cap_dev, st_q.ws)
+        pre.append((sel, sel_d, x_q, src_q, sh_q, st_q))
+    torch.cuda.synchronize()
+    delta = min(max(min(float(p[5].delta_e.min().item()) for p in pre), 0.0), 1.0)
+    rule_g = B.CapacityRule(1.0, cf, delta, 0, w.T)
+    for q in range(world):
+        sel, sel_d, x_q, src_q, sh_q, st_q = pre[q]
+        devs = sharding.devices_of_rank(D, world, q)
+        B.locmoe_capacity(sh_q, st_q.idx, st_q.cos_sim, rule_g, st_q.delta_e, st_q.theta_e, st_q.cap_dev, st_q.ws)
+        cap_q = B.locmoe_capacity_read(st_q.cap_dev)
+        assert (cap_q.C_local, cap_q.C_expert, cap_q.delta, cap_q.ec_min) == (cap.C_local, cap.C_expert, cap.delta, cap.ec_min)
+        B.locmoe_route(sh_q, st_q.idx, src_q, st_q.cap_dev, Ca, st_q.pos, st_q.slot, st_q.drop, st_q.inv, st_q.counts,
+                       st_q.kept, st_q.send_counts, st_q.load, st_q.locality, st_q.status, st_q.ws)
+        B.locmoe_dispatch_peer(sh_q, Ca, x_q, st_q.inv, st_q.slot, bufs, devs.start, devs.stop, True)
+        torch.cuda.synchronize()
+        assert np.array_equal(st_q.slot.cpu().numpy(), ref.slot[sel])       # local routing = the global one, restricted
+        if q == 0 and world > 1:
+            # rows that belong to other ranks' source devices have not been touched yet
+            allb = torch.cat(bufs).float()
+            untouched = (allb == sentinel).all(dim=1).cpu().numpy()
+            src_of_row = _row_sources(rows, Ca, D, w.E // D, w.n_nodes, w.dev_per_node)
+            mine = (src_of_row >= devs.start) & (src_of_row < devs.stop)
+            assert np.array_equal(untouched, ~mine)
+        ranks.append((sel, sel_d, sh_q, st_q))
+
+    got = torch.cat(bufs)
+    assert np.array_equal(W.host_bits(got), want), "receive buffers differ from the oracle's"
+
+    # combine through peer loads: identity experts, so y = the receive buffers themselves
+    ydt = B.dtype_code(x.dtype)
+    g = oracle.gate(W.host_bits(x), sh_g.x_dtype, w.E)
+    for sel, sel_d, sh_q, st_q in ranks:
+        out = torch.empty(len(sel), w.H, dtype=x.dtype, device=dev)
+        B.locmoe_combine_peer(sh_q, Ca, bufs, ydt, st_q.slot, st_q.gate_w, out)
+        torch.cuda.synchronize()
+        R = np.where(g.idx[sel] == st_q.idx.cpu().numpy(), g.R[sel], st_q.gate_w.cpu().numpy().astype(np.float64))
+        ref_out = oracle.combine(want, sh_g.x_dtype, ref.slot[sel], R)
+        P._out_close(W.host_bits(out), ref_out, sh_g.x_dtype)
+
+
+def _row_sources(rows, C, D, Ed, N, Dn):
+    """Source device of every receive-layout row, from the layout's definition (written out independently)."""
+    r = np.arange(rows) // C
+    e, rho = r // D, r % D
+    a = e // Ed
+    return ((a // Dn + rho // Dn) % N) * Dn + (a % Dn + rho % Dn) % Dn
+
+
+def test_peer_calls_reject_bad_arguments(P):
+    B = P.B
+    dev = torch.device("cuda:0")
+    sh = B.make_shape(64, 64, 8, 2, 2, torch.float32, B.LAYOUT_SEND)
+    x = torch.zeros(64, 64, device=dev)
+    inv = torch.full((4 * 8 * 4,), -1, dtype=torch.int32, device=dev)
+    slot = torch.full((64,), -1, dtype=torch.int32, device=dev)
+    buf = torch.zeros(4 * 8 * 4, 64, device=dev)
+    with pytest.raises(B.LocMoEError):            # send-side layout
+        B.locmoe_dispatch_peer(sh, 4, x, inv, slot, [buf], 0, 4)
+    sh = B.make_shape(64, 64, 8, 2, 2, torch.float32, B.LAYOUT_RECV)
+    with pytest.raises(B.LocMoEError):            # three peers do not divide four devices
+        B.locmoe_dispatch_peer(sh, 4, x, inv, slot, [buf, buf, buf], 0, 4)
+    with pytest.raises(B.LocMoEError):            # source range outside the map
+        B.locmoe_dispatch_peer(sh, 4, x, inv, slot, [buf], 0, 5)

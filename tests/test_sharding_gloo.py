@@ -53,6 +53,15 @@ def _worker(rank, world, port, layout, q):
         # a rank only fills rows of its own source devices (SEND layout) -- disjoint row sets
         occupied = sharding.sum_over_ranks((part.inv >= 0).astype(np.int64))
         ok &= bool(occupied.max() <= 1) and int(occupied.sum()) == int((whole.inv >= 0).sum())
+        # capacity of the whole batch from per-rank minima: every rank gets the batch-wide delta and token count
+        import torch
+        de = torch.full((E,), 1.0)
+        de[rank] = 0.25 - 0.5 * rank                  # rank 1 holds a negative minimum: clamped to 0
+        de[5] = 0.125 + rank
+        delta, Tg = sharding.global_capacity_inputs(de, len(mine))
+        ok &= delta == 0.0 and Tg == T
+        delta2, _ = sharding.global_capacity_inputs(torch.full((E,), 0.5 + 0.25 * rank), 1)
+        ok &= delta2 == 0.5
         # timing helper: the slowest rank decides
         slow = sharding.max_over_ranks(10.0 + 5.0 * rank)
         thr = sharding.aggregate_throughput(1000, 4, 10.0 + 5.0 * rank, world)
