@@ -88,6 +88,12 @@ def lib():
         L.oracle_cos_hist.restype = C.c_int64
         L.oracle_cos_hist.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_int32,
                                       C.c_int32, C.c_double, C.c_double, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_gate_topk.restype = C.c_int
+        L.oracle_gate_topk.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
+                                       C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_combine_topk.restype = C.c_int
+        L.oracle_combine_topk.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                          C.c_void_p]
         _lib = L
     return _lib
 
@@ -308,3 +314,31 @@ def cos_hist(x, dtype, E, idx, e, j, nbins, lo=-1.0, hi=1.0):
     if n < 0:
         raise ValueError("oracle_cos_hist: bad argument")
     return n, he, hj, ce, cj
+
+
+def gate_topk(x, dtype, E, K, eps=None):
+    """(idx_k [K][T], R_k [K][T], gap [T]) of the top-k variant of the gate."""
+    x = _raw(x, dtype)
+    T, H = x.shape
+    idx_k = np.empty((K, T), np.int32)
+    R_k = np.empty((K, T), np.float64)
+    gap = np.empty(T, np.float64)
+    if eps is not None:
+        eps = np.ascontiguousarray(eps, dtype=np.float32)
+    rc = lib().oracle_gate_topk(_p(x), dtype, T, H, E, _p(eps), int(K), _p(idx_k), _p(R_k), _p(gap))
+    if rc != 0:
+        raise ValueError("oracle_gate_topk: error %d" % rc)
+    return idx_k, R_k, gap
+
+
+def combine_topk(y, y_dtype, slot_k, R_k) -> np.ndarray:
+    y = _raw(y, y_dtype)
+    H = y.shape[1]
+    slot_k = np.ascontiguousarray(slot_k, dtype=np.int32)
+    R_k = np.ascontiguousarray(R_k, dtype=np.float64)
+    K, T = slot_k.shape
+    out = np.empty((T, H), np.float64)
+    rc = lib().oracle_combine_topk(_p(y), y_dtype, T, H, K, _p(slot_k), _p(R_k), _p(out))
+    if rc != 0:
+        raise ValueError("oracle_combine_topk: error %d" % rc)
+    return out

@@ -30,6 +30,11 @@
  *   oracle_combine   y_m = R_m * expert_out (first equation of Sec. 3.2.1,
  *                    top-1 so a single term; a dropped token has no term).
  *
+ *   oracle_gate_topk, oracle_combine_topk
+ *                    the same gate and the same sum of Sec. 3.2.1's first
+ *                    equation with the k largest scores per token instead of
+ *                    one (a variant: the paper itself routes top-1).
+ *
  *   oracle_aux_loss  L_aux = alpha n sum_i f_i P_i (Sec. 3.2.2, first loss
  *                    equation), forward value.
  *   oracle_cos_hist  the two histograms of the second cosine-frequency figure of
@@ -537,4 +542,72 @@ int64_t oracle_cos_hist(const void *x, int dtype, int64_t T, int32_t H, int32_t 
         ++n;
     }
     return n;
+}
+
+/*
+ * Top-k variant of the gate (the paper routes every token to its single best expert; Sec. 2 describes top-k
+ * routers as the family it departs from).  Same logits as oracle_gate: G[i] = max(mean_i + eps_i, 0).  The K
+ * experts with the largest G are taken in descending order of G, a tie going to the lower index; the score of a
+ * chosen expert is its softmax value R = exp(G_i) / sum_k exp(G_k) (not renormalised over the chosen ones), so
+ * that y_m = sum over the chosen experts of R * expert(x) is the first equation of Sec. 3.2.1 restricted to them.
+ *   idx_k[j][t], R_k[j][t]  j-th choice of token t (j = 0 is oracle_gate's idx and R)
+ *   gap[t]                  smallest difference between consecutive logits among the K + 1 largest (how close the
+ *                           choice, or the order of the choices, is to a tie); +inf when E == K == 1
+ * Returns 0, or -2 on a bad argument.
+ */
+int oracle_gate_topk(const void *x, int dtype, int64_t T, int32_t H, int32_t E, const float *eps, int32_t K,
+                     int32_t *idx_k /* [K][T] */, double *R_k /* [K][T] */, double *gap /* [T] */)
+{
+    if (T < 0 || H <= 0 || E <= 0 || H % E != 0 || K < 1 || K > E) return -2;
+    const int32_t g = H / E;
+    double *G = (double *)malloc(sizeof(double) * (size_t)E);
+    char *taken = (char *)malloc((size_t)E);
+    if (!G || !taken) { free(G); free(taken); return -6; }
+    for (int64_t t = 0; t < T; ++t) {
+        for (int32_t i = 0; i < E; ++i) {
+            double s = 0.0;
+            for (int32_t j = 0; j < g; ++j) s += widen(x, dtype, t * H + (int64_t)i * g + j);
+            const double pre = s * ((double)E / (double)H) + (eps ? (double)eps[i] : 0.0);
+            G[i] = pre > 0.0 ? pre : 0.0;
+            taken[i] = 0;
+        }
+        double gmax = G[0];
+        for (int32_t i = 1; i < E; ++i) if (G[i] > gmax) gmax = G[i];
+        double denom = 0.0;
+        for (int32_t i = 0; i < E; ++i) denom += exp(G[i] - gmax);
+        double prev = 0.0, mingap = INFINITY;
+        for (int32_t j = 0; j <= K && j < E; ++j) {       /* one more than K: the best expert left out */
+            int32_t best = -1;
+            for (int32_t i = 0; i < E; ++i)
+                if (!taken[i] && (best < 0 || G[i] > G[best])) best = i;
+            taken[best] = 1;
+            if (j > 0 && prev - G[best] < mingap) mingap = prev - G[best];
+            prev = G[best];
+            if (j < K) {
+                idx_k[(int64_t)j * T + t] = best;
+                R_k[(int64_t)j * T + t] = exp(G[best] - gmax) / denom;
+            }
+        }
+        gap[t] = mingap;
+    }
+    free(G);
+    free(taken);
+    return 0;
+}
+
+/* Combine of the top-k variant: out[t][j] = sum over the K choices c of R_k[c][t] * y[slot_k[c][t]][j] (double);
+ * a dropped choice (slot < 0) has no term. */
+int oracle_combine_topk(const void *y, int y_dtype, int64_t T, int32_t H, int32_t K, const int32_t *slot_k /* [K][T] */,
+                        const double *R_k /* [K][T] */, double *out /* [T][H] */)
+{
+    for (int64_t t = 0; t < T; ++t)
+        for (int32_t j = 0; j < H; ++j) {
+            double v = 0.0;
+            for (int32_t c = 0; c < K; ++c) {
+                const int32_t sl = slot_k[(int64_t)c * T + t];
+                if (sl >= 0) v += R_k[(int64_t)c * T + t] * widen(y, y_dtype, (int64_t)sl * H + j);
+            }
+            out[t * H + j] = v;
+        }
+    return 0;
 }
