@@ -257,6 +257,38 @@ int locmoe_combine_peer(const locmoe_shape_t *shape, int32_t C_alloc, void *cons
                         void *out, void *stream);
 
 /*
+ * Top-k variant (the paper routes each token to its single best expert, Sec.
+ * 3.2.1; routers that keep the k best are the family it departs from, Sec. 2).
+ * The sum of Sec. 3.2.1's first equation then runs over the K chosen experts,
+ * each with its softmax score (not renormalised over the chosen ones).
+ *
+ * locmoe_topk_select: probs float[T][E], idx int32[T], gate_w float[T] as written
+ * by locmoe_gate.  Choice 0 of a token is idx / gate_w; choice c > 0 is the
+ * expert with the largest probability among those not yet chosen, a tie going
+ * to the lower index.  idx_k int32[K][T], w_k float[K][T]; 1 <= K <= min(8, E).
+ *
+ * Routing: run locmoe_capacity on the first choices with rule.T_global = K * T
+ * and locmoe_route with a shape whose T is K * T on the K * T "virtual tokens"
+ * v = c * T + t (idx_k as int32[K * T], src_dev repeated K times): all first
+ * choices come before all second choices in a queue.  Then
+ * locmoe_topk_fold (shape->T = T tokens, the same C_alloc) rewrites inv[row]
+ * from v to the token v mod T, after which locmoe_dispatch (slot = NULL) fills
+ * the buffer from x [T][H].
+ *
+ * locmoe_combine_topk: out[t][:] = sum over c < K of w_k[c][t] * y[slot_k[c][t]][:],
+ * a dropped choice (slot < 0) having no term, accumulated in fp32 in the order
+ * c = 0, 1, ... (first term a product, the others fused multiply-adds) and
+ * rounded once to shape->x_dtype.  slot_k int32[K][T] is the route stage's slot
+ * array of the K * T virtual tokens.  Rows must be multiples of 8 elements and
+ * the pointers 16-byte aligned.
+ */
+int locmoe_topk_select(const locmoe_shape_t *shape, const float *probs, const int32_t *idx,
+                       const float *gate_w, int32_t K, int32_t *idx_k, float *w_k, void *stream);
+int locmoe_topk_fold(const locmoe_shape_t *shape, int32_t C_alloc, int32_t *inv, void *stream);
+int locmoe_combine_topk(const locmoe_shape_t *shape, int32_t C_alloc, const void *y, int32_t y_dtype,
+                        int32_t K, const int32_t *slot_k, const float *w_k, void *out, void *stream);
+
+/*
  * Auxiliary load-balance loss, forward value (Sec. 3.2.2):
  *   L_aux = alpha * n * sum_i f_i * P_i,  f_i = load[i] / T (share of tokens whose
  *   arg-max is expert i),  P_i = (1/T) sum_t probs[t][i]  (the paper uses alpha = 0.01).

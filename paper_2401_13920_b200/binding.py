@@ -24,7 +24,7 @@ FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
     "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route",
-    "locmoe_dispatch", "locmoe_combine", "locmoe_dispatch_peer", "locmoe_combine_peer", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
+    "locmoe_dispatch", "locmoe_combine", "locmoe_dispatch_peer", "locmoe_combine_peer", "locmoe_topk_select", "locmoe_topk_fold", "locmoe_combine_topk", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
 
@@ -84,6 +84,9 @@ def _load() -> C.CDLL:
     lib.locmoe_cos_hist.argtypes = [C.POINTER(Shape), vp, vp, i32, i32, i32, C.c_float, C.c_float, vp, vp, vp, vp]
     lib.locmoe_dispatch_peer.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, C.POINTER(vp), i32, i32, i32, i32, vp]
     lib.locmoe_combine_peer.argtypes = [C.POINTER(Shape), i32, C.POINTER(vp), i32, i32, vp, vp, vp, vp]
+    lib.locmoe_topk_select.argtypes = [C.POINTER(Shape), vp, vp, vp, i32, vp, vp, vp]
+    lib.locmoe_topk_fold.argtypes = [C.POINTER(Shape), i32, vp, vp]
+    lib.locmoe_combine_topk.argtypes = [C.POINTER(Shape), i32, vp, i32, i32, vp, vp, vp, vp]
     lib.locmoe_launch_counts.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32 * 5)]
     lib.locmoe_device_flags.argtypes = [C.POINTER(C.c_int32), vp]
     lib.locmoe_status_string.argtypes = [C.c_int]
@@ -303,6 +306,32 @@ def locmoe_combine_peer(shape: Shape, C_alloc, peer_y, y_dtype, slot, gate_w, ou
                                                                   _ptr(gate_w), _ptr(out), _stream(stream)))
 
 
+def locmoe_topk_select(shape: Shape, probs, idx, gate_w, K, idx_k, w_k, stream=None) -> int:
+    _want(probs, torch.float32, shape.T * shape.E, "probs")
+    _want(idx, torch.int32, shape.T, "idx")
+    _want(gate_w, torch.float32, shape.T, "gate_w")
+    _want(idx_k, torch.int32, K * shape.T, "idx_k")
+    _want(w_k, torch.float32, K * shape.T, "w_k")
+    return _check("locmoe_topk_select", _lib.locmoe_topk_select(C.byref(shape), _ptr(probs), _ptr(idx), _ptr(gate_w), int(K),
+                                                                _ptr(idx_k), _ptr(w_k), _stream(stream)))
+
+
+def locmoe_topk_fold(shape: Shape, C_alloc, inv, stream=None) -> int:
+    _want(inv, torch.int32, shape.D * shape.E * C_alloc, "inv")
+    return _check("locmoe_topk_fold", _lib.locmoe_topk_fold(C.byref(shape), int(C_alloc), _ptr(inv), _stream(stream)))
+
+
+def locmoe_combine_topk(shape: Shape, C_alloc, y, K, slot_k, w_k, out, stream=None) -> int:
+    rows = shape.D * shape.E * C_alloc
+    dt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
+    _want(y, y.dtype, rows * shape.H, "y")
+    _want(slot_k, torch.int32, K * shape.T, "slot_k")
+    _want(w_k, torch.float32, K * shape.T, "w_k")
+    _want(out, dt, shape.T * shape.H, "out")
+    return _check("locmoe_combine_topk", _lib.locmoe_combine_topk(C.byref(shape), int(C_alloc), _ptr(y), dtype_code(y.dtype), int(K),
+                                                                  _ptr(slot_k), _ptr(w_k), _ptr(out), _stream(stream)))
+
+
 def locmoe_loc_loss(shape: Shape, counts, level, mu, smooth, dc_out, kl_out, group_tokens, loss_out, stream=None) -> int:
     G = shape.n_nodes if level else shape.D
     _want(counts, torch.int32, shape.D * shape.E, "counts")
@@ -417,6 +446,46 @@ def router_forward(st: RouterState, x, src_dev, y=None, eps=None, stream=None, o
     locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream, slot=st.slot)
     locmoe_combine(sh, Ca, st.buf if y is None else y, st.slot, st.gate_w, out, False, stream)
     return out
+
+
+def router_forward_topk(shape: Shape, x, src_dev, K: int, C_alloc: int, rule: CapacityRule, y=None, stream=None) -> dict:
+    """The top-k variant end to end on one stream (allocates its tensors: a convenience for tests and examples).
+
+    gate (with probabilities) -> capacity on the first choices, counting K * T assignments -> K best experts ->
+    route of the K * T virtual tokens -> fold -> dispatch -> combine over the K choices.  ``y`` are the expert outputs
+    in slot layout (identity experts when None).  Returns the tensors by name.
+    """
+    dev = x.device
+    T, H, E, D = shape.T, shape.H, shape.E, shape.D
+    i32 = dict(dtype=torch.int32, device=dev)
+    f32 = dict(dtype=torch.float32, device=dev)
+    xdt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
+    shape_v = Shape(K * T, H, E, shape.n_nodes, shape.dev_per_node, shape.x_dtype, shape.layout)
+    rows = D * E * C_alloc
+    r = dict(
+        idx=torch.empty(T, **i32), gate_w=torch.empty(T, **f32), cos_sim=torch.empty(T, **f32), probs=torch.empty(T, E, **f32),
+        delta_e=torch.empty(E, **f32), theta_e=torch.empty(E, **f32),
+        cap_dev=torch.zeros(CAPACITY_BYTES, dtype=torch.uint8, device=dev),
+        idx_k=torch.empty(K, T, **i32), w_k=torch.empty(K, T, **f32),
+        pos=torch.empty(K, T, **i32), slot=torch.empty(K, T, **i32), drop=torch.empty(K, T, dtype=torch.uint8, device=dev),
+        inv=torch.empty(rows, **i32), counts=torch.empty(D * E, **i32), kept=torch.empty(D * E, **i32),
+        send_counts=torch.empty(D * D, **i32), load=torch.empty(E, **i32),
+        locality=torch.empty(6, dtype=torch.int64, device=dev), status=torch.zeros(1, **i32),
+        ws=torch.empty(max(locmoe_workspace_bytes(shape_v, C_alloc), locmoe_workspace_bytes(shape, C_alloc)),
+                       dtype=torch.uint8, device=dev),
+        buf=torch.empty(rows, H, dtype=xdt, device=dev), out=torch.empty(T, H, dtype=xdt, device=dev),
+        src_k=src_dev.repeat(K).contiguous(),
+    )
+    rule_k = CapacityRule(rule.min_mult, rule.capacity_factor, rule.delta_override, rule.bound_form, K * T)
+    locmoe_gate(shape, x, None, r["idx"], r["gate_w"], r["cos_sim"], r["probs"], stream)
+    locmoe_capacity(shape, r["idx"], r["cos_sim"], rule_k, r["delta_e"], r["theta_e"], r["cap_dev"], r["ws"], stream)
+    locmoe_topk_select(shape, r["probs"], r["idx"], r["gate_w"], K, r["idx_k"], r["w_k"], stream)
+    locmoe_route(shape_v, r["idx_k"], r["src_k"], r["cap_dev"], C_alloc, r["pos"], r["slot"], r["drop"], r["inv"],
+                 r["counts"], r["kept"], r["send_counts"], r["load"], r["locality"], r["status"], r["ws"], stream)
+    locmoe_topk_fold(shape, C_alloc, r["inv"], stream)
+    locmoe_dispatch(shape, C_alloc, x, r["inv"], r["buf"], True, stream)
+    locmoe_combine_topk(shape, C_alloc, r["buf"] if y is None else y, K, r["slot"], r["w_k"], r["out"], stream)
+    return r
 
 
 class HostRouter:

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "liblocmoe.so")
-SOURCES = ["api.cu", "gate.cu", "capacity.cu", "capacity_noalloc.cu", "route.cu", "movers.cu", "ffn.cu", "aux_loss.cu", "loc_loss.cu", "cos_hist.cu", "peer.cu"]
+SOURCES = ["api.cu", "gate.cu", "capacity.cu", "capacity_noalloc.cu", "route.cu", "movers.cu", "ffn.cu", "aux_loss.cu", "loc_loss.cu", "cos_hist.cu", "peer.cu", "topk.cu"]
 
 
 def _nvcc() -> str:

@@ -229,6 +229,37 @@ int locmoe_combine_peer(const locmoe_shape_t* shape, int32_t C_alloc, void* cons
     return launch_combine_peer(*shape, rows, peer_y, n_peers, y_dtype, slot, gate_w, out, static_cast<cudaStream_t>(stream));
 }
 
+int locmoe_topk_select(const locmoe_shape_t* shape, const float* probs, const int32_t* idx, const float* gate_w, int32_t K,
+                       int32_t* idx_k, float* w_k, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!probs || !idx || !gate_w || !idx_k || !w_k) return LOCMOE_ERR_NULL;
+    if (K < 1 || K > 8 || K > shape->E) return LOCMOE_ERR_SHAPE;
+    return launch_topk_select(*shape, probs, idx, gate_w, K, idx_k, w_k, static_cast<cudaStream_t>(stream));
+}
+
+int locmoe_topk_fold(const locmoe_shape_t* shape, int32_t C_alloc, int32_t* inv, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!inv) return LOCMOE_ERR_NULL;
+    const long long rows = buffer_rows(shape, C_alloc);
+    if (rows < 0) return LOCMOE_ERR_SHAPE;
+    return launch_topk_fold(shape->T, rows, inv, static_cast<cudaStream_t>(stream));
+}
+
+int locmoe_combine_topk(const locmoe_shape_t* shape, int32_t C_alloc, const void* y, int32_t y_dtype, int32_t K,
+                        const int32_t* slot_k, const float* w_k, void* out, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!y || !slot_k || !w_k || !out) return LOCMOE_ERR_NULL;
+    if (y_dtype != LOCMOE_F32 && y_dtype != LOCMOE_BF16) return LOCMOE_ERR_DTYPE;
+    if (K < 1 || K > 8) return LOCMOE_ERR_SHAPE;
+    const long long rows = buffer_rows(shape, C_alloc);
+    if (rows < 0) return LOCMOE_ERR_SHAPE;
+    if (shape->H % 8 || (uintptr_t)y % 16 || (uintptr_t)out % 16) return LOCMOE_ERR_ALIGN;
+    return launch_combine_topk(*shape, rows, y, y_dtype, K, slot_k, w_k, out, static_cast<cudaStream_t>(stream));
+}
+
 int locmoe_expert_ffn(const locmoe_shape_t* shape, int32_t C_alloc, int32_t F, const void* buf, const void* w_in,
                       const void* w_out, void* h1, void* y, int32_t y_dtype, void* stream) {
     int rc = check_shape(shape);

@@ -70,6 +70,12 @@ int launch_dispatch_peer(const locmoe_shape_t& s, int C_alloc, int64_t rows, con
 int launch_combine_peer(const locmoe_shape_t& s, int64_t rows, void* const* peer_y, int n_peers, int y_dtype,
                         const int32_t* slot, const float* gate_w, void* out, cudaStream_t st);
 
+int launch_topk_select(const locmoe_shape_t& s, const float* probs, const int32_t* idx, const float* gate_w, int K,
+                       int32_t* idx_k, float* w_k, cudaStream_t st);
+int launch_topk_fold(int T, long long rows, int32_t* inv, cudaStream_t st);
+int launch_combine_topk(const locmoe_shape_t& s, int64_t rows, const void* y, int y_dtype, int K, const int32_t* slot_k,
+                        const float* w_k, void* out, cudaStream_t st);
+
 int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* buf, const void* w_in,
                       const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st);
 int read_ffn_flags(int* out, cudaStream_t st);

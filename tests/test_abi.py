@@ -68,6 +68,9 @@ def test_null_pointers_are_rejected_before_any_launch(B):
     assert lib.locmoe_dispatch(C.byref(sh), 4, None, None, None, None, 1, None) == -1
     assert lib.locmoe_combine(C.byref(sh), 4, None, 0, None, None, None, 0, None) == -1
     assert lib.locmoe_loc_loss(C.byref(sh), None, 0, 1.0, 1e-3, None, None, None, None, None) == -1
+    assert lib.locmoe_topk_select(C.byref(sh), None, None, None, 2, None, None, None) == -1
+    assert lib.locmoe_topk_fold(C.byref(sh), 4, None, None) == -1
+    assert lib.locmoe_combine_topk(C.byref(sh), 4, None, 0, 2, None, None, None, None) == -1
     assert lib.locmoe_dispatch_peer(C.byref(sh), 4, None, None, None, None, 1, 0, 1, 1, None) == -1
     assert lib.locmoe_combine_peer(C.byref(sh), 4, None, 1, 0, None, None, None, None) == -1
     assert lib.locmoe_cos_hist(C.byref(sh), None, None, 0, 1, 8, -1.0, 1.0, None, None, None, None) == -1
