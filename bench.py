@@ -439,7 +439,7 @@ def main():
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
 # profiles/dram_traffic_config2.md, taken at the bench's full size.
 NCU_TRAFFIC = {
-    (2, 1.0): {"gate": 671118080 + 3236352, "dispatch": 605918208 + 615610624, "combine": 606182656 + 618102272},
+    (2, 1.0): {"gate": 671117568 + 3323136, "dispatch": 606188288 + 612412416, "combine": 606180864 + 610791680},
 }
 
 
