@@ -43,6 +43,7 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=12)
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     ap.add_argument("--event-every", type=int, default=8, help="carry per-stage CUDA events on every n-th timed step")
+    ap.add_argument("--unfused", action="store_true", help="capacity and route as two calls instead of locmoe_capacity_route")
     ap.add_argument("--no-ffn", action="store_true", help="config 5 only: identity experts instead of the expert FFN")
     ap.add_argument("--ffn-inner", type=int, default=10240, help="config 5: inner size F of the expert FFN")
     ap.add_argument("--tokens", type=int, default=0, help="override T (profiling-sized case; not the metric's workload)")
@@ -252,7 +253,9 @@ def main():
     ysrc = st.buf if y is None else y
 
     stream = torch.cuda.current_stream()
-    stages = ["gate", "capacity", "route", "dispatch"] + (["ffn"] if use_ffn else []) + ["combine"]
+    fused = not args.unfused
+    stages = ["gate"] + (["capacity_route"] if fused else ["capacity", "route"]) + ["dispatch"] + \
+             (["ffn"] if use_ffn else []) + ["combine"]
 
     def step(ev=None):
         sh, Ca = st.shape, st.C_alloc
@@ -265,10 +268,15 @@ def main():
         mark()
         B.locmoe_gate(sh, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
         mark()
-        B.locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
-        mark()
-        B.locmoe_route(sh, st.idx, src, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
-                       st.send_counts, st.load, st.locality, st.status, st.ws, stream)
+        if fused:
+            B.locmoe_capacity_route(sh, st.idx, st.cos_sim, src, st.rule, st.delta_e, st.theta_e, st.cap_dev, Ca, st.pos,
+                                    st.slot, st.drop, st.inv, st.counts, st.kept, st.send_counts, st.load, st.locality,
+                                    st.status, st.ws, stream)
+        else:
+            B.locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
+            mark()
+            B.locmoe_route(sh, st.idx, src, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
+                           st.send_counts, st.load, st.locality, st.status, st.ws, stream)
         mark()
         B.locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream, slot=st.slot)
         mark()
@@ -361,6 +369,11 @@ def main():
                          "hbm_kernels": kernels})
 
     launches = B.locmoe_launch_counts(shape)
+    if fused:
+        # the capacity stage rides on the route stage's launches (up to 8192 experts)
+        cr = launches.pop("route") + (launches["capacity"] if shape.E > 8192 else 0)
+        launches.pop("capacity")
+        launches = {"gate": launches["gate"], "capacity_route": cr, "dispatch": launches["dispatch"], "combine": launches["combine"]}
     if use_ffn:
         launches["ffn"] = 2
     launches_per_step = sum(launches.values())

@@ -197,6 +197,22 @@ int locmoe_route(const locmoe_shape_t *shape, const int32_t *idx, const int32_t 
                  int64_t *locality, int32_t *status, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * locmoe_capacity followed by locmoe_route as ONE call with the same inputs,
+ * outputs and results (Sec. 3.2.3): the per-expert minima of the cosines are
+ * taken by the route stage's first pass over the tokens and the closed forms
+ * are evaluated beside its first sorting pass, so the capacity stage costs no
+ * launch and no pass of its own; the last sorting pass reads the record from
+ * cap_dev.  Beyond 8192 experts the two stages simply run one after the other.
+ * ws: at least locmoe_workspace_bytes() bytes.
+ */
+int locmoe_capacity_route(const locmoe_shape_t *shape, const int32_t *idx, const float *cos_sim,
+                          const int32_t *src_dev, const locmoe_capacity_rule_t *rule,
+                          float *delta_e, float *theta_e, locmoe_capacity_t *cap_dev, int32_t C_alloc,
+                          int32_t *pos, int32_t *slot, uint8_t *drop, int32_t *inv, int32_t *counts,
+                          int32_t *kept, int32_t *send_counts, int32_t *load, int64_t *locality,
+                          int32_t *status, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Dispatch: buf[row][:] = x[inv[row]][:] bit for bit for occupied rows; rows
  * with inv < 0 are zero-filled when zero_pad != 0 and left untouched otherwise.
  * x [T][H], buf [D * E * C_alloc][H], both of shape->x_dtype.

@@ -23,7 +23,7 @@ WARN_CLAMPED, WARN_BAD_SRC, WARN_BAD_IDX = 1, 2, 4
 FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
-    "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route",
+    "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route", "locmoe_capacity_route",
     "locmoe_dispatch", "locmoe_combine", "locmoe_dispatch_peer", "locmoe_combine_peer", "locmoe_topk_select", "locmoe_topk_fold", "locmoe_combine_topk", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
@@ -74,6 +74,8 @@ def _load() -> C.CDLL:
     lib.locmoe_capacity_noalloc.argtypes = [C.POINTER(Shape), vp, vp, C.POINTER(CapacityRule), vp, vp, vp, vp]
     lib.locmoe_capacity_read.argtypes = [vp, C.POINTER(Capacity), vp]
     lib.locmoe_route.argtypes = [C.POINTER(Shape), vp, vp, vp, i32] + [vp] * 10 + [vp, C.c_size_t, vp]
+    lib.locmoe_capacity_route.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(CapacityRule), vp, vp, vp, i32] + [vp] * 10 + \
+                                         [vp, C.c_size_t, vp]
     lib.locmoe_dispatch.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, vp, i32, vp]
     lib.locmoe_combine.argtypes = [C.POINTER(Shape), i32, vp, i32, vp, vp, vp, i32, vp]
     lib.locmoe_expert_ffn.argtypes = [C.POINTER(Shape), i32, i32, vp, vp, vp, vp, vp, i32, vp]
@@ -230,6 +232,23 @@ def locmoe_route(shape: Shape, idx, src_dev, cap_dev, C_alloc, pos, slot, drop, 
         C.byref(shape), _ptr(idx), _ptr(src_dev), _ptr(cap_dev), int(C_alloc), _ptr(pos), _ptr(slot), _ptr(drop),
         _ptr(inv), _ptr(counts), _ptr(kept), _ptr(send_counts), _ptr(load), _ptr(locality), _ptr(status),
         _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def locmoe_capacity_route(shape: Shape, idx, cos_sim, src_dev, rule: CapacityRule, delta_e, theta_e, cap_dev, C_alloc, pos, slot,
+                          drop, inv, counts, kept, send_counts, load, locality, status, ws, stream=None) -> int:
+    D, E, T = shape.D, shape.E, shape.T
+    for t, dt, n, name in ((idx, torch.int32, T, "idx"), (cos_sim, torch.float32, T, "cos_sim"), (src_dev, torch.int32, T, "src_dev"),
+                           (delta_e, torch.float32, E, "delta_e"), (theta_e, torch.float32, E, "theta_e"),
+                           (cap_dev, torch.uint8, CAPACITY_BYTES, "cap_dev"), (pos, torch.int32, T, "pos"),
+                           (slot, torch.int32, T, "slot"), (drop, torch.uint8, T, "drop"), (inv, torch.int32, D * E * C_alloc, "inv"),
+                           (counts, torch.int32, D * E, "counts"), (kept, torch.int32, D * E, "kept"),
+                           (send_counts, torch.int32, D * D, "send_counts"), (load, torch.int32, E, "load"),
+                           (locality, torch.int64, 6, "locality"), (status, torch.int32, 1, "status")):
+        _want(t, dt, n, name)
+    return _check("locmoe_capacity_route", _lib.locmoe_capacity_route(
+        C.byref(shape), _ptr(idx), _ptr(cos_sim), _ptr(src_dev), C.byref(rule), _ptr(delta_e), _ptr(theta_e), _ptr(cap_dev),
+        int(C_alloc), _ptr(pos), _ptr(slot), _ptr(drop), _ptr(inv), _ptr(counts), _ptr(kept), _ptr(send_counts), _ptr(load),
+        _ptr(locality), _ptr(status), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def locmoe_dispatch(shape: Shape, C_alloc, x, inv, buf, zero_pad=True, stream=None, slot=None) -> int:
@@ -430,19 +449,26 @@ def make_router(shape: Shape, C_alloc: int, rule: CapacityRule, device="cuda") -
     )
 
 
-def router_forward(st: RouterState, x, src_dev, y=None, eps=None, stream=None, out=None):
+def router_forward(st: RouterState, x, src_dev, y=None, eps=None, stream=None, out=None, fused=True):
     """gate -> capacity -> route -> dispatch -> combine on one stream.
 
     ``y`` are the expert outputs in slot layout; with ``y=None`` the experts are
-    the identity and the dispatched buffer itself is combined.  Returns the
-    combined output (``st.out`` unless ``out`` is given).
+    the identity and the dispatched buffer itself is combined.  ``fused`` runs the
+    capacity and route stages as the single call ``locmoe_capacity_route`` (same
+    results, one stage less in the launch chain).  Returns the combined output
+    (``st.out`` unless ``out`` is given).
     """
     sh, Ca = st.shape, st.C_alloc
     out = st.out if out is None else out
     locmoe_gate(sh, x, eps, st.idx, st.gate_w, st.cos_sim, None, stream)
-    locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
-    locmoe_route(sh, st.idx, src_dev, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
-                 st.send_counts, st.load, st.locality, st.status, st.ws, stream)
+    if fused:
+        locmoe_capacity_route(sh, st.idx, st.cos_sim, src_dev, st.rule, st.delta_e, st.theta_e, st.cap_dev, Ca, st.pos,
+                              st.slot, st.drop, st.inv, st.counts, st.kept, st.send_counts, st.load, st.locality,
+                              st.status, st.ws, stream)
+    else:
+        locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
+        locmoe_route(sh, st.idx, src_dev, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,
+                     st.send_counts, st.load, st.locality, st.status, st.ws, stream)
     locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream, slot=st.slot)
     locmoe_combine(sh, Ca, st.buf if y is None else y, st.slot, st.gate_w, out, False, stream)
     return out

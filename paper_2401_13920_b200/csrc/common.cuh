@@ -37,7 +37,7 @@ struct RoutePlan {
     int hstride;      // row stride of the histogram matrices: ntiles rounded up to a multiple of 4
     int launches;     // kernel launches of one route call
     int prescan;      // 1: histogram matrices are prefix-scanned by a launch of their own (large batches)
-    size_t off_keys[2], off_toks[2], off_hist[4], off_keystart, off_rowbase, off_rowtot, total;
+    size_t off_keys[2], off_toks[2], off_hist[4], off_keystart, off_rowbase, off_rowtot, off_cap_part, total;
 };
 int plan_route(const locmoe_shape_t& s, RoutePlan* p);
 size_t capacity_ws_bytes(const locmoe_shape_t& s);
@@ -47,6 +47,13 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
                  int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
                  int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
                  void* ws, cudaStream_t st);
+
+bool capacity_route_fusable(const locmoe_shape_t& s);
+int launch_capacity_route(const locmoe_shape_t& s, const int32_t* idx, const float* cos_sim, const int32_t* src,
+                          const locmoe_capacity_rule_t& rule, float* delta_e, float* theta_e, locmoe_capacity_t* cap_dev,
+                          int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
+                          int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
+                          void* ws, cudaStream_t st);
 
 int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const int32_t* inv, const int32_t* slot,
                     void* buf, int zero_pad, cudaStream_t st);

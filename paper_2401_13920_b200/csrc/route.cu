@@ -20,6 +20,7 @@
 //             of their own before the only scatter when P = 1.
 #include <stdlib.h>
 
+#include "capacity_finish.cuh"
 #include "common.cuh"
 
 namespace locmoe {
@@ -52,6 +53,16 @@ struct RouteArgs {
     int hstride, tile_shift;    // row stride of the histogram matrices (a multiple of 4 >= ntiles); log2(tile)
     int32_t* rowtot;            // [256] per-digit totals of the pass being scattered (prescan mode)
     int prescan;                // 1: a prescan launch turned hist[p] into exclusive prefixes along the tiles
+    // capacity carried along (the fused call): hist0 also takes the per-expert minima of the cosines per tile,
+    // an extra CTA of the first scatter combines them and writes the capacity record the last scatter reads
+    int fuse_cap, H;
+    double lnbeta;              // ln B(1/2, (H-1)/2), from the host
+    const float* cos;
+    uint32_t* cap_part;         // [ntiles][E] order-preserving codes
+    locmoe_capacity_rule_t rule;
+    float* delta_e;
+    float* theta_e;
+    locmoe_capacity_t* cap_out;
 };
 
 __device__ __forceinline__ int dest_rank(int a, int b, int N, int Dn) {
@@ -90,7 +101,10 @@ __global__ void __launch_bounds__(kThreads) route_hist0_kernel(const RouteArgs a
     pdl_trigger();
     extern __shared__ int sh[];
     const int nbins = 1 << a.bits[0];
+    uint32_t* smin = reinterpret_cast<uint32_t*>(sh + nbins);   // [E] minima of this tile (fused capacity only)
     for (int d = threadIdx.x; d < nbins; d += blockDim.x) sh[d] = 0;
+    if (a.fuse_cap)
+        for (int e = threadIdx.x; e < a.E; e += blockDim.x) smin[e] = 0xffffffffu;
     __syncthreads();
     const int base = blockIdx.x * a.tile;
     const uint32_t mask = (uint32_t)nbins - 1u;
@@ -98,17 +112,22 @@ __global__ void __launch_bounds__(kThreads) route_hist0_kernel(const RouteArgs a
     constexpr int kU = 4;   // tokens in flight per thread
     for (int o0 = threadIdx.x; o0 < a.tile; o0 += kU * kThreads) {
         int e[kU], sd[kU];
+        float cv[kU];
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
             const int o = o0 + u * kThreads, t = base + o;
-            e[u] = 0; sd[u] = 0;
-            if (o < a.tile && t < a.T) { e[u] = a.idx[t]; sd[u] = a.src[t]; }
+            e[u] = 0; sd[u] = 0; cv[u] = 0.0f;
+            if (o < a.tile && t < a.T) {
+                e[u] = a.idx[t]; sd[u] = a.src[t];
+                if (a.fuse_cap) cv[u] = a.cos[t];
+            }
         }
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
             const int o = o0 + u * kThreads, t = base + o;
             if (o >= a.tile || t >= a.T) continue;
             const bool bad_s = (unsigned)sd[u] >= (unsigned)a.D, bad_e = (unsigned)e[u] >= (unsigned)a.E;
+            if (a.fuse_cap && !bad_e) atomicMin(&smin[e[u]], order_code(cv[u]));
             if (bad_s || bad_e) {
                 warn |= bad_s ? LOCMOE_WARN_BAD_SRC : LOCMOE_WARN_BAD_IDX;
                 a.pos[t] = -1; a.slot[t] = -1; a.drop[t] = 1;
@@ -122,6 +141,8 @@ __global__ void __launch_bounds__(kThreads) route_hist0_kernel(const RouteArgs a
     if (warn) atomicOr(a.status, warn);
     __syncthreads();
     for (int d = threadIdx.x; d < nbins; d += blockDim.x) a.hist[0][(size_t)d * a.hstride + blockIdx.x] = sh[d];
+    if (a.fuse_cap)
+        for (int e = threadIdx.x; e < a.E; e += blockDim.x) a.cap_part[(size_t)blockIdx.x * a.E + e] = smin[e];
 }
 
 // Exclusive scan of in[0..n) into out[0..n) by one CTA of kThreads threads (in == out allowed).  Every warp owns a
@@ -161,23 +182,57 @@ __device__ void block_exclusive_scan(const int32_t* in, int32_t* out, int n) {
     __syncthreads();
 }
 
-// Extra CTAs (index x = 0, 1, ... of nx): x = 0 builds the key-class starts, the others the count matrices.
-__device__ void route_extras(const RouteArgs& a, int x, int nx) {
+// Extra CTAs of the first scatter (index x = 0, 1, ... of nx), none of which needs the capacity: x = 0 builds the
+// key-class starts, the next ones the first buffer row of every class; in the fused call the last one combines the
+// per-tile minima and evaluates the capacity rule (dyn = the CTA's dynamic shared memory, at least E words).
+__device__ void route_extras_a(const RouteArgs& a, int x, int nx, int* dyn) {
     if (x == 0) {
         block_exclusive_scan(a.counts, a.keystart, a.K);
         return;
     }
+    if (a.fuse_cap && x == nx - 1) {
+        __shared__ FinishShared fs;
+        uint32_t* comb = reinterpret_cast<uint32_t*>(dyn);
+        for (int e = threadIdx.x; e < a.E; e += kThreads) comb[e] = 0xffffffffu;
+        __syncthreads();
+        constexpr int kWorkers = kThreads, kU = 8;
+        {
+            const long long n = (long long)a.ntiles * a.E;
+            for (long long i0 = threadIdx.x; i0 < n; i0 += (long long)kU * kWorkers) {
+                uint32_t c[kU];
+#pragma unroll
+                for (int u = 0; u < kU; ++u) {
+                    const long long i = i0 + (long long)u * kWorkers;
+                    c[u] = i < n ? __ldcg(a.cap_part + i) : 0xffffffffu;
+                }
+#pragma unroll
+                for (int u = 0; u < kU; ++u) {
+                    const long long i = i0 + (long long)u * kWorkers;
+                    if (c[u] != 0xffffffffu) atomicMin(&comb[(int)(i % a.E)], c[u]);
+                }
+            }
+        }
+        __syncthreads();
+        capacity_finish<false>(fs, comb, 1, a.T, a.E, a.H, a.D, a.lnbeta, a.rule, a.delta_e, a.theta_e, a.cap_out);
+        return;
+    }
+    const int nrb = nx - 1 - (a.fuse_cap ? 1 : 0);
+    for (int k = (x - 1) * kThreads + threadIdx.x; k < a.K; k += nrb * kThreads)
+        a.rowbase[k] = (int)(route_row_base(a, k) * a.C_alloc);
+}
+
+// Extra CTAs of the last scatter: the count matrices, which need the capacity.
+__device__ void route_extras_b(const RouteArgs& a, int x, int nx) {
     int C = a.cap->C_local;
     if (C > a.C_alloc) {
         C = a.C_alloc;
-        if (x == 1 && threadIdx.x == 0) atomicOr(a.status, LOCMOE_WARN_CLAMPED);
+        if (x == 0 && threadIdx.x == 0) atomicOr(a.status, LOCMOE_WARN_CLAMPED);
     }
     unsigned long long raw0 = 0, raw1 = 0, raw2 = 0, kp0 = 0, kp1 = 0, kp2 = 0;
-    for (int k = (x - 1) * kThreads + threadIdx.x; k < a.K; k += (nx - 1) * kThreads) {
+    for (int k = x * kThreads + threadIdx.x; k < a.K; k += nx * kThreads) {
         const int c = a.counts[k];
         const int kp = c < C ? c : C;
         a.kept[k] = kp;
-        a.rowbase[k] = (int)(route_row_base(a, k) * a.C_alloc);
         if (c == 0) continue;
         const int s = k / a.E, e = k - s * a.E, b = e / a.Ed;
         if (b == s) { raw0 += c; kp0 += kp; }
@@ -202,10 +257,12 @@ __device__ void route_extras(const RouteArgs& a, int x, int nx) {
     }
 }
 
+// Single-pass sorts have no first scatter to ride on: the capacity-free extras get a launch of their own.
 __global__ void __launch_bounds__(kThreads) route_extras_kernel(const RouteArgs a) {
     pdl_wait();
     pdl_trigger();
-    route_extras(a, blockIdx.x, gridDim.x);
+    extern __shared__ int dyn[];
+    route_extras_a(a, blockIdx.x, gridDim.x, dyn);
 }
 
 // Large batches only: turns every digit row of hist[pass] into its exclusive prefix along the tiles (in place)
@@ -240,11 +297,12 @@ template <bool FIRST, bool LAST, int R>
 __global__ void __launch_bounds__(kThreads) route_scatter_kernel(const RouteArgs a, int pass, int shift) {
     pdl_wait();
     pdl_trigger();
+    extern __shared__ int sm[];
     if ((int)blockIdx.x >= a.ntiles) {
-        route_extras(a, blockIdx.x - a.ntiles, gridDim.x - a.ntiles);
+        if (LAST) route_extras_b(a, blockIdx.x - a.ntiles, gridDim.x - a.ntiles);
+        else route_extras_a(a, blockIdx.x - a.ntiles, gridDim.x - a.ntiles, sm);
         return;
     }
-    extern __shared__ int sm[];
     const int nbins = 1 << a.bits[pass];
     int* cnt = sm;                       // [kWarps][nbins] per-warp digit counters, then running offsets
     int* pre = sm + kWarps * nbins;      // [nbins] tokens of the digit in earlier tiles
@@ -474,6 +532,7 @@ int plan_route(const locmoe_shape_t& s, RoutePlan* p) {
     p->off_keystart = off; off += align256((size_t)K * 4);
     p->off_rowbase = off; off += align256((size_t)K * 4);
     p->off_rowtot = off; off += 1024;
+    p->off_cap_part = off; off += align256((size_t)p->ntiles * s.E * 4);
     p->total = off;
     p->prescan = ((long long)p->ntiles << p->bits[0]) > 32768 ? 1 : 0;
     {   // testing aid: LOCMOE_PATH=grid forces the large-batch variants at any size
@@ -484,10 +543,19 @@ int plan_route(const locmoe_shape_t& s, RoutePlan* p) {
     return LOCMOE_OK;
 }
 
-int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src, const locmoe_capacity_t* cap_dev,
-                 int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
-                 int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
-                 void* ws, cudaStream_t st) {
+// The route stage; with `fuse` != nullptr also the capacity stage (its minima ride on hist0, its finish on an extra
+// CTA of the first scatter), writing the record to cap_dev before the last scatter reads it.
+struct FusedCapacity {
+    const float* cos_sim;
+    locmoe_capacity_rule_t rule;
+    float* delta_e;
+    float* theta_e;
+};
+
+static int launch_route_impl(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src, locmoe_capacity_t* cap_dev,
+                             const FusedCapacity* fuse, int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop,
+                             int32_t* inv, int32_t* counts, int32_t* kept, int32_t* send_counts, int32_t* load,
+                             int64_t* locality, int32_t* status, void* ws, cudaStream_t st) {
     RoutePlan p;
     int rc = plan_route(s, &p);
     if (rc) return rc;
@@ -517,6 +585,15 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
     while ((1 << a.tile_shift) < p.tile) ++a.tile_shift;
     a.rowtot = reinterpret_cast<int32_t*>(w + p.off_rowtot);
     a.prescan = p.prescan;
+    a.fuse_cap = fuse ? 1 : 0;
+    a.H = s.H;
+    if (fuse) {
+        a.cos = fuse->cos_sim; a.rule = fuse->rule; a.delta_e = fuse->delta_e; a.theta_e = fuse->theta_e;
+        a.cap_out = cap_dev;
+        a.lnbeta = ln_beta_half(s.H);
+        a.cap_part = reinterpret_cast<uint32_t*>(w + p.off_cap_part);
+    }
+    const size_t cap_smem = fuse ? (size_t)s.E * sizeof(uint32_t) : 0;
 
     long long init_items = a.rows > a.K ? a.rows : a.K;
     int init_blocks = (int)((init_items + kThreads * 4 - 1) / (kThreads * 4));
@@ -524,13 +601,14 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
     if (init_blocks < 1) init_blocks = 1;
     if ((rc = launch_pdl(route_init_kernel, init_blocks, kThreads, 0, st, a))) return rc;
 
-    if ((rc = launch_pdl(route_hist0_kernel, p.ntiles, kThreads, sizeof(int) << p.bits[0], st, a))) return rc;
+    if ((rc = launch_pdl(route_hist0_kernel, p.ntiles, kThreads, (sizeof(int) << p.bits[0]) + cap_smem, st, a))) return rc;
 
-    int extras = 1 + (a.K + kThreads * 4 - 1) / (kThreads * 4);
-    if (extras > 33) extras = 33;
-    if (extras < 2) extras = 2;
+    int per_key = (a.K + kThreads * 4 - 1) / (kThreads * 4);   // CTAs that walk the K key classes
+    if (per_key > 32) per_key = 32;
+    if (per_key < 1) per_key = 1;
+    const int extras_a = 1 + per_key + (fuse ? 1 : 0), extras_b = per_key;
     if (p.passes == 1) {
-        if ((rc = launch_pdl(route_extras_kernel, extras, kThreads, 0, st, a))) return rc;
+        if ((rc = launch_pdl(route_extras_kernel, extras_a, kThreads, cap_smem, st, a))) return rc;
     }
     int shift = 0;
     for (int pass = 0; pass < p.passes; ++pass) {
@@ -538,13 +616,40 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
         if (p.prescan) {
             if ((rc = launch_pdl(route_prescan_kernel, ((1 << p.bits[pass]) + kWarps - 1) / kWarps, kThreads, 0, st, a, pass))) return rc;
         }
-        const size_t smb = ((size_t)(kWarps + 2) * sizeof(int)) << p.bits[pass];
-        const int grid = p.ntiles + ((first && !last) ? extras : 0);
+        size_t smb = ((size_t)(kWarps + 2) * sizeof(int)) << p.bits[pass];
+        if (first && !last && cap_smem > smb) smb = cap_smem;
+        const int grid = p.ntiles + (last ? extras_b : (first ? extras_a : 0));
         rc = launch_scatter(p.rounds, first, last, grid, smb, st, a, pass, shift);
         if (rc) return rc;
         shift += p.bits[pass];
     }
     return LOCMOE_OK;
+}
+
+int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src, const locmoe_capacity_t* cap_dev,
+                 int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
+                 int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
+                 void* ws, cudaStream_t st) {
+    return launch_route_impl(s, idx, src, const_cast<locmoe_capacity_t*>(cap_dev), nullptr, C_alloc, pos, slot, drop, inv,
+                             counts, kept, send_counts, load, locality, status, ws, st);
+}
+
+bool capacity_route_fusable(const locmoe_shape_t& s) { return s.E <= 8192; }
+
+int launch_capacity_route(const locmoe_shape_t& s, const int32_t* idx, const float* cos_sim, const int32_t* src,
+                          const locmoe_capacity_rule_t& rule, float* delta_e, float* theta_e, locmoe_capacity_t* cap_dev,
+                          int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
+                          int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
+                          void* ws, cudaStream_t st) {
+    if (!capacity_route_fusable(s)) {
+        int rc = launch_capacity(s, idx, cos_sim, rule, delta_e, theta_e, cap_dev, ws, st);
+        if (rc) return rc;
+        return launch_route(s, idx, src, cap_dev, C_alloc, pos, slot, drop, inv, counts, kept, send_counts, load, locality,
+                            status, ws, st);
+    }
+    const FusedCapacity f{cos_sim, rule, delta_e, theta_e};
+    return launch_route_impl(s, idx, src, cap_dev, &f, C_alloc, pos, slot, drop, inv, counts, kept, send_counts, load,
+                             locality, status, ws, st);
 }
 
 }  // namespace locmoe

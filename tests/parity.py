@@ -165,7 +165,8 @@ def check_combine_sampled(y, shape, st, ref_route, gate_info, tokens_sample):
 
 
 def run_staged(w: W.Workload, capacity_factor=1.0, min_mult=None, layout=B.LAYOUT_SEND, delta_override=-1.0,
-               bound_form=B.BOUND_BETA, C_alloc=None, full=True, n_sample=512, y_random=False, eps=None, seed=0):
+               bound_form=B.BOUND_BETA, C_alloc=None, full=True, n_sample=512, y_random=False, eps=None, seed=0,
+               fused=True):
     """Runs the five calls on the workload and compares every stage; returns a small report."""
     dev = torch.device("cuda:0")
     x = W.make_tokens(w, dev)
@@ -179,7 +180,7 @@ def run_staged(w: W.Workload, capacity_factor=1.0, min_mult=None, layout=B.LAYOU
     y = None
     if y_random:
         y = W.make_expert_out(w, st.rows, dev, "f32" if w.y_dtype == "f32" else w.dtype)
-    B.router_forward(st, x, src, y=y, eps=eps_dev)
+    B.router_forward(st, x, src, y=y, eps=eps_dev, fused=fused)
     torch.cuda.synchronize()
     assert B.locmoe_device_flags() == 0, "a kernel reported a failed bounded wait"
 

@@ -77,3 +77,5 @@ def test_null_pointers_are_rejected_before_any_launch(B):
     rule = B.CapacityRule(1.0, 1.0, -1.0, 0, 0)
     assert lib.locmoe_capacity(C.byref(sh), None, None, C.byref(rule), None, None, None, None, 0, None) == -1
     assert lib.locmoe_route(C.byref(sh), None, None, None, 4, *([None] * 10), None, 0, None) == -1
+    assert lib.locmoe_capacity_route(C.byref(sh), None, None, None, C.byref(rule), None, None, None, 4, *([None] * 10),
+                                     None, 0, None) == -1

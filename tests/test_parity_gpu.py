@@ -114,6 +114,33 @@ def test_warp_per_row_dispatch_variant(P, monkeypatch):
     P.run_staged(P.W.CONFIGS[1], 1.0, layout=1, full=True)
 
 
+# ---- capacity and route as two separate calls (the default path runs them as the one fused call) ----
+
+@pytest.mark.parametrize("cfg,T", [(1, 4096), (2, 6000), (3, 8229), (4, 5003), (5, 7001)])
+def test_separate_capacity_and_route_calls(P, cfg, T):
+    rep = P.run_staged(P.W.CONFIGS[cfg].scaled(T), 1.0, full=True, y_random=cfg == 4, fused=False)
+    assert rep["status"] == 0
+
+
+@pytest.mark.parametrize("kw", [
+    dict(T=1, H=64, E=4, n_nodes=1, dev_per_node=2),
+    dict(T=31, H=64, E=1, n_nodes=1, dev_per_node=1),
+    dict(T=513, H=1024, E=512, n_nodes=4, dev_per_node=8),
+    dict(T=4097, H=2048, E=2048, n_nodes=8, dev_per_node=8),
+])
+def test_separate_calls_shapes(P, kw):
+    P.run_staged(_wl(P, **kw), 1.0, layout=1, full=True, fused=False)
+
+
+def test_separate_calls_grid_path(P, grid_path):
+    P.run_staged(P.W.CONFIGS[2].scaled(70001), 1.0, full=True, fused=False)
+
+
+def test_separate_calls_full_size_config2(P):
+    rep = P.run_staged(P.W.CONFIGS[2], 1.0, full=False, n_sample=512, fused=False)
+    assert rep["C_local"] == 16
+
+
 # ---- edge cases and degenerate inputs ----
 
 @pytest.mark.parametrize("kw", [
