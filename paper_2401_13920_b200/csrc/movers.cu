@@ -1,11 +1,12 @@
 // Dispatch (row gather into the All-to-All shaped buffer) and gate-weighted
 // combine (first equation of Sec. 3.2.1, top-1: y_m = R_m * expert output).
 //
-// Both are row movers: one warp owns one destination row, reads the whole
-// source row with 16-byte streaming loads and writes the destination row with
-// fully coalesced 16-byte streaming stores.  Rows are at least a few KB, so a
-// gather of whole rows runs at the same DRAM efficiency as a flat copy.  The
-// loads of the next chunk are issued before the stores of the current one.
+// Both are row movers bound by HBM: whole rows of a few KB are read with
+// 16-byte streaming loads and written with coalesced 16-byte stores, several
+// loads per thread in flight before their stores, and grids of many short CTAs
+// (a gather of whole rows runs at the DRAM efficiency of a flat copy).
+// Dispatch has a token-major kernel (default, needs slot[]), two row-major ones
+// and a bulk-copy variant; combine is one warp per token.
 #include <stdlib.h>
 
 #include "common.cuh"
@@ -17,9 +18,9 @@ namespace {
 constexpr int kCH = 4;
 constexpr int kThreads = 256;
 
-// buf[row] = x[inv[row]] or zeros.  V = 16-byte vectors per row.  Four loads per lane are issued before their
-// stores; the register count is held at 32 so that 2048 threads per SM are resident (128 KB of loads in flight per
-// SM), which measured faster than a deeper software pipeline at half the occupancy.
+// Row-major, one warp per buffer row: buf[row] = x[inv[row]] or zeros.  V = 16-byte vectors per row.  Four loads
+// per lane are issued before their stores; six CTAs (1536 threads) per SM are resident, which measured faster than
+// a deeper software pipeline at half the occupancy.  Used beyond 2^32 vectors, or with LOCMOE_DISPATCH=vec.
 __global__ void __launch_bounds__(kThreads, 6) dispatch_vec_kernel(const uint4* __restrict__ x, const int32_t* __restrict__ inv,
                                                                    uint4* __restrict__ buf, long long rows, int V, int T,
                                                                    int zero_pad) {
@@ -333,6 +334,36 @@ int grid_for(long long units, int warps_per_block, int blocks_per_sm) {
 
 }  // namespace
 
+// Bulk-copy dispatch: segments of at most 16 KB that divide the row into equal multiples of 16 bytes.
+// Returns 1 when the row size does not suit it.
+static int launch_dispatch_tma(const locmoe_shape_t& s, int64_t rows, size_t rb, const void* x, const int32_t* inv, void* buf,
+                               int zero_pad, cudaStream_t st) {
+    int nseg = (int)((rb + 16383) / 16384);
+    while (nseg <= 64 && (rb % ((size_t)nseg * 16) != 0)) ++nseg;
+    if (nseg > 64) return 1;
+    const uint32_t seg = (uint32_t)(rb / nseg);
+    int nw = (int)((220 * 1024 - seg) / (seg + 8));
+    if (nw > 24) nw = 24;
+    if (nw < 4) return 1;
+    const size_t smem = (size_t)seg * (nw + 1) + (size_t)nw * 8;
+    static bool attr_done_dev[64] = {false};   // the attribute is per device
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_done_dev[dev & 63]) {
+        if (cudaFuncSetAttribute(dispatch_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
+            cudaGetLastError();
+            return LOCMOE_ERR_CUDA;
+        }
+        attr_done_dev[dev & 63] = true;
+    }
+    const long long want = (rows * nseg + nw - 1) / nw;
+    int g = sm_count();
+    if (want < g) g = (int)want;
+    dispatch_tma_kernel<<<g, nw * 32, smem, st>>>(static_cast<const unsigned char*>(x), inv, static_cast<unsigned char*>(buf),
+                                                  rows, nseg, seg, (long long)rb, s.T, zero_pad);
+    return check_launch();
+}
+
 int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const int32_t* inv, const int32_t* slot,
                     void* buf, int zero_pad, cudaStream_t st) {
     const int esz = s.x_dtype == LOCMOE_F32 ? 4 : 2;
@@ -340,39 +371,13 @@ int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const 
     const bool vec_ok = rb % 16 == 0 && (uintptr_t)x % 16 == 0 && (uintptr_t)buf % 16 == 0;
     // 16 CTAs per SM (more, shorter CTAs than are resident measured ~4 % faster than a resident-only grid)
     const int grid = grid_for(rows, kThreads / 32, 16);
-    // The load/store kernel is the default: on B200 the bulk-copy variant measured 218 us against 213 us on the
-    // 65536 x 5120 bf16 case (both are bound by the HBM write rate).  LOCMOE_DISPATCH=tma selects it.
+    // LOCMOE_DISPATCH = tma | vec | flat forces one of the other kernels (testing aid).  The load/store kernels are
+    // the default: the bulk-copy variant measured 218 us against 213 us for the warp-per-row kernel on the
+    // 65536 x 5120 bf16 case.
     const char* mode = getenv("LOCMOE_DISPATCH");
     if (vec_ok && mode && mode[0] == 't') {
-        // bulk-copy path: segments of at most 16 KB that divide the row into equal multiples of 16 bytes
-        int nseg = (int)((rb + 16383) / 16384);
-        while (nseg <= 64 && (rb % ((size_t)nseg * 16) != 0)) ++nseg;
-        if (nseg <= 64) {
-            const uint32_t seg = (uint32_t)(rb / nseg);
-            int nw = (int)((220 * 1024 - seg) / (seg + 8));
-            if (nw > 24) nw = 24;
-            if (nw >= 4) {
-                const size_t smem = (size_t)seg * (nw + 1) + (size_t)nw * 8;
-                static bool attr_done_dev[64] = {false};   // the attribute is per device
-    int attr_dev = 0;
-    cudaGetDevice(&attr_dev);
-    bool& attr_done = attr_done_dev[attr_dev & 63];
-                if (!attr_done) {
-                    if (cudaFuncSetAttribute(dispatch_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
-                        cudaGetLastError();
-                        return LOCMOE_ERR_CUDA;
-                    }
-                    attr_done = true;
-                }
-                long long want = (rows * nseg + nw - 1) / nw;
-                int g = sm_count();
-                if (want < g) g = (int)want;
-                dispatch_tma_kernel<<<g, nw * 32, smem, st>>>(static_cast<const unsigned char*>(x), inv,
-                                                              static_cast<unsigned char*>(buf), rows, nseg, seg,
-                                                              (long long)rb, s.T, zero_pad);
-                return check_launch();
-            }
-        }
+        const int rc = launch_dispatch_tma(s, rows, rb, x, inv, buf, zero_pad, st);
+        if (rc != 1) return rc;   // 1: the row size does not suit the bulk-copy kernel, fall through
     }
     if (vec_ok && slot && !mode && (unsigned long long)s.T * (rb / 16) < 0xf0000000ull) {
         const unsigned total = (unsigned)((unsigned long long)s.T * (rb / 16));

@@ -416,3 +416,17 @@ def test_flat_dispatch_variant(P, monkeypatch):
     monkeypatch.setenv("LOCMOE_DISPATCH", "flat")
     P.run_staged(P.W.CONFIGS[2].scaled(6000), 1.25, full=True)
     P.run_staged(P.W.CONFIGS[1], 1.0, layout=1, full=True)
+
+
+def test_plain_launches_without_programmatic_dependent_launch():
+    # LOCMOE_PDL=0 is read once per process: run the staged comparison in a child process
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = ("import oracle; oracle.build(); from tests import parity as P; "
+            "P.run_staged(P.W.CONFIGS[2].scaled(6000), 1.0, full=True); "
+            "P.run_staged(P.W.CONFIGS[1], 1.0, layout=1, full=True, fused=False); print('ok')")
+    env = dict(os.environ, LOCMOE_PDL="0")
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and r.stdout.strip().endswith("ok"), r.stderr[-2000:]
