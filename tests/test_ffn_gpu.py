@@ -48,7 +48,11 @@ def _check_rows(P, buf, w_in, w_out, y, E, M, rows, y_is_bf16=True):
     (4, 2, 2, 70, 264, 520, torch.float32),
     (8, 1, 8, 40, 512, 1024, torch.bfloat16),    # M = 320, several k-blocks and n-tiles
 ])
-def test_expert_ffn_small_shapes_all_rows(P, E, N, Dn, C, H, F, ydt):
+@pytest.mark.parametrize("kernel", ["one_sm", "two_sm_single_acc", "two_sm"])
+def test_expert_ffn_small_shapes_all_rows(P, monkeypatch, kernel, E, N, Dn, C, H, F, ydt):
+    # the default is the two-SM kernel (cluster of two CTAs, tcgen05 cta_group::2); LOCMOE_FFN selects the others
+    if kernel != "two_sm":
+        monkeypatch.setenv("LOCMOE_FFN", "2s" if kernel == "two_sm_single_acc" else "1")
     B = P.B
     dev = torch.device("cuda:0")
     D = N * Dn
