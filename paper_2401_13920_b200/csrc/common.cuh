@@ -1,6 +1,9 @@
 // Internal declarations shared by the LocMoE kernels and the C-ABI front end.
 #pragma once
 
+#include <stdio.h>
+#include <stdlib.h>
+
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -14,8 +17,13 @@ constexpr int kNumSMsB200 = 148;
 // Number of SMs of the current device (cached per process; B200 has 148).
 int sm_count();
 
+// LOCMOE_DEBUG=1 prints the CUDA error behind a LOCMOE_ERR_CUDA to stderr.
 inline int check_launch() {
     cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        const char* d = getenv("LOCMOE_DEBUG");
+        if (d && d[0] == '1') fprintf(stderr, "locmoe: CUDA error %d (%s)\n", (int)e, cudaGetErrorString(e));
+    }
     return e == cudaSuccess ? LOCMOE_OK : LOCMOE_ERR_CUDA;
 }
 

@@ -11,7 +11,7 @@
 //   - eight epilogue warps read the accumulator with tcgen05.ld (one row per thread, half of the columns per
 //     warp), apply GeLU (first GEMM), convert and store.
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = epilogue.  Persistent CTAs, one per SM.
-// Two kernels share these pieces: ffn_gemm_kernel (one CTA per 128 x 256 tile) and, the default,
+// Two kernels share these pieces: ffn_gemm_kernel (one CTA per 128 x 256 tile, the default) and
 // ffn_gemm2_kernel (a cluster of two CTAs per 256 x 256 tile, tcgen05 cta_group::2; described at the kernel).
 // Every barrier wait is bounded; on a timeout the kernel raises the device diagnostics flag, leaves its
 // loops, frees its TMEM and returns.
@@ -222,6 +222,11 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
                 if (!ok) break;
             }
+            // tail: all asynchronous commits to this CTA's stage barriers have arrived before the CTA leaves
+            for (int i = 0; i < NSTAGE; ++i) {
+                if (!wait_or_abort(&empty[stage], phase ^ 1u, abort_word)) break;
+                if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
+            }
         }
     } else if (warp == 1) {
         if (lane == 0) {  // ---- MMA issuer ----
@@ -431,6 +436,12 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
                 if (!ok) break;
             }
+            // tail: every stage has been released, i.e. every commit that targets this CTA's barriers has arrived,
+            // before the CTA may leave (the commits are asynchronous and multicast to both CTAs)
+            for (int i = 0; i < NSTAGE2; ++i) {
+                if (!wait_or_abort(&empty[stage], phase ^ 1u, abort_word)) break;
+                if (++stage == NSTAGE2) { stage = 0; phase ^= 1u; }
+            }
         }
     } else if (warp == 1) {
         if (lane == 0 && leader) {  // ---- MMA issuer (leader CTA) ----
@@ -604,12 +615,13 @@ int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* 
                       const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st) {
     const int E = s.E;
     const int M = (int)(rows / E);
-    // The two-SM kernel is the default (4.68 ms against 4.81 ms for the one-SM kernel on E = 32, M = 2048,
-    // H = 2560, F = 10240 at full clocks).  LOCMOE_FFN=1 selects the one-SM kernel, 2s the single-accumulator form
-    // of the two-SM kernel (testing aids).
+    // LOCMOE_FFN=2 selects the two-SM kernel (4.68 ms against 4.81 ms for the one-SM kernel on E = 32, M = 2048,
+    // H = 2560, F = 10240 at full clocks), 2s its single-accumulator form.  It is opt-in: it passes every test and
+    // runs clean in the bench, but launches of it failed under multi-metric profiler captures for a reason that
+    // reading the code has not shown, so the one-SM kernel stays the default.
     const char* mode = getenv("LOCMOE_FFN");
-    if (!(mode && mode[0] == '1') && sm_count() >= 2) {
-        const int nacc = (mode && mode[0] == '2' && mode[1] == 's') ? 1 : 2;
+    if (mode && mode[0] == '2' && sm_count() >= 2) {
+        const int nacc = mode[1] == 's' ? 1 : 2;
         int rc = launch_gemm2(buf, w_in, h1, 0, 1, E, M, F, s.H, nacc, st);
         if (rc) return rc;
         return launch_gemm2(h1, w_out, y, y_dtype == LOCMOE_F32 ? 1 : 0, 0, E, M, s.H, F, nacc, st);

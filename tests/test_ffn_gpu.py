@@ -50,9 +50,9 @@ def _check_rows(P, buf, w_in, w_out, y, E, M, rows, y_is_bf16=True):
 ])
 @pytest.mark.parametrize("kernel", ["one_sm", "two_sm_single_acc", "two_sm"])
 def test_expert_ffn_small_shapes_all_rows(P, monkeypatch, kernel, E, N, Dn, C, H, F, ydt):
-    # the default is the two-SM kernel (cluster of two CTAs, tcgen05 cta_group::2); LOCMOE_FFN selects the others
-    if kernel != "two_sm":
-        monkeypatch.setenv("LOCMOE_FFN", "2s" if kernel == "two_sm_single_acc" else "1")
+    # LOCMOE_FFN=2 selects the two-SM kernel (cluster of two CTAs, tcgen05 cta_group::2), 2s its one-accumulator form
+    if kernel != "one_sm":
+        monkeypatch.setenv("LOCMOE_FFN", "2s" if kernel == "two_sm_single_acc" else "2")
     B = P.B
     dev = torch.device("cuda:0")
     D = N * Dn
@@ -83,8 +83,11 @@ def test_expert_ffn_rejects_send_layout_and_bad_sizes(P):
     assert B._lib.locmoe_expert_ffn(C.byref(sh), 4, 64, C.c_void_p(8), one, one, one, one, B.BF16, None) == -4
 
 
-def test_full_layer_config5_scaled(P):
+@pytest.mark.parametrize("kernel", ["one_sm", "two_sm"])
+def test_full_layer_config5_scaled(P, monkeypatch, kernel):
     # config 5: router + dispatch (RECV layout), expert FFN with random-init weights, combine; one C-ABI call
+    if kernel == "two_sm":
+        monkeypatch.setenv("LOCMOE_FFN", "2")
     W, B = P.W, P.B
     dev = torch.device("cuda:0")
     w = W.CONFIGS[5].scaled(8192)
