@@ -40,7 +40,7 @@ def parse_args():
     ap.add_argument("--layout", choices=["send", "recv"], default="send")
     ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--e2e-steps", type=int, default=12)
+    ap.add_argument("--e2e-steps", type=int, default=48, help="end-to-end steps (the three-stream pipeline needs a few steps to fill)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     ap.add_argument("--event-every", type=int, default=8, help="carry per-stage CUDA events on every n-th timed step")
     ap.add_argument("--unfused", action="store_true", help="capacity and route as two calls instead of locmoe_capacity_route")
