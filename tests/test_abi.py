@@ -79,3 +79,35 @@ def test_null_pointers_are_rejected_before_any_launch(B):
     assert lib.locmoe_route(C.byref(sh), None, None, None, 4, *([None] * 10), None, 0, None) == -1
     assert lib.locmoe_capacity_route(C.byref(sh), None, None, None, C.byref(rule), None, None, None, 4, *([None] * 10),
                                      None, 0, None) == -1
+
+
+def test_header_is_plain_c_and_links_from_a_c_program(tmp_path):
+    # the boundary is a C ABI: the header must compile as C99 (and C++), and a C program must link against the library
+    import shutil
+    import subprocess
+    from paper_2401_13920_b200 import build
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    hdr = os.path.join(root, "include", "locmoe.h")
+    gcc, gxx = shutil.which("gcc"), shutil.which("g++")
+    if not gcc or not gxx:
+        pytest.skip("no host compiler")
+    subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c", hdr], check=True)
+    subprocess.run([gxx, "-std=c++17", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", hdr], check=True)
+    src = tmp_path / "probe.c"
+    src.write_text(
+        '#include <stdio.h>\n#include "locmoe.h"\n'
+        "int main(void) {\n"
+        "    locmoe_shape_t s = {4096, 1024, 8, 2, 4, LOCMOE_F32, LOCMOE_LAYOUT_SEND};\n"
+        "    size_t bytes = 0;\n"
+        "    int rc = locmoe_workspace_bytes(&s, 64, &bytes);\n"
+        '    printf("%d %zu %s\\n", rc, bytes, locmoe_status_string(LOCMOE_ERR_SHAPE));\n'
+        "    s.H = 1023;\n"
+        "    return locmoe_workspace_bytes(&s, 64, &bytes) == LOCMOE_ERR_SHAPE && rc == LOCMOE_OK && bytes > 0 ? 0 : 1;\n"
+        "}\n")
+    lib = build.build()
+    exe = tmp_path / "probe"
+    subprocess.run([gcc, "-std=c99", "-I", os.path.join(root, "include"), str(src), "-o", str(exe), lib,
+                    "-Wl,-rpath," + os.path.dirname(lib)], check=True)
+    r = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert r.returncode == 0, r.stdout + r.stderr
+    assert r.stdout.split()[0] == "0" and "invalid shape" in r.stdout
