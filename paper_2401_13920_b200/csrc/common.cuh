@@ -153,7 +153,7 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
     asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-// ---- bulk asynchronous copies (TMA, untiled form) and their mbarrier, shared::cta only, never multicast ----
+// ---- bulk asynchronous copies (TMA, untiled form) and their mbarrier: the issuing CTA's shared memory only ----
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {

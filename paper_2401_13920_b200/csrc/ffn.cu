@@ -4,7 +4,7 @@
 //
 // Two grouped GEMMs (all experts in one launch each), both "NT": the activations [rows][K] and the
 // weights [E][N][K] are K-major, so both operands are loaded as 128-byte-swizzled K-major tiles.
-//   - TMA (cp.async.bulk.tensor, no multicast) fills a 4-stage ring of 128x64 (A) and 256x64 (B) bf16 tiles,
+//   - TMA (cp.async.bulk.tensor, each load into the issuing CTA only) fills a 4-stage ring of 128x64 (A) and 256x64 (B) bf16 tiles,
 //   - one elected thread issues tcgen05.mma (128 x 256 x 16 per instruction, fp32 accumulators in TMEM),
 //   - two 128x256 accumulators (512 TMEM columns) alternate, so the epilogue of a tile overlaps the MMAs
 //     of the next one,
@@ -305,7 +305,7 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 // into 128 x 256 accumulators in each CTA's own TMEM.  Per SM and k-block 32 KB instead of 48 KB come out of L2,
 // and the ring holds six stages instead of four.
 //   full[s]      leader only: both CTAs' TMA loads of stage s have landed (the peer's loads count their bytes on
-//                the leader's barrier: cp.async.bulk.tensor ... .cta_group::2, no multicast)
+//                the leader's barrier: cp.async.bulk.tensor ... .cta_group::2, data into the issuing CTA only)
 //   empty[s]     MMAs that read stage s are done (tcgen05.commit multicast to both CTAs)
 //   acc_full[i]  accumulator i complete (multicast)     acc_empty[i]  leader only: both CTAs' epilogues drained i
 // Remote arrives use mapa + mbarrier.arrive.release.cluster; waits that order cross-CTA data use acquire.cluster.
