@@ -1,6 +1,7 @@
 """Builds the C-ABI library ``liblocmoe.so`` in-tree with nvcc for sm_100a."""
 from __future__ import annotations
 
+import hashlib
 import os
 import shutil
 import subprocess
@@ -10,6 +11,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "liblocmoe.so")
+STAMP = LIB + ".sha256"   # digest of the sources the library was built from
 SOURCES = ["api.cu", "gate.cu", "capacity.cu", "capacity_noalloc.cu", "route.cu", "movers.cu", "ffn.cu", "aux_loss.cu", "loc_loss.cu", "cos_hist.cu", "peer.cu", "topk.cu"]
 
 
@@ -24,13 +26,27 @@ def sources() -> list[str]:
     return [os.path.join(CSRC, s) for s in SOURCES if os.path.exists(os.path.join(CSRC, s))]
 
 
-def stale() -> bool:
-    if not os.path.exists(LIB):
-        return True
-    t = os.path.getmtime(LIB)
-    deps = sources() + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cuh")]
+def _deps() -> list[str]:
+    deps = sources() + sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cuh"))
     deps.append(os.path.join(ROOT, "include", "locmoe.h"))
-    return any(os.path.getmtime(d) > t for d in deps)
+    return deps
+
+
+def _digest() -> str:
+    """Hash of everything the library is built from (file times do not survive every copy of the tree)."""
+    h = hashlib.sha256()
+    for d in _deps():
+        h.update(os.path.basename(d).encode())
+        with open(d, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def stale() -> bool:
+    if not os.path.exists(LIB) or not os.path.exists(STAMP):
+        return True
+    with open(STAMP) as f:
+        return f.read().strip() != _digest()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -53,6 +69,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
     os.replace(tmp, LIB)
+    with open(STAMP + ".tmp%d" % os.getpid(), "w") as f:
+        f.write(_digest())
+    os.replace(STAMP + ".tmp%d" % os.getpid(), STAMP)
     return LIB
 
 
