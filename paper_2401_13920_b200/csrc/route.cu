@@ -15,9 +15,13 @@
 //             with warp match operations and per-warp digit counters, moves
 //             (key, token) to the sorted position and adds to the next pass's
 //             histogram with integer atomics; the last pass emits the outputs.
-//   extras    key-class starts and count matrices (kept, send_counts, load,
-//             locality tallies): extra CTAs of scatter_0 when P > 1, a launch
-//             of their own before the only scatter when P = 1.
+//   extras    ride on the scatters as extra CTAs: key-class starts and first buffer rows (no capacity needed) on
+//             the first scatter -- a launch of their own before the only scatter when P = 1 --, the count
+//             matrices (kept, send_counts, load, locality tallies), which need the capacity, on the last one.
+//   prescan   large batches only: one launch per pass that prefix-scans the histogram matrix along the tiles.
+// In the fused call (locmoe_capacity_route) the capacity stage has no launch of its own: hist0 also takes the
+// per-expert minima of the cosines of its tile, and one more extra CTA of the first scatter combines them and
+// evaluates the capacity rule; the last scatter reads the record.
 #include <stdlib.h>
 
 #include "capacity_finish.cuh"
