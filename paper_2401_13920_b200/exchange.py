@@ -103,3 +103,44 @@ class PeerBuffers:
             return
         (stream or torch.cuda.current_stream()).synchronize()
         dist.barrier(group=self.group)
+
+
+def peer_layer_forward(B, sharding, shape_local, C_alloc, rule, x, src_dev, recv: "PeerBuffers", y: "PeerBuffers",
+                       st, w_in=None, w_out=None, F=0, h1=None, out=None, group=None, stream=None):
+    """One MoE layer pass on this rank with the exchange fused into dispatch and combine.
+
+    ``shape_local`` describes the WHOLE logical map with ``T`` = this rank's tokens and the receive-side layout;
+    ``x`` / ``src_dev`` are this rank's tokens and their (global) source devices; ``st`` is a ``binding.RouterState``
+    for ``shape_local``; ``recv`` / ``y`` hold every rank's slice of the receive-side buffer and of the expert
+    outputs (``y`` may be ``recv`` itself for identity experts).  ``w_in`` / ``w_out`` are the weights of THIS
+    rank's experts ([E / world][F][H] and [E / world][H][F]).  Sequence: gate -> per-rank minima -> batch-wide
+    capacity (All-Reduce MIN / SUM on the host side of ``sharding.global_capacity_inputs``) -> route -> peer-store
+    dispatch -> barrier -> local experts -> barrier -> peer-load combine.  Only call sequencing lives here.
+    """
+    world = recv.world
+    rank = dist.get_rank(group) if world > 1 else 0
+    D = shape_local.D
+    devs = sharding.devices_of_rank(D, world, rank)
+    out = st.out if out is None else out
+    B.locmoe_gate(shape_local, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
+    B.locmoe_capacity(shape_local, st.idx, st.cos_sim, rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
+    if world > 1:
+        (stream or torch.cuda.current_stream()).synchronize()
+    delta, T_global = sharding.global_capacity_inputs(st.delta_e, shape_local.T, group)
+    rule_g = B.CapacityRule(rule.min_mult, rule.capacity_factor, delta if rule.delta_override < 0 else rule.delta_override,
+                            rule.bound_form, T_global)
+    B.locmoe_capacity_route(shape_local, st.idx, st.cos_sim, src_dev, rule_g, st.delta_e, st.theta_e, st.cap_dev, C_alloc,
+                            st.pos, st.slot, st.drop, st.inv, st.counts, st.kept, st.send_counts, st.load, st.locality,
+                            st.status, st.ws, stream)
+    B.locmoe_dispatch_peer(shape_local, C_alloc, x, st.inv, st.slot, recv.pointers, devs.start, devs.stop, True, stream)
+    recv.barrier(stream)
+    ydt = B.dtype_code(y.local.dtype)
+    if w_in is not None:
+        # this rank's experts on its slice of the receive buffer: a shape whose experts are the local ones
+        # (one logical device holding E / world experts with D * C_alloc rows each: the same rows, regrouped)
+        E_loc = shape_local.E // world
+        sh_ffn = B.make_shape(shape_local.T, shape_local.H, E_loc, 1, 1, recv.local.dtype, B.LAYOUT_RECV)
+        B.locmoe_expert_ffn(sh_ffn, D * C_alloc, F, recv.local, w_in, w_out, h1, y.local, stream)
+    y.barrier(stream)
+    B.locmoe_combine_peer(shape_local, C_alloc, y.pointers, ydt, st.slot, st.gate_w, out, stream)
+    return out

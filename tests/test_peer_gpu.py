@@ -133,3 +133,39 @@ def test_peer_calls_reject_bad_arguments(P):
         B.locmoe_dispatch_peer(sh, 4, x, inv, slot, [buf, buf, buf], 0, 4)
     with pytest.raises(B.LocMoEError):            # source range outside the map
         B.locmoe_dispatch_peer(sh, 4, x, inv, slot, [buf], 0, 5)
+
+
+@pytest.mark.parametrize("with_ffn", [False, True])
+def test_single_rank_peer_layer_equals_the_layer_call(P, with_ffn):
+    # with one rank the fused-exchange sequence must reproduce locmoe_moe_layer bit for bit
+    from paper_2401_13920_b200 import exchange, sharding
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    w = W.CONFIGS[5].scaled(4096)
+    F = 512
+    x, src = W.make_tokens(w, dev), W.make_src(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, B.LAYOUT_RECV)
+    rule = B.CapacityRule(1.0, 1.0, -1.0, 0, 0)
+    Ca = B.conventional_capacity(w.T, sh.D, w.E, 1.0)
+    w_in = w_out = None
+    if with_ffn:
+        w_in, w_out = W.make_expert_weights(w, F, dev)
+    # reference: the one-call layer
+    st = B.make_router(sh, Ca, rule, dev)
+    h1 = torch.empty(st.rows, F, dtype=torch.bfloat16, device=dev)
+    y = torch.empty(st.rows, w.H, dtype=torch.bfloat16, device=dev)
+    want = torch.empty(w.T, w.H, dtype=x.dtype, device=dev)
+    B.locmoe_moe_layer(sh, x, src, None, rule, Ca, F, w_in, w_out, B.layer_buffers(st, h1, y), want)
+    torch.cuda.synchronize()
+    # the per-rank sequence with peer stores / loads
+    st2 = B.make_router(sh, Ca, rule, dev)
+    recv = exchange.PeerBuffers(st.rows, w.H, x.dtype, dev)
+    yb = exchange.PeerBuffers(st.rows, w.H, torch.bfloat16, dev) if with_ffn else recv
+    recv.local.fill_(3.0)
+    h1b = torch.empty(st.rows, F, dtype=torch.bfloat16, device=dev)
+    got = torch.empty(w.T, w.H, dtype=x.dtype, device=dev)
+    exchange.peer_layer_forward(B, sharding, sh, Ca, rule, x, src, recv, yb, st2, w_in, w_out, F, h1b, out=got)
+    torch.cuda.synchronize()
+    assert B.locmoe_device_flags() == 0
+    assert torch.equal(st2.slot, st.slot) and torch.equal(recv.local.view(torch.int16), st.buf.view(torch.int16))
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
