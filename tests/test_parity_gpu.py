@@ -153,6 +153,8 @@ def test_separate_calls_full_size_config2(P):
     dict(T=2049, H=2048, E=8, n_nodes=2, dev_per_node=4, dtype="f32"),  # group spans whole warp iterations
     dict(T=3000, H=4096, E=2048, n_nodes=1, dev_per_node=1),            # > 1024 keys on a single device
     dict(T=4097, H=2048, E=2048, n_nodes=8, dev_per_node=8),            # 131072 keys: three radix passes; g = 1
+    dict(T=300, H=16384, E=16384, n_nodes=1, dev_per_node=1),           # > 8192 experts: minima by global atomics,
+                                                                        # capacity and route not fused
 ])
 @pytest.mark.parametrize("layout", [0, 1])
 def test_shapes(P, kw, layout):
