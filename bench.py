@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=48, help="end-to-end steps (the three-stream pipeline needs a few steps to fill)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     ap.add_argument("--event-every", type=int, default=8, help="carry per-stage CUDA events on every n-th timed step")
+    ap.add_argument("--variant", choices=["router", "peer8", "topk2"], default="router",
+                    help="router: the metric's path; peer8: dispatch / combine through a table of eight receive buffers "
+                         "(the fused-exchange kernels, all buffers on this GPU); topk2: the top-2 variant")
     ap.add_argument("--unfused", action="store_true", help="capacity and route as two calls instead of locmoe_capacity_route")
     ap.add_argument("--no-ffn", action="store_true", help="config 5 only: identity experts instead of the expert FFN")
     ap.add_argument("--ffn-inner", type=int, default=10240, help="config 5: inner size F of the expert FFN")
@@ -192,7 +195,10 @@ def workload_config(w, args, n_tokens=None):
     return {
         "workload": "config %d (%s): T=%d H=%d E=%d %s tokens, %dx%d logical devices, c_f=%g, %s layout" % (
             w.config, w.name, n_tokens or w.T, w.H, w.E, w.dtype, w.n_nodes, w.dev_per_node, args.cf, args.layout),
-        "expert_ffn": bool((w.config % 10) == 5 and not getattr(args, "no_ffn", False)),
+        "expert_ffn": bool((w.config % 10) == 5 and not getattr(args, "no_ffn", False) and getattr(args, "variant", "router") == "router"),
+        "variant": {"router": "the metric's path (top-1, one GPU)",
+                    "peer8": "dispatch / combine through a table of eight receive buffers (fused-exchange kernels, all on this GPU)",
+                    "topk2": "top-2 variant: 2T assignments routed, two-term combine"}[getattr(args, "variant", "router")],
         "T": n_tokens or w.T, "H": w.H, "E": w.E, "token_dtype": w.dtype, "n_nodes": w.n_nodes,
         "dev_per_node": w.dev_per_node, "capacity_factor": args.cf, "layout": args.layout,
         "l2": "inputs exceed the 126 MB L2, no flush" if (n_tokens or w.T) * w.H * (2 if w.dtype == "bf16" else 4) > 126e6
@@ -232,8 +238,11 @@ def main():
         # every rank routes its own batch: same shape, its own seed
         w = W.Workload(**{**w.__dict__, "config": w.config + 10 * rank, "name": w.name})
     use_ffn = (w.config % 10) == 5 and not args.no_ffn
-    if use_ffn:
-        args.layout = "recv"      # the expert FFN works on the per-expert contiguous (receive-side) layout
+    variant = args.variant
+    if variant != "router":
+        use_ffn = False
+    if use_ffn or variant == "peer8":
+        args.layout = "recv"      # the expert FFN and the peer kernels work on the receive-side layout
     layout = B.LAYOUT_SEND if args.layout == "send" else B.LAYOUT_RECV
     x = W.make_tokens(w, dev)
     src = W.make_src(w, dev)
@@ -257,6 +266,21 @@ def main():
     stages = ["gate"] + (["capacity_route"] if fused else ["capacity", "route"]) + ["dispatch"] + \
              (["ffn"] if use_ffn else []) + ["combine"]
 
+    tk = None
+    if variant == "peer8":
+        n_peers = 8
+        while shape.D % n_peers:
+            n_peers //= 2
+        rpp = st.rows // n_peers
+        peer_bufs = [st.buf[q * rpp:(q + 1) * rpp] for q in range(n_peers)]   # eight receive buffers, all on this GPU
+        stages = ["gate", "capacity_route", "dispatch", "combine"]
+    elif variant == "topk2":
+        K2 = 2
+        C_alloc = B.conventional_capacity(K2 * w.T, shape.D, w.E, args.cf)
+        tk = B.make_topk_state(shape, K2, C_alloc, dev)
+        src_k = src.repeat(K2).contiguous()
+        stages = ["gate", "capacity", "select", "route", "dispatch", "combine"]
+
     def step(ev=None):
         sh, Ca = st.shape, st.C_alloc
         i = 0
@@ -265,6 +289,22 @@ def main():
             if ev:
                 ev[i].record(stream)
             i += 1
+        if variant == "topk2":
+            B.topk_forward(tk, x, src_k, rule, stream=stream, mark=mark)
+            return
+        if variant == "peer8":
+            mark()
+            B.locmoe_gate(sh, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
+            mark()
+            B.locmoe_capacity_route(sh, st.idx, st.cos_sim, src, st.rule, st.delta_e, st.theta_e, st.cap_dev, Ca, st.pos,
+                                    st.slot, st.drop, st.inv, st.counts, st.kept, st.send_counts, st.load, st.locality,
+                                    st.status, st.ws, stream)
+            mark()
+            B.locmoe_dispatch_peer(sh, Ca, x, st.inv, st.slot, peer_bufs, 0, sh.D, True, stream)
+            mark()
+            B.locmoe_combine_peer(sh, Ca, peer_bufs, B.dtype_code(x.dtype), st.slot, st.gate_w, st.out, stream)
+            mark()
+            return
         mark()
         B.locmoe_gate(sh, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
         mark()
@@ -337,14 +377,15 @@ def main():
 
     stage_ms = {s: float(np.mean([evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(n_ev)])) for i, s in enumerate(stages)}
     # ---- algorithmic bytes per launch (per token: see the per-kernel byte model in the design notes) ----
-    kept = int((st.slot >= 0).sum().item())
+    slot_t = tk["slot"] if tk is not None else st.slot
+    kept = int((slot_t >= 0).sum().item())            # kept assignments (tokens, or token-choice pairs for top-k)
     bx = x.element_size()
     by = ysrc.element_size()
-    rows = st.rows
+    rows = st.rows if tk is None else shape.D * w.E * C_alloc
     bytes_per_launch = {
-        "gate": w.T * w.H * bx + 12 * w.T,
+        "gate": w.T * w.H * bx + 12 * w.T + (4 * w.T * w.E if tk is not None else 0),
         "dispatch": kept * w.H * bx + rows * w.H * bx + 4 * rows,
-        "combine": kept * w.H * by + w.T * w.H * bx + 8 * w.T,
+        "combine": kept * w.H * by + w.T * w.H * bx + 8 * w.T * (tk["K"] if tk is not None else 1),
     }
     peak, peak_kind = measured_peak()
     kernels = {}
@@ -352,7 +393,7 @@ def main():
         gbs = bytes_per_launch[s] / (stage_ms[s] * 1e-3) / 1e9
         kernels[s] = {"ms": stage_ms[s], "bytes": bytes_per_launch[s], "achieved_gbs": gbs, "frac": gbs / peak}
     dominant = max(("gate", "dispatch", "combine"), key=lambda s: stage_ms[s])
-    traffic = ncu_traffic(dominant, w, args.cf, args.tokens)
+    traffic = ncu_traffic(dominant, w, args.cf, args.tokens) if variant == "router" else None
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["achieved_gbs"], "peak": peak,
                 "peak_kind": peak_kind + " (copy, MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
                 "unit": "GB/s", "frac": kernels[dominant]["frac"], "traffic": traffic,
@@ -369,7 +410,10 @@ def main():
                          "hbm_kernels": kernels})
 
     launches = B.locmoe_launch_counts(shape)
-    if fused:
+    if variant == "topk2":
+        lv = B.locmoe_launch_counts(tk["shape_v"])
+        launches = {"gate": 1, "capacity": launches["capacity"], "select": 1, "route": lv["route"] + 1, "dispatch": 1, "combine": 1}
+    elif fused:
         # the capacity stage rides on the route stage's launches (up to 8192 experts)
         cr = launches.pop("route") + (launches["capacity"] if shape.E > 8192 else 0)
         launches.pop("capacity")
@@ -377,11 +421,11 @@ def main():
     if use_ffn:
         launches["ffn"] = 2
     launches_per_step = sum(launches.values())
-    cap = B.locmoe_capacity_read(st.cap_dev)
+    cap = B.locmoe_capacity_read(tk["cap_dev"] if tk is not None else st.cap_dev)
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
     e2e = None
-    if args.e2e_steps > 0 and not use_ffn:
+    if args.e2e_steps > 0 and not use_ffn and variant == "router":
         xh = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
         xh.copy_(x)
         srch = torch.empty(src.shape, dtype=src.dtype, pin_memory=True)

@@ -474,21 +474,17 @@ def router_forward(st: RouterState, x, src_dev, y=None, eps=None, stream=None, o
     return out
 
 
-def router_forward_topk(shape: Shape, x, src_dev, K: int, C_alloc: int, rule: CapacityRule, y=None, stream=None) -> dict:
-    """The top-k variant end to end on one stream (allocates its tensors: a convenience for tests and examples).
-
-    gate (with probabilities) -> capacity on the first choices, counting K * T assignments -> K best experts ->
-    route of the K * T virtual tokens -> fold -> dispatch -> combine over the K choices.  ``y`` are the expert outputs
-    in slot layout (identity experts when None).  Returns the tensors by name.
-    """
-    dev = x.device
+def make_topk_state(shape: Shape, K: int, C_alloc: int, device="cuda") -> dict:
+    """Tensors of the top-k variant for T tokens and K choices (memory plumbing only)."""
+    dev = torch.device(device)
     T, H, E, D = shape.T, shape.H, shape.E, shape.D
     i32 = dict(dtype=torch.int32, device=dev)
     f32 = dict(dtype=torch.float32, device=dev)
     xdt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
     shape_v = Shape(K * T, H, E, shape.n_nodes, shape.dev_per_node, shape.x_dtype, shape.layout)
     rows = D * E * C_alloc
-    r = dict(
+    return dict(
+        K=K, C_alloc=C_alloc, shape=shape, shape_v=shape_v,
         idx=torch.empty(T, **i32), gate_w=torch.empty(T, **f32), cos_sim=torch.empty(T, **f32), probs=torch.empty(T, E, **f32),
         delta_e=torch.empty(E, **f32), theta_e=torch.empty(E, **f32),
         cap_dev=torch.zeros(CAPACITY_BYTES, dtype=torch.uint8, device=dev),
@@ -500,18 +496,40 @@ def router_forward_topk(shape: Shape, x, src_dev, K: int, C_alloc: int, rule: Ca
         ws=torch.empty(max(locmoe_workspace_bytes(shape_v, C_alloc), locmoe_workspace_bytes(shape, C_alloc)),
                        dtype=torch.uint8, device=dev),
         buf=torch.empty(rows, H, dtype=xdt, device=dev), out=torch.empty(T, H, dtype=xdt, device=dev),
-        src_k=src_dev.repeat(K).contiguous(),
     )
-    rule_k = CapacityRule(rule.min_mult, rule.capacity_factor, rule.delta_override, rule.bound_form, K * T)
+
+
+def topk_forward(r: dict, x, src_k, rule: CapacityRule, y=None, stream=None, mark=None) -> dict:
+    """The top-k variant on one stream: gate (with probabilities) -> capacity on the first choices, counting K * T
+    assignments -> K best experts -> route of the K * T virtual tokens -> fold -> dispatch -> combine over the K
+    choices.  ``src_k`` is the source-device array repeated K times; ``y`` are the expert outputs in slot layout
+    (identity experts when None); ``mark`` is called between the stages (the bench records events there)."""
+    shape, shape_v, K, C_alloc = r["shape"], r["shape_v"], r["K"], r["C_alloc"]
+    mark = mark or (lambda: None)
+    rule_k = CapacityRule(rule.min_mult, rule.capacity_factor, rule.delta_override, rule.bound_form, K * shape.T)
+    mark()
     locmoe_gate(shape, x, None, r["idx"], r["gate_w"], r["cos_sim"], r["probs"], stream)
+    mark()
     locmoe_capacity(shape, r["idx"], r["cos_sim"], rule_k, r["delta_e"], r["theta_e"], r["cap_dev"], r["ws"], stream)
+    mark()
     locmoe_topk_select(shape, r["probs"], r["idx"], r["gate_w"], K, r["idx_k"], r["w_k"], stream)
-    locmoe_route(shape_v, r["idx_k"], r["src_k"], r["cap_dev"], C_alloc, r["pos"], r["slot"], r["drop"], r["inv"],
+    mark()
+    locmoe_route(shape_v, r["idx_k"], src_k, r["cap_dev"], C_alloc, r["pos"], r["slot"], r["drop"], r["inv"],
                  r["counts"], r["kept"], r["send_counts"], r["load"], r["locality"], r["status"], r["ws"], stream)
     locmoe_topk_fold(shape, C_alloc, r["inv"], stream)
+    mark()
     locmoe_dispatch(shape, C_alloc, x, r["inv"], r["buf"], True, stream)
+    mark()
     locmoe_combine_topk(shape, C_alloc, r["buf"] if y is None else y, K, r["slot"], r["w_k"], r["out"], stream)
+    mark()
     return r
+
+
+def router_forward_topk(shape: Shape, x, src_dev, K: int, C_alloc: int, rule: CapacityRule, y=None, stream=None) -> dict:
+    """Allocates the state and runs the top-k variant once (a convenience for tests and examples)."""
+    r = make_topk_state(shape, K, C_alloc, x.device)
+    r["src_k"] = src_dev.repeat(K).contiguous()
+    return topk_forward(r, x, r["src_k"], rule, y=y, stream=stream)
 
 
 class HostRouter:

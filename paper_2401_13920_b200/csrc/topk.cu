@@ -55,21 +55,28 @@ __global__ void __launch_bounds__(kThreads) topk_fold_kernel(int32_t* __restrict
     }
 }
 
-__device__ __forceinline__ void load8(const void* base, size_t octet, int dt, float (&f)[8]) {
+// One octet (8 elements) of a row: raw 16-byte loads now, widening to fp32 at the point of use (fewer live registers).
+struct RawOctet { uint4 a, b; };
+__device__ __forceinline__ void load_raw(const void* base, size_t octet, int dt, RawOctet& r) {
     if (dt == LOCMOE_F32) {
         const uint4* p = reinterpret_cast<const uint4*>(base) + octet * 2;
-        const uint4 a = ld_stream(p), b = ld_stream(p + 1);
-        f[0] = __uint_as_float(a.x); f[1] = __uint_as_float(a.y); f[2] = __uint_as_float(a.z); f[3] = __uint_as_float(a.w);
-        f[4] = __uint_as_float(b.x); f[5] = __uint_as_float(b.y); f[6] = __uint_as_float(b.z); f[7] = __uint_as_float(b.w);
+        r.a = ld_stream(p); r.b = ld_stream(p + 1);
     } else {
-        const uint4 a = ld_stream(reinterpret_cast<const uint4*>(base) + octet);
-        f[0] = bf16_lo(a.x); f[1] = bf16_hi(a.x); f[2] = bf16_lo(a.y); f[3] = bf16_hi(a.y);
-        f[4] = bf16_lo(a.z); f[5] = bf16_hi(a.z); f[6] = bf16_lo(a.w); f[7] = bf16_hi(a.w);
+        r.a = ld_stream(reinterpret_cast<const uint4*>(base) + octet);
+    }
+}
+__device__ __forceinline__ void widen8(const RawOctet& r, int dt, float (&f)[8]) {
+    if (dt == LOCMOE_F32) {
+        f[0] = __uint_as_float(r.a.x); f[1] = __uint_as_float(r.a.y); f[2] = __uint_as_float(r.a.z); f[3] = __uint_as_float(r.a.w);
+        f[4] = __uint_as_float(r.b.x); f[5] = __uint_as_float(r.b.y); f[6] = __uint_as_float(r.b.z); f[7] = __uint_as_float(r.b.w);
+    } else {
+        f[0] = bf16_lo(r.a.x); f[1] = bf16_hi(r.a.x); f[2] = bf16_lo(r.a.y); f[3] = bf16_hi(r.a.y);
+        f[4] = bf16_lo(r.a.z); f[5] = bf16_hi(r.a.z); f[6] = bf16_lo(r.a.w); f[7] = bf16_hi(r.a.w);
     }
 }
 
-template <int K>
-__global__ void __launch_bounds__(kThreads) combine_topk_kernel(const void* __restrict__ y, int ydt,
+template <int K, int YDT>
+__global__ void __launch_bounds__(kThreads) combine_topk_kernel(const void* __restrict__ y,
                                                                 const int32_t* __restrict__ slot_k,
                                                                 const float* __restrict__ w_k, void* __restrict__ out, int odt,
                                                                 int T, int O, long long rows, int tpc) {
@@ -85,28 +92,43 @@ __global__ void __launch_bounds__(kThreads) combine_topk_kernel(const void* __re
             w[c] = w_k[(size_t)c * T + t];
             if (s[c] < 0 || s[c] >= rows) s[c] = -1;
         }
-        for (int o = lane; o < O; o += 32) {
-            float v[K][8];
+        // octets in flight per lane: two for small K (as the top-1 combine), one otherwise (registers)
+        constexpr int NO = K <= 2 ? 2 : 1;
+        for (int o0 = lane; o0 < O; o0 += 32 * NO) {
+            RawOctet raw[NO][K];
 #pragma unroll
-            for (int c = 0; c < K; ++c)
-                if (s[c] >= 0) load8(y, (size_t)s[c] * O + o, ydt, v[c]);
-            float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-            bool first = true;
+            for (int h = 0; h < NO; ++h) {
+                const int o = o0 + 32 * h;
+                if (o < O) {
 #pragma unroll
-            for (int c = 0; c < K; ++c) {
-                if (s[c] < 0) continue;
-#pragma unroll
-                for (int k = 0; k < 8; ++k) acc[k] = first ? __fmul_rn(w[c], v[c][k]) : __fmaf_rn(w[c], v[c][k], acc[k]);
-                first = false;
+                    for (int c = 0; c < K; ++c)
+                        if (s[c] >= 0) load_raw(y, (size_t)s[c] * O + o, YDT, raw[h][c]);
+                }
             }
-            if (odt == LOCMOE_F32) {
-                uint4* p = reinterpret_cast<uint4*>(out) + ((size_t)t * O + o) * 2;
-                st_stream(p, make_uint4(__float_as_uint(acc[0]), __float_as_uint(acc[1]), __float_as_uint(acc[2]), __float_as_uint(acc[3])));
-                st_stream(p + 1, make_uint4(__float_as_uint(acc[4]), __float_as_uint(acc[5]), __float_as_uint(acc[6]), __float_as_uint(acc[7])));
-            } else {
-                st_stream(reinterpret_cast<uint4*>(out) + (size_t)t * O + o,
-                          make_uint4(cvt_bf16x2(make_float2(acc[0], acc[1])), cvt_bf16x2(make_float2(acc[2], acc[3])),
-                                     cvt_bf16x2(make_float2(acc[4], acc[5])), cvt_bf16x2(make_float2(acc[6], acc[7]))));
+#pragma unroll
+            for (int h = 0; h < NO; ++h) {
+                const int o = o0 + 32 * h;
+                if (o >= O) continue;
+                float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                bool first = true;
+#pragma unroll
+                for (int c = 0; c < K; ++c) {
+                    if (s[c] < 0) continue;
+                    float v[8];
+                    widen8(raw[h][c], YDT, v);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) acc[k] = first ? __fmul_rn(w[c], v[k]) : __fmaf_rn(w[c], v[k], acc[k]);
+                    first = false;
+                }
+                if (odt == LOCMOE_F32) {
+                    uint4* p = reinterpret_cast<uint4*>(out) + ((size_t)t * O + o) * 2;
+                    st_stream(p, make_uint4(__float_as_uint(acc[0]), __float_as_uint(acc[1]), __float_as_uint(acc[2]), __float_as_uint(acc[3])));
+                    st_stream(p + 1, make_uint4(__float_as_uint(acc[4]), __float_as_uint(acc[5]), __float_as_uint(acc[6]), __float_as_uint(acc[7])));
+                } else {
+                    st_stream(reinterpret_cast<uint4*>(out) + (size_t)t * O + o,
+                              make_uint4(cvt_bf16x2(make_float2(acc[0], acc[1])), cvt_bf16x2(make_float2(acc[2], acc[3])),
+                                         cvt_bf16x2(make_float2(acc[4], acc[5])), cvt_bf16x2(make_float2(acc[6], acc[7]))));
+                }
             }
         }
     }
@@ -138,7 +160,10 @@ int launch_combine_topk(const locmoe_shape_t& s, int64_t rows, const void* y, in
     const int O = s.H / 8;
 #define LOCMOE_TOPK_CASE(KK)                                                                                           \
     case KK:                                                                                                           \
-        combine_topk_kernel<KK><<<grid, kThreads, 0, st>>>(y, y_dtype, slot_k, w_k, out, s.x_dtype, s.T, O, rows, tpc); \
+        if (y_dtype == LOCMOE_F32)                                                                                     \
+            combine_topk_kernel<KK, LOCMOE_F32><<<grid, kThreads, 0, st>>>(y, slot_k, w_k, out, s.x_dtype, s.T, O, rows, tpc);  \
+        else                                                                                                           \
+            combine_topk_kernel<KK, LOCMOE_BF16><<<grid, kThreads, 0, st>>>(y, slot_k, w_k, out, s.x_dtype, s.T, O, rows, tpc); \
         break;
     switch (K) {
         LOCMOE_TOPK_CASE(1) LOCMOE_TOPK_CASE(2) LOCMOE_TOPK_CASE(3) LOCMOE_TOPK_CASE(4)
