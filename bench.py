@@ -298,7 +298,7 @@ def main():
             mark()
             B.locmoe_capacity_route(sh, st.idx, st.cos_sim, src, st.rule, st.delta_e, st.theta_e, st.cap_dev, Ca, st.pos,
                                     st.slot, st.drop, st.inv, st.counts, st.kept, st.send_counts, st.load, st.locality,
-                                    st.status, st.ws, stream)
+                                    st.status, st.ws, stream, early_init=not ev)
             mark()
             B.locmoe_dispatch_peer(sh, Ca, x, st.inv, st.slot, peer_bufs, 0, sh.D, True, stream)
             mark()
@@ -311,7 +311,7 @@ def main():
         if fused:
             B.locmoe_capacity_route(sh, st.idx, st.cos_sim, src, st.rule, st.delta_e, st.theta_e, st.cap_dev, Ca, st.pos,
                                     st.slot, st.drop, st.inv, st.counts, st.kept, st.send_counts, st.load, st.locality,
-                                    st.status, st.ws, stream)
+                                    st.status, st.ws, stream, early_init=not ev)   # eager steps record an event in between
         else:
             B.locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
             mark()

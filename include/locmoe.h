@@ -204,13 +204,21 @@ int locmoe_route(const locmoe_shape_t *shape, const int32_t *idx, const int32_t 
  * launch and no pass of its own; the last sorting pass reads the record from
  * cap_dev.  Beyond 8192 experts the two stages simply run one after the other.
  * ws: at least locmoe_workspace_bytes() bytes.
+ * flags: 0, or LOCMOE_ROUTE_EARLY_INIT: the caller states that the kernel queued
+ * on the stream immediately before this call (typically locmoe_gate of the same
+ * step) neither reads nor writes any output array or the workspace of this
+ * call, and, if it was itself launched for programmatic dependent launch, that
+ * it waits for its own predecessors before it lets its successor start (every
+ * kernel of this library does).  The stage's fill of inv / counters may then
+ * run while that kernel drains instead of after it.  Results are the same.
  */
+enum { LOCMOE_ROUTE_EARLY_INIT = 1 };
 int locmoe_capacity_route(const locmoe_shape_t *shape, const int32_t *idx, const float *cos_sim,
                           const int32_t *src_dev, const locmoe_capacity_rule_t *rule,
                           float *delta_e, float *theta_e, locmoe_capacity_t *cap_dev, int32_t C_alloc,
                           int32_t *pos, int32_t *slot, uint8_t *drop, int32_t *inv, int32_t *counts,
                           int32_t *kept, int32_t *send_counts, int32_t *load, int64_t *locality,
-                          int32_t *status, void *ws, size_t ws_bytes, void *stream);
+                          int32_t *status, int32_t flags, void *ws, size_t ws_bytes, void *stream);
 
 /*
  * Dispatch: buf[row][:] = x[inv[row]][:] bit for bit for occupied rows; rows

@@ -19,6 +19,7 @@ from . import build as _build
 F32, BF16 = 0, 1
 LAYOUT_SEND, LAYOUT_RECV = 0, 1
 BOUND_BETA, BOUND_ERFC, BOUND_EXP = 0, 1, 2
+ROUTE_EARLY_INIT = 1
 WARN_CLAMPED, WARN_BAD_SRC, WARN_BAD_IDX = 1, 2, 4
 FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
@@ -75,7 +76,7 @@ def _load() -> C.CDLL:
     lib.locmoe_capacity_read.argtypes = [vp, C.POINTER(Capacity), vp]
     lib.locmoe_route.argtypes = [C.POINTER(Shape), vp, vp, vp, i32] + [vp] * 10 + [vp, C.c_size_t, vp]
     lib.locmoe_capacity_route.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(CapacityRule), vp, vp, vp, i32] + [vp] * 10 + \
-                                         [vp, C.c_size_t, vp]
+                                         [i32, vp, C.c_size_t, vp]
     lib.locmoe_dispatch.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, vp, i32, vp]
     lib.locmoe_combine.argtypes = [C.POINTER(Shape), i32, vp, i32, vp, vp, vp, i32, vp]
     lib.locmoe_expert_ffn.argtypes = [C.POINTER(Shape), i32, i32, vp, vp, vp, vp, vp, i32, vp]
@@ -235,7 +236,7 @@ def locmoe_route(shape: Shape, idx, src_dev, cap_dev, C_alloc, pos, slot, drop, 
 
 
 def locmoe_capacity_route(shape: Shape, idx, cos_sim, src_dev, rule: CapacityRule, delta_e, theta_e, cap_dev, C_alloc, pos, slot,
-                          drop, inv, counts, kept, send_counts, load, locality, status, ws, stream=None) -> int:
+                          drop, inv, counts, kept, send_counts, load, locality, status, ws, stream=None, early_init=False) -> int:
     D, E, T = shape.D, shape.E, shape.T
     for t, dt, n, name in ((idx, torch.int32, T, "idx"), (cos_sim, torch.float32, T, "cos_sim"), (src_dev, torch.int32, T, "src_dev"),
                            (delta_e, torch.float32, E, "delta_e"), (theta_e, torch.float32, E, "theta_e"),
@@ -248,7 +249,8 @@ def locmoe_capacity_route(shape: Shape, idx, cos_sim, src_dev, rule: CapacityRul
     return _check("locmoe_capacity_route", _lib.locmoe_capacity_route(
         C.byref(shape), _ptr(idx), _ptr(cos_sim), _ptr(src_dev), C.byref(rule), _ptr(delta_e), _ptr(theta_e), _ptr(cap_dev),
         int(C_alloc), _ptr(pos), _ptr(slot), _ptr(drop), _ptr(inv), _ptr(counts), _ptr(kept), _ptr(send_counts), _ptr(load),
-        _ptr(locality), _ptr(status), _ptr(ws), ws.numel() * ws.element_size(), _stream(stream)))
+        _ptr(locality), _ptr(status), ROUTE_EARLY_INIT if early_init else 0, _ptr(ws), ws.numel() * ws.element_size(),
+        _stream(stream)))
 
 
 def locmoe_dispatch(shape: Shape, C_alloc, x, inv, buf, zero_pad=True, stream=None, slot=None) -> int:
@@ -464,7 +466,7 @@ def router_forward(st: RouterState, x, src_dev, y=None, eps=None, stream=None, o
     if fused:
         locmoe_capacity_route(sh, st.idx, st.cos_sim, src_dev, st.rule, st.delta_e, st.theta_e, st.cap_dev, Ca, st.pos,
                               st.slot, st.drop, st.inv, st.counts, st.kept, st.send_counts, st.load, st.locality,
-                              st.status, st.ws, stream)
+                              st.status, st.ws, stream, early_init=True)   # the kernel before it is the gate above
     else:
         locmoe_capacity(sh, st.idx, st.cos_sim, st.rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
         locmoe_route(sh, st.idx, src_dev, st.cap_dev, Ca, st.pos, st.slot, st.drop, st.inv, st.counts, st.kept,

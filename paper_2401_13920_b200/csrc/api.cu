@@ -127,8 +127,8 @@ int locmoe_route(const locmoe_shape_t* shape, const int32_t* idx, const int32_t*
 int locmoe_capacity_route(const locmoe_shape_t* shape, const int32_t* idx, const float* cos_sim, const int32_t* src_dev,
                           const locmoe_capacity_rule_t* rule, float* delta_e, float* theta_e, locmoe_capacity_t* cap_dev,
                           int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
-                          int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status, void* ws,
-                          size_t ws_bytes, void* stream) {
+                          int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
+                          int32_t flags, void* ws, size_t ws_bytes, void* stream) {
     int rc = check_shape(shape);
     if (rc) return rc;
     if (!idx || !cos_sim || !src_dev || !rule || !delta_e || !theta_e || !cap_dev || !pos || !slot || !drop || !inv ||
@@ -140,6 +140,7 @@ int locmoe_capacity_route(const locmoe_shape_t* shape, const int32_t* idx, const
     if (!(rule->min_mult >= 0.0) || !(rule->capacity_factor >= 0.0) || rule->delta_override != rule->delta_override)
         return LOCMOE_ERR_SHAPE;
     if (buffer_rows(shape, C_alloc) < 0) return LOCMOE_ERR_SHAPE;
+    if (flags & ~LOCMOE_ROUTE_EARLY_INIT) return LOCMOE_ERR_DTYPE;
     RoutePlan p;
     if ((rc = plan_route(*shape, &p))) return rc;
     size_t need = p.total;
@@ -147,8 +148,8 @@ int locmoe_capacity_route(const locmoe_shape_t* shape, const int32_t* idx, const
     if (!ws || ws_bytes < need || (uintptr_t)ws % 256) return LOCMOE_ERR_WORKSPACE;
     if ((uintptr_t)locality % 8 || (uintptr_t)cap_dev % 8) return LOCMOE_ERR_ALIGN;
     return launch_capacity_route(*shape, idx, cos_sim, src_dev, *rule, delta_e, theta_e, cap_dev, C_alloc, pos, slot, drop,
-                                 inv, counts, kept, send_counts, load, locality, status, ws,
-                                 static_cast<cudaStream_t>(stream));
+                                 inv, counts, kept, send_counts, load, locality, status,
+                                 (flags & LOCMOE_ROUTE_EARLY_INIT) ? 1 : 0, ws, static_cast<cudaStream_t>(stream));
 }
 
 int locmoe_dispatch(const locmoe_shape_t* shape, int32_t C_alloc, const void* x, const int32_t* inv,
@@ -312,7 +313,8 @@ int locmoe_moe_layer(const locmoe_shape_t* shape, const void* x, const int32_t* 
     warn |= rc;
     rc = locmoe_capacity_route(shape, b->idx, b->cos_sim, src_dev, rule, b->delta_e, b->theta_e, b->cap_dev, C_alloc, b->pos,
                                b->slot, b->drop, b->inv, b->counts, b->kept, b->send_counts, b->load, b->locality, b->status,
-                               b->ws, b->ws_bytes, stream);
+                               LOCMOE_ROUTE_EARLY_INIT /* the kernel before it is this call's own gate */, b->ws,
+                               b->ws_bytes, stream);
     if (rc < 0) return rc;
     warn |= rc;
     rc = locmoe_dispatch(shape, C_alloc, x, b->inv, b->slot, b->buf, 1, stream);

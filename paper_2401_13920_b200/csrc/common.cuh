@@ -61,7 +61,7 @@ int launch_capacity_route(const locmoe_shape_t& s, const int32_t* idx, const flo
                           const locmoe_capacity_rule_t& rule, float* delta_e, float* theta_e, locmoe_capacity_t* cap_dev,
                           int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
                           int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
-                          void* ws, cudaStream_t st);
+                          int early_init, void* ws, cudaStream_t st);
 
 int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const int32_t* inv, const int32_t* slot,
                     void* buf, int zero_pad, cudaStream_t st);

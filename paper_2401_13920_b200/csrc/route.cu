@@ -83,8 +83,11 @@ __device__ __forceinline__ long long route_row_base(const RouteArgs& a, int k) {
     return (long long)e * a.D + dest_rank(b, s, a.N, a.Dn);
 }
 
-__global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a) {
-    pdl_wait();
+// early != 0: nothing this kernel writes is touched by the kernel queued before it (the caller says so), so the
+// fill runs while that kernel drains and the wait comes last -- it must still come, so that this kernel's
+// completion implies its predecessor's for the kernels after it.
+__global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a, int early) {
+    if (!early) pdl_wait();
     pdl_trigger();
     const long long stride = (long long)gridDim.x * blockDim.x;
     const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -98,6 +101,7 @@ __global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a)
     }
     if (i0 < 6) a.locality[i0] = 0ull;
     if (i0 == 0) *a.status = 0;
+    if (early) pdl_wait();
 }
 
 __global__ void __launch_bounds__(kThreads) route_hist0_kernel(const RouteArgs a) {
@@ -557,7 +561,7 @@ struct FusedCapacity {
 };
 
 static int launch_route_impl(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src, locmoe_capacity_t* cap_dev,
-                             const FusedCapacity* fuse, int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop,
+                             const FusedCapacity* fuse, int early_init, int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop,
                              int32_t* inv, int32_t* counts, int32_t* kept, int32_t* send_counts, int32_t* load,
                              int64_t* locality, int32_t* status, void* ws, cudaStream_t st) {
     RoutePlan p;
@@ -603,7 +607,7 @@ static int launch_route_impl(const locmoe_shape_t& s, const int32_t* idx, const 
     int init_blocks = (int)((init_items + kThreads * 4 - 1) / (kThreads * 4));
     if (init_blocks > 4 * sm_count()) init_blocks = 4 * sm_count();
     if (init_blocks < 1) init_blocks = 1;
-    if ((rc = launch_pdl(route_init_kernel, init_blocks, kThreads, 0, st, a))) return rc;
+    if ((rc = launch_pdl(route_init_kernel, init_blocks, kThreads, 0, st, a, early_init))) return rc;
 
     if ((rc = launch_pdl(route_hist0_kernel, p.ntiles, kThreads, (sizeof(int) << p.bits[0]) + cap_smem, st, a))) return rc;
 
@@ -634,7 +638,7 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
                  int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
                  int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
                  void* ws, cudaStream_t st) {
-    return launch_route_impl(s, idx, src, const_cast<locmoe_capacity_t*>(cap_dev), nullptr, C_alloc, pos, slot, drop, inv,
+    return launch_route_impl(s, idx, src, const_cast<locmoe_capacity_t*>(cap_dev), nullptr, 0, C_alloc, pos, slot, drop, inv,
                              counts, kept, send_counts, load, locality, status, ws, st);
 }
 
@@ -644,7 +648,7 @@ int launch_capacity_route(const locmoe_shape_t& s, const int32_t* idx, const flo
                           const locmoe_capacity_rule_t& rule, float* delta_e, float* theta_e, locmoe_capacity_t* cap_dev,
                           int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
                           int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
-                          void* ws, cudaStream_t st) {
+                          int early_init, void* ws, cudaStream_t st) {
     if (!capacity_route_fusable(s)) {
         int rc = launch_capacity(s, idx, cos_sim, rule, delta_e, theta_e, cap_dev, ws, st);
         if (rc) return rc;
@@ -652,7 +656,7 @@ int launch_capacity_route(const locmoe_shape_t& s, const int32_t* idx, const flo
                             status, ws, st);
     }
     const FusedCapacity f{cos_sim, rule, delta_e, theta_e};
-    return launch_route_impl(s, idx, src, cap_dev, &f, C_alloc, pos, slot, drop, inv, counts, kept, send_counts, load,
+    return launch_route_impl(s, idx, src, cap_dev, &f, early_init, C_alloc, pos, slot, drop, inv, counts, kept, send_counts, load,
                              locality, status, ws, st);
 }
 

@@ -78,7 +78,7 @@ def test_null_pointers_are_rejected_before_any_launch(B):
     assert lib.locmoe_capacity(C.byref(sh), None, None, C.byref(rule), None, None, None, None, 0, None) == -1
     assert lib.locmoe_route(C.byref(sh), None, None, None, 4, *([None] * 10), None, 0, None) == -1
     assert lib.locmoe_capacity_route(C.byref(sh), None, None, None, C.byref(rule), None, None, None, 4, *([None] * 10),
-                                     None, 0, None) == -1
+                                     0, None, 0, None) == -1
 
 
 def test_header_is_plain_c_and_links_from_a_c_program(tmp_path):
