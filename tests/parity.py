@@ -100,9 +100,26 @@ def check_capacity(shape, st, rule, gate_info):
     return cap, ref
 
 
-def check_route(shape, st, src, cap):
+def check_route(shape, st, src, cap, gate_info=None, ref_cap=None):
+    """Integer outputs of the route stage against the oracle's route.
+
+    The oracle's inputs come from the oracle's own chain: its arg-max indices (``gate_info``) and its capacity
+    (``ref_cap``, evaluated on its own fp64 cosines).  Two substitutions keep one stage's allowed freedom from
+    shifting every later queue position: at a token whose two best logits are within 1e-6 (check_gate has verified
+    that these are the only tokens where the indices differ, and that the GPU's pick is a maximiser within that gap)
+    the GPU's pick is used; and the integer capacity is the GPU's when the last bit of the fp32 cosine minimum moved
+    a ceiling (reported, never seen on the test workloads).  Without ``gate_info`` (callers that validated the
+    gate themselves) the indices under test are routed as they are."""
     idx_g = _np(st.idx)
-    ref = oracle.route(idx_g, _np(src), shape.E, shape.n_nodes, shape.dev_per_node, cap.C_local, st.C_alloc, shape.layout)
+    idx_in, C_local = idx_g, cap.C_local
+    if gate_info is not None:
+        idx_in = gate_info["idx_o"].copy()
+        flip = idx_in != idx_g
+        assert (gate_info["gap"][flip] < GAP_EXCUSE).all()
+        idx_in[flip] = idx_g[flip]
+    if ref_cap is not None and (ref_cap.C_local, ref_cap.C_expert) == (cap.C_local, cap.C_expert):
+        C_local = ref_cap.C_local
+    ref = oracle.route(idx_in, _np(src), shape.E, shape.n_nodes, shape.dev_per_node, C_local, st.C_alloc, shape.layout)
     for name in ("pos", "slot", "drop", "inv", "load"):
         got = _np(getattr(st, name))
         want = getattr(ref, name)
@@ -187,9 +204,11 @@ def run_staged(w: W.Workload, capacity_factor=1.0, min_mult=None, layout=B.LAYOU
     rep = {"workload": w.name, "T": w.T, "C_alloc": C_alloc}
     gi = check_gate(x, shape, st, eps_dev)
     rep.update(n_excused=gi["n_excused"], n_differ=gi["n_differ"], max_rel_R=gi["max_rel_R"])
-    cap, _ = check_capacity(shape, st, rule, gi)
+    cap, ref_cap = check_capacity(shape, st, rule, gi)
     rep.update(delta=cap.delta, ec_min=cap.ec_min, C_local=cap.C_local, C_expert=cap.C_expert)
-    rr = check_route(shape, st, src, cap)
+    rr = check_route(shape, st, src, cap, gi, ref_cap)
+    # True when every expected value below comes from the oracle's chain on the seeded inputs alone
+    rep["oracle_chain_only"] = (gi["n_differ"] == 0) and (ref_cap.C_local, ref_cap.C_expert) == (cap.C_local, cap.C_expert)
     rep.update(drop_frac=float(rr.drop.mean()), status=rr.status)
     ysrc = st.buf if y is None else y
     rng = np.random.default_rng(seed)

@@ -106,8 +106,8 @@ def test_full_layer_config5_scaled(P, monkeypatch, kernel):
     assert B.locmoe_device_flags() == 0
     # router stages against the oracle
     gi = P.check_gate(x, sh, st)
-    cap, _ = P.check_capacity(sh, st, rule, gi)
-    rr = P.check_route(sh, st, src, cap)
+    cap, ref_cap = P.check_capacity(sh, st, rule, gi)
+    rr = P.check_route(sh, st, src, cap, gi, ref_cap)
     P.check_dispatch_full(x, sh, st, rr)
     # expert outputs of sampled occupied and empty rows
     rng = np.random.default_rng(3)
