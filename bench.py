@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--variant", choices=["router", "peer8", "topk2"], default="router",
                     help="router: the metric's path; peer8: dispatch / combine through a table of eight receive buffers "
                          "(the fused-exchange kernels, all buffers on this GPU); topk2: the top-2 variant")
+    ap.add_argument("--fuse-gate", action="store_true",
+                    help="gate, capacity and route as the one call locmoe_gate_route (the gate's time is then part of that stage)")
     ap.add_argument("--unfused", action="store_true", help="capacity and route as two calls instead of locmoe_capacity_route")
     ap.add_argument("--no-ffn", action="store_true", help="config 5 only: identity experts instead of the expert FFN")
     ap.add_argument("--ffn-inner", type=int, default=10240, help="config 5: inner size F of the expert FFN")
@@ -263,8 +265,9 @@ def main():
 
     stream = torch.cuda.current_stream()
     fused = not args.unfused
-    stages = ["gate"] + (["capacity_route"] if fused else ["capacity", "route"]) + ["dispatch"] + \
-             (["ffn"] if use_ffn else []) + ["combine"]
+    fuse_gate = args.fuse_gate and variant == "router"
+    stages = (["gate_route"] if fuse_gate else ["gate"] + (["capacity_route"] if fused else ["capacity", "route"])) + \
+             ["dispatch"] + (["ffn"] if use_ffn else []) + ["combine"]
 
     tk = None
     if variant == "peer8":
@@ -306,9 +309,14 @@ def main():
             mark()
             return
         mark()
-        B.locmoe_gate(sh, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
-        mark()
-        if fused:
+        if fuse_gate:
+            B.locmoe_gate_route(sh, x, None, src, st.rule, st, stream)
+        else:
+            B.locmoe_gate(sh, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
+            mark()
+        if fuse_gate:
+            pass
+        elif fused:
             B.locmoe_capacity_route(sh, st.idx, st.cos_sim, src, st.rule, st.delta_e, st.theta_e, st.cap_dev, Ca, st.pos,
                                     st.slot, st.drop, st.inv, st.counts, st.kept, st.send_counts, st.load, st.locality,
                                     st.status, st.ws, stream, early_init=not ev)   # eager steps record an event in between
@@ -388,11 +396,15 @@ def main():
         "combine": kept * w.H * by + w.T * w.H * bx + 8 * w.T * (tk["K"] if tk is not None else 1),
     }
     peak, peak_kind = measured_peak()
+    if fuse_gate:   # the gate's bytes over the time of the whole gate + capacity + route chain
+        bytes_per_launch = {"gate_route": bytes_per_launch["gate"], "dispatch": bytes_per_launch["dispatch"],
+                            "combine": bytes_per_launch["combine"]}
+    hbm_stages = tuple(bytes_per_launch)
     kernels = {}
-    for s in ("gate", "dispatch", "combine"):
+    for s in hbm_stages:
         gbs = bytes_per_launch[s] / (stage_ms[s] * 1e-3) / 1e9
         kernels[s] = {"ms": stage_ms[s], "bytes": bytes_per_launch[s], "achieved_gbs": gbs, "frac": gbs / peak}
-    dominant = max(("gate", "dispatch", "combine"), key=lambda s: stage_ms[s])
+    dominant = max(hbm_stages, key=lambda s: stage_ms[s])
     traffic = ncu_traffic(dominant, w, args.cf, args.tokens) if variant == "router" else None
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["achieved_gbs"], "peak": peak,
                 "peak_kind": peak_kind + " (copy, MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
@@ -413,6 +425,8 @@ def main():
     if variant == "topk2":
         lv = B.locmoe_launch_counts(tk["shape_v"])
         launches = {"gate": 1, "capacity": launches["capacity"], "select": 1, "route": lv["route"] + 1, "dispatch": 1, "combine": 1}
+    elif fuse_gate:
+        launches = {"gate_route": launches["route"], "dispatch": launches["dispatch"], "combine": launches["combine"]}
     elif fused:
         # the capacity stage rides on the route stage's launches (up to 8192 experts)
         cr = launches.pop("route") + (launches["capacity"] if shape.E > 8192 else 0)

@@ -221,6 +221,27 @@ int locmoe_capacity_route(const locmoe_shape_t *shape, const int32_t *idx, const
                           int32_t *status, int32_t flags, void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * locmoe_gate, locmoe_capacity and locmoe_route as ONE call with the same
+ * inputs, outputs and results (probabilities are not available in this form).
+ * The route stage's fill kernel runs first; the gate kernel, as it finishes a
+ * token, also takes that token's share of the route stage's first pass (the
+ * demand count of its (source, expert) pair, the digit histogram of the first
+ * sorting pass, the minimum cosine of its expert) with integer atomics; the
+ * sorting passes follow, the first of them carrying the capacity rule.  Two
+ * launches and one pass over the index arrays less than the separate calls.
+ * flags: 0 or LOCMOE_ROUTE_EARLY_INIT, which here speaks about the kernel
+ * queued before THIS call (for instance the combine of the previous step):
+ * it touches none of this call's route outputs or workspace.
+ */
+int locmoe_gate_route(const locmoe_shape_t *shape, const void *x, const float *eps,
+                      const int32_t *src_dev, const locmoe_capacity_rule_t *rule, int32_t *idx,
+                      float *gate_w, float *cos_sim, float *delta_e, float *theta_e,
+                      locmoe_capacity_t *cap_dev, int32_t C_alloc, int32_t *pos, int32_t *slot,
+                      uint8_t *drop, int32_t *inv, int32_t *counts, int32_t *kept,
+                      int32_t *send_counts, int32_t *load, int64_t *locality, int32_t *status,
+                      int32_t flags, void *ws, size_t ws_bytes, void *stream);
+
+/*
  * Dispatch: buf[row][:] = x[inv[row]][:] bit for bit for occupied rows; rows
  * with inv < 0 are zero-filled when zero_pad != 0 and left untouched otherwise.
  * x [T][H], buf [D * E * C_alloc][H], both of shape->x_dtype.

@@ -24,7 +24,7 @@ WARN_CLAMPED, WARN_BAD_SRC, WARN_BAD_IDX = 1, 2, 4
 FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
-    "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route", "locmoe_capacity_route",
+    "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route", "locmoe_capacity_route", "locmoe_gate_route",
     "locmoe_dispatch", "locmoe_combine", "locmoe_dispatch_peer", "locmoe_combine_peer", "locmoe_topk_select", "locmoe_topk_fold", "locmoe_combine_topk", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
@@ -77,6 +77,8 @@ def _load() -> C.CDLL:
     lib.locmoe_route.argtypes = [C.POINTER(Shape), vp, vp, vp, i32] + [vp] * 10 + [vp, C.c_size_t, vp]
     lib.locmoe_capacity_route.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(CapacityRule), vp, vp, vp, i32] + [vp] * 10 + \
                                          [i32, vp, C.c_size_t, vp]
+    lib.locmoe_gate_route.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(CapacityRule)] + [vp] * 6 + [i32] + [vp] * 10 + \
+                                     [i32, vp, C.c_size_t, vp]
     lib.locmoe_dispatch.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, vp, i32, vp]
     lib.locmoe_combine.argtypes = [C.POINTER(Shape), i32, vp, i32, vp, vp, vp, i32, vp]
     lib.locmoe_expert_ffn.argtypes = [C.POINTER(Shape), i32, i32, vp, vp, vp, vp, vp, i32, vp]
@@ -251,6 +253,20 @@ def locmoe_capacity_route(shape: Shape, idx, cos_sim, src_dev, rule: CapacityRul
         int(C_alloc), _ptr(pos), _ptr(slot), _ptr(drop), _ptr(inv), _ptr(counts), _ptr(kept), _ptr(send_counts), _ptr(load),
         _ptr(locality), _ptr(status), ROUTE_EARLY_INIT if early_init else 0, _ptr(ws), ws.numel() * ws.element_size(),
         _stream(stream)))
+
+
+def locmoe_gate_route(shape: Shape, x, eps, src_dev, rule: CapacityRule, st: "RouterState", stream=None, early_init=False) -> int:
+    """Gate, capacity and route as one call chain on the tensors of a RouterState."""
+    dt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
+    _want(x, dt, shape.T * shape.H, "x")
+    _want(src_dev, torch.int32, shape.T, "src_dev")
+    if eps is not None:
+        _want(eps, torch.float32, shape.E, "eps")
+    return _check("locmoe_gate_route", _lib.locmoe_gate_route(
+        C.byref(shape), _ptr(x), _ptr(eps), _ptr(src_dev), C.byref(rule), _ptr(st.idx), _ptr(st.gate_w), _ptr(st.cos_sim),
+        _ptr(st.delta_e), _ptr(st.theta_e), _ptr(st.cap_dev), int(st.C_alloc), _ptr(st.pos), _ptr(st.slot), _ptr(st.drop),
+        _ptr(st.inv), _ptr(st.counts), _ptr(st.kept), _ptr(st.send_counts), _ptr(st.load), _ptr(st.locality), _ptr(st.status),
+        ROUTE_EARLY_INIT if early_init else 0, _ptr(st.ws), st.ws.numel() * st.ws.element_size(), _stream(stream)))
 
 
 def locmoe_dispatch(shape: Shape, C_alloc, x, inv, buf, zero_pad=True, stream=None, slot=None) -> int:
@@ -455,13 +471,19 @@ def router_forward(st: RouterState, x, src_dev, y=None, eps=None, stream=None, o
     """gate -> capacity -> route -> dispatch -> combine on one stream.
 
     ``y`` are the expert outputs in slot layout; with ``y=None`` the experts are
-    the identity and the dispatched buffer itself is combined.  ``fused`` runs the
-    capacity and route stages as the single call ``locmoe_capacity_route`` (same
-    results, one stage less in the launch chain).  Returns the combined output
+    the identity and the dispatched buffer itself is combined.  ``fused`` = True runs the
+    capacity and route stages as the single call ``locmoe_capacity_route``, "gate" runs
+    gate, capacity and route as ``locmoe_gate_route``, False the three separate calls
+    (same results).  Returns the combined output
     (``st.out`` unless ``out`` is given).
     """
     sh, Ca = st.shape, st.C_alloc
     out = st.out if out is None else out
+    if fused == "gate":
+        locmoe_gate_route(sh, x, eps, src_dev, st.rule, st, stream)
+        locmoe_dispatch(sh, Ca, x, st.inv, st.buf, True, stream, slot=st.slot)
+        locmoe_combine(sh, Ca, st.buf if y is None else y, st.slot, st.gate_w, out, False, stream)
+        return out
     locmoe_gate(sh, x, eps, st.idx, st.gate_w, st.cos_sim, None, stream)
     if fused:
         locmoe_capacity_route(sh, st.idx, st.cos_sim, src_dev, st.rule, st.delta_e, st.theta_e, st.cap_dev, Ca, st.pos,

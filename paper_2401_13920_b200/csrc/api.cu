@@ -152,6 +152,34 @@ int locmoe_capacity_route(const locmoe_shape_t* shape, const int32_t* idx, const
                                  (flags & LOCMOE_ROUTE_EARLY_INIT) ? 1 : 0, ws, static_cast<cudaStream_t>(stream));
 }
 
+int locmoe_gate_route(const locmoe_shape_t* shape, const void* x, const float* eps, const int32_t* src_dev,
+                      const locmoe_capacity_rule_t* rule, int32_t* idx, float* gate_w, float* cos_sim, float* delta_e,
+                      float* theta_e, locmoe_capacity_t* cap_dev, int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop,
+                      int32_t* inv, int32_t* counts, int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality,
+                      int32_t* status, int32_t flags, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!x || !src_dev || !rule || !idx || !gate_w || !cos_sim || !delta_e || !theta_e || !cap_dev || !pos || !slot || !drop ||
+        !inv || !counts || !kept || !send_counts || !load || !locality || !status)
+        return LOCMOE_ERR_NULL;
+    if (shape->H < 2) return LOCMOE_ERR_SHAPE;
+    const int esz = shape->x_dtype == LOCMOE_F32 ? 4 : 2;
+    if ((uintptr_t)x % esz) return LOCMOE_ERR_ALIGN;
+    if (rule->bound_form < LOCMOE_BOUND_BETA || rule->bound_form > LOCMOE_BOUND_EXP) return LOCMOE_ERR_DTYPE;
+    if (rule->T_global < 0) return LOCMOE_ERR_SHAPE;
+    if (!(rule->min_mult >= 0.0) || !(rule->capacity_factor >= 0.0) || rule->delta_override != rule->delta_override)
+        return LOCMOE_ERR_SHAPE;
+    if (buffer_rows(shape, C_alloc) < 0) return LOCMOE_ERR_SHAPE;
+    if (flags & ~LOCMOE_ROUTE_EARLY_INIT) return LOCMOE_ERR_DTYPE;
+    RoutePlan p;
+    if ((rc = plan_route(*shape, &p))) return rc;
+    if (!ws || ws_bytes < p.total || (uintptr_t)ws % 256) return LOCMOE_ERR_WORKSPACE;
+    if ((uintptr_t)locality % 8 || (uintptr_t)cap_dev % 8) return LOCMOE_ERR_ALIGN;
+    return launch_gate_route(*shape, x, eps, src_dev, *rule, idx, gate_w, cos_sim, delta_e, theta_e, cap_dev, C_alloc, pos, slot,
+                             drop, inv, counts, kept, send_counts, load, locality, status,
+                             (flags & LOCMOE_ROUTE_EARLY_INIT) ? 1 : 0, ws, static_cast<cudaStream_t>(stream));
+}
+
 int locmoe_dispatch(const locmoe_shape_t* shape, int32_t C_alloc, const void* x, const int32_t* inv,
                     const int32_t* slot, void* buf, int32_t zero_pad, void* stream) {
     int rc = check_shape(shape);
@@ -308,13 +336,9 @@ int locmoe_moe_layer(const locmoe_shape_t* shape, const void* x, const int32_t* 
                      const void* w_out, const locmoe_layer_buffers_t* b, void* out, void* stream) {
     if (!b) return LOCMOE_ERR_NULL;
     int warn = 0;
-    int rc = locmoe_gate(shape, x, eps, b->idx, b->gate_w, b->cos_sim, nullptr, stream);
-    if (rc < 0) return rc;
-    warn |= rc;
-    rc = locmoe_capacity_route(shape, b->idx, b->cos_sim, src_dev, rule, b->delta_e, b->theta_e, b->cap_dev, C_alloc, b->pos,
-                               b->slot, b->drop, b->inv, b->counts, b->kept, b->send_counts, b->load, b->locality, b->status,
-                               LOCMOE_ROUTE_EARLY_INIT /* the kernel before it is this call's own gate */, b->ws,
-                               b->ws_bytes, stream);
+    int rc = locmoe_gate_route(shape, x, eps, src_dev, rule, b->idx, b->gate_w, b->cos_sim, b->delta_e, b->theta_e, b->cap_dev,
+                               C_alloc, b->pos, b->slot, b->drop, b->inv, b->counts, b->kept, b->send_counts, b->load,
+                               b->locality, b->status, 0, b->ws, b->ws_bytes, stream);
     if (rc < 0) return rc;
     warn |= rc;
     rc = locmoe_dispatch(shape, C_alloc, x, b->inv, b->slot, b->buf, 1, stream);

@@ -28,8 +28,21 @@ inline int check_launch() {
 }
 
 // ---- launchers (each queues its kernels on `st` and returns a LOCMOE_* code) ----
+// What the gate also does per token when the route stage rides on it (locmoe_gate_route): the per-expert minimum
+// of the cosines, the per-key demand counts and the (digit, tile) histogram of the first radix pass, all by
+// integer atomics on arrays the route stage's fill kernel has initialised.  src == nullptr: nothing.
+struct GateFuse {
+    const int32_t* src;
+    int32_t* counts;      // [D * E]
+    int32_t* hist0;       // [1 << bits0][hstride]
+    uint32_t* cap_min;    // [min_sets][E] order-preserving codes, 0xffffffff = no token yet
+    int min_sets;         // a power of two
+    int32_t* pos; int32_t* slot; uint8_t* drop; int32_t* status;   // a token with an impossible source is dropped here
+    int D, digit_mask, hstride, tile_shift;
+};
+
 int launch_gate(const locmoe_shape_t& s, const void* x, const float* eps, int32_t* idx, float* gate_w,
-                float* cos_sim, float* probs, cudaStream_t st);
+                float* cos_sim, float* probs, cudaStream_t st, const GateFuse* fuse = nullptr);
 
 int launch_capacity(const locmoe_shape_t& s, const int32_t* idx, const float* cos_sim,
                     const locmoe_capacity_rule_t& rule, float* delta_e, float* theta_e,
@@ -62,6 +75,12 @@ int launch_capacity_route(const locmoe_shape_t& s, const int32_t* idx, const flo
                           int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
                           int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
                           int early_init, void* ws, cudaStream_t st);
+
+int launch_gate_route(const locmoe_shape_t& s, const void* x, const float* eps, const int32_t* src,
+                      const locmoe_capacity_rule_t& rule, int32_t* idx, float* gate_w, float* cos_sim, float* delta_e,
+                      float* theta_e, locmoe_capacity_t* cap_dev, int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop,
+                      int32_t* inv, int32_t* counts, int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality,
+                      int32_t* status, int early_init, void* ws, cudaStream_t st);
 
 int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const int32_t* inv, const int32_t* slot,
                     void* buf, int zero_pad, cudaStream_t st);

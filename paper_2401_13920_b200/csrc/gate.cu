@@ -11,6 +11,7 @@
 #include <math.h>
 #include <stdlib.h>
 
+#include "capacity_finish.cuh"
 #include "common.cuh"
 
 namespace locmoe {
@@ -33,7 +34,25 @@ struct GateArgs {
     int warp_floats;  // shared floats per warp
     int tab_ints;     // shared ints of the strip-offset table (one per unit of a row)
     float inv_g, sqrt_g;
+    GateFuse f;       // route-stage work carried by the gate (f.src == nullptr: none)
 };
+
+// Lane 0 of the warp that finished token `row`: the route stage's first pass over the tokens, done here.
+// sd = src[row], fetched by the caller (the specialised kernel prefetches it with the row).
+__device__ __forceinline__ void gate_route_hook(const GateArgs& a, int row, int bi, float cosv, int sd) {
+    if (!a.f.src) return;
+    // min_sets copies of the row of minima, chosen by the token index: 1 / min_sets of the same-address atomics
+    // (64 experts and 65536 tokens on one row cost 29 us of L2 atomic back-pressure)
+    atomicMin(&a.f.cap_min[(size_t)(row & (a.f.min_sets - 1)) * a.E + bi], order_code(cosv));
+    if ((unsigned)sd >= (unsigned)a.f.D) {
+        a.f.pos[row] = -1; a.f.slot[row] = -1; a.f.drop[row] = 1;
+        atomicOr(a.f.status, LOCMOE_WARN_BAD_SRC);
+        return;
+    }
+    const int key = sd * a.E + bi;
+    atomicAdd(&a.f.counts[key], 1);
+    atomicAdd(&a.f.hist0[(size_t)(key & a.f.digit_mask) * a.f.hstride + (row >> a.f.tile_shift)], 1);
+}
 
 // A 16-byte vector as NP packed pairs of floats (Blackwell has two-wide fp32 add / fma).
 template <int DT>
@@ -99,9 +118,11 @@ __device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gs
     }
     if (lane == 0) {
         float nrm = sqrtf(sq);
+        const float cosv = nrm > 0.0f ? gsum[bi] / (a.sqrt_g * nrm) : 0.0f;
         a.idx[row] = bi;
         a.gate_w[row] = R;
-        a.cos_sim[row] = nrm > 0.0f ? gsum[bi] / (a.sqrt_g * nrm) : 0.0f;
+        a.cos_sim[row] = cosv;
+        gate_route_hook(a, row, bi, cosv, a.f.src ? a.f.src[row] : 0);
     }
 }
 
@@ -264,11 +285,13 @@ __global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
 
     uint4 bufA[CH], bufB[CH];
     float2 sq2 = make_float2(0.0f, 0.0f);
+    int sd_cur = 0, sd_new = 0;   // source device of the row being reduced / of the row whose first chunk is in flight
 
     auto load = [&](uint4 (&buf)[CH], int r, int c) {
         const uint4* base = xv + (size_t)r * a.V + c * (CH * kWarp) + lane;
 #pragma unroll
         for (int k = 0; k < CH; ++k) buf[k] = ld_stream(base + k * kWarp);
+        if (c == 0 && a.f.src) sd_new = a.f.src[r];
     };
 
     auto consume = [&](const uint4 (&buf)[CH], int c) {
@@ -329,16 +352,20 @@ __global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
         const float wsum = __shfl_sync(full, cand, bi & 31);
         if (lane == 0) {
             const float nrm = sqrtf(sq);
+            const float cosv = nrm > 0.0f ? wsum / (a.sqrt_g * nrm) : 0.0f;
             a.idx[row] = bi;
             a.gate_w[row] = 1.0f / se;
-            a.cos_sim[row] = nrm > 0.0f ? wsum / (a.sqrt_g * nrm) : 0.0f;
+            a.cos_sim[row] = cosv;
+            gate_route_hook(a, row, bi, cosv, sd_cur);
         }
         sq2 = make_float2(0.0f, 0.0f);
+        sd_cur = sd_new;
     };
 
     int row = blockIdx.x * wpb + wib, ch = 0;
     if (row >= a.T) return;
     load(bufA, row, 0);
+    sd_cur = sd_new;
     while (true) {
         int ch2 = ch + 1, row2 = row;
         if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
@@ -421,8 +448,9 @@ int launch_persistent(K kernel, const GateArgs& a, int max_warps, cudaStream_t s
 }  // namespace
 
 int launch_gate(const locmoe_shape_t& s, const void* x, const float* eps, int32_t* idx, float* gate_w,
-                float* cos_sim, float* probs, cudaStream_t st) {
+                float* cos_sim, float* probs, cudaStream_t st, const GateFuse* fuse) {
     GateArgs a{};
+    if (fuse) a.f = *fuse;
     a.x = x; a.eps = eps; a.idx = idx; a.gate_w = gate_w; a.cos_sim = cos_sim; a.probs = probs;
     a.T = s.T; a.H = s.H; a.E = s.E; a.g = s.H / s.E;
     a.inv_g = 1.0f / (float)a.g;

@@ -60,6 +60,8 @@ struct RouteArgs {
     // capacity carried along (the fused call): hist0 also takes the per-expert minima of the cosines per tile,
     // an extra CTA of the first scatter combines them and writes the capacity record the last scatter reads
     int fuse_cap, H;
+    int hist_by_gate;           // the gate kernel has already taken hist[0], counts and the minima
+    int cap_sets;               // rows of cap_part: tiles (hist0 took the minima) or the gate's replica count
     double lnbeta;              // ln B(1/2, (H-1)/2), from the host
     const float* cos;
     uint32_t* cap_part;         // [ntiles][E] order-preserving codes
@@ -95,10 +97,12 @@ __global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a,
     for (long long i = i0; i < a.K; i += stride) a.counts[i] = 0;
     for (long long i = i0; i < (long long)a.D * a.D; i += stride) a.send_counts[i] = 0;
     for (long long i = i0; i < a.E; i += stride) a.load[i] = 0;
-    for (int p = 1; p < a.passes; ++p) {
+    for (int p = a.hist_by_gate ? 0 : 1; p < a.passes; ++p) {
         const long long n = ((long long)a.hstride) << a.bits[p];
         for (long long i = i0; i < n; i += stride) a.hist[p][i] = 0;
     }
+    if (a.hist_by_gate)
+        for (long long i = i0; i < (long long)a.cap_sets * a.E; i += stride) a.cap_part[i] = 0xffffffffu;
     if (i0 < 6) a.locality[i0] = 0ull;
     if (i0 == 0) *a.status = 0;
     if (early) pdl_wait();
@@ -200,12 +204,16 @@ __device__ void route_extras_a(const RouteArgs& a, int x, int nx, int* dyn) {
     }
     if (a.fuse_cap && x == nx - 1) {
         __shared__ FinishShared fs;
+        if (a.cap_sets == 1) {   // one row of minima, taken by the gate kernel with global atomics
+            capacity_finish<true>(fs, a.cap_part, 1, a.T, a.E, a.H, a.D, a.lnbeta, a.rule, a.delta_e, a.theta_e, a.cap_out);
+            return;
+        }
         uint32_t* comb = reinterpret_cast<uint32_t*>(dyn);
         for (int e = threadIdx.x; e < a.E; e += kThreads) comb[e] = 0xffffffffu;
         __syncthreads();
         constexpr int kWorkers = kThreads, kU = 8;
         {
-            const long long n = (long long)a.ntiles * a.E;
+            const long long n = (long long)a.cap_sets * a.E;
             for (long long i0 = threadIdx.x; i0 < n; i0 += (long long)kU * kWorkers) {
                 uint32_t c[kU];
 #pragma unroll
@@ -540,7 +548,7 @@ int plan_route(const locmoe_shape_t& s, RoutePlan* p) {
     p->off_keystart = off; off += align256((size_t)K * 4);
     p->off_rowbase = off; off += align256((size_t)K * 4);
     p->off_rowtot = off; off += 1024;
-    p->off_cap_part = off; off += align256((size_t)p->ntiles * s.E * 4);
+    p->off_cap_part = off; off += align256((size_t)(p->ntiles > 64 ? p->ntiles : 64) * s.E * 4);
     p->total = off;
     p->prescan = ((long long)p->ntiles << p->bits[0]) > 32768 ? 1 : 0;
     {   // testing aid: LOCMOE_PATH=grid forces the large-batch variants at any size
@@ -559,9 +567,17 @@ struct FusedCapacity {
     float* delta_e;
     float* theta_e;
 };
+// The gate of the same step, when it carries the route stage's first pass (locmoe_gate_route).
+struct FusedGate {
+    const void* x;
+    const float* eps;
+    int32_t* idx;
+    float* gate_w;
+    float* cos_sim;
+};
 
 static int launch_route_impl(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src, locmoe_capacity_t* cap_dev,
-                             const FusedCapacity* fuse, int early_init, int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop,
+                             const FusedCapacity* fuse, const FusedGate* gate, int early_init, int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop,
                              int32_t* inv, int32_t* counts, int32_t* kept, int32_t* send_counts, int32_t* load,
                              int64_t* locality, int32_t* status, void* ws, cudaStream_t st) {
     RoutePlan p;
@@ -594,6 +610,12 @@ static int launch_route_impl(const locmoe_shape_t& s, const int32_t* idx, const 
     a.rowtot = reinterpret_cast<int32_t*>(w + p.off_rowtot);
     a.prescan = p.prescan;
     a.fuse_cap = fuse ? 1 : 0;
+    a.hist_by_gate = gate ? 1 : 0;
+    a.cap_sets = p.ntiles;
+    if (gate) {   // replicas of the row of minima: as many as keep sets * E within 8192 words, at most 64
+        a.cap_sets = 1;
+        while (a.cap_sets < 64 && (long long)a.cap_sets * 2 * s.E <= 8192) a.cap_sets *= 2;
+    }
     a.H = s.H;
     if (fuse) {
         a.cos = fuse->cos_sim; a.rule = fuse->rule; a.delta_e = fuse->delta_e; a.theta_e = fuse->theta_e;
@@ -601,7 +623,8 @@ static int launch_route_impl(const locmoe_shape_t& s, const int32_t* idx, const 
         a.lnbeta = ln_beta_half(s.H);
         a.cap_part = reinterpret_cast<uint32_t*>(w + p.off_cap_part);
     }
-    const size_t cap_smem = fuse ? (size_t)s.E * sizeof(uint32_t) : 0;
+    const size_t hist_smem = (fuse && !gate) ? (size_t)s.E * sizeof(uint32_t) : 0;           // hist0's minima of its tile
+    const size_t cap_smem = (fuse && a.cap_sets > 1) ? (size_t)s.E * sizeof(uint32_t) : 0;   // the row of combined minima
 
     long long init_items = a.rows > a.K ? a.rows : a.K;
     int init_blocks = (int)((init_items + kThreads * 4 - 1) / (kThreads * 4));
@@ -609,7 +632,15 @@ static int launch_route_impl(const locmoe_shape_t& s, const int32_t* idx, const 
     if (init_blocks < 1) init_blocks = 1;
     if ((rc = launch_pdl(route_init_kernel, init_blocks, kThreads, 0, st, a, early_init))) return rc;
 
-    if ((rc = launch_pdl(route_hist0_kernel, p.ntiles, kThreads, (sizeof(int) << p.bits[0]) + cap_smem, st, a))) return rc;
+    if (gate) {
+        GateFuse gf{};
+        gf.src = src; gf.counts = counts; gf.hist0 = a.hist[0]; gf.cap_min = a.cap_part; gf.min_sets = a.cap_sets;
+        gf.pos = pos; gf.slot = slot; gf.drop = drop; gf.status = status;
+        gf.D = a.D; gf.digit_mask = (1 << p.bits[0]) - 1; gf.hstride = a.hstride; gf.tile_shift = a.tile_shift;
+        if ((rc = launch_gate(s, gate->x, gate->eps, gate->idx, gate->gate_w, gate->cos_sim, nullptr, st, &gf))) return rc;
+    } else if ((rc = launch_pdl(route_hist0_kernel, p.ntiles, kThreads, (sizeof(int) << p.bits[0]) + hist_smem, st, a))) {
+        return rc;
+    }
 
     int per_key = (a.K + kThreads * 4 - 1) / (kThreads * 4);   // CTAs that walk the K key classes
     if (per_key > 32) per_key = 32;
@@ -638,7 +669,7 @@ int launch_route(const locmoe_shape_t& s, const int32_t* idx, const int32_t* src
                  int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop, int32_t* inv, int32_t* counts,
                  int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality, int32_t* status,
                  void* ws, cudaStream_t st) {
-    return launch_route_impl(s, idx, src, const_cast<locmoe_capacity_t*>(cap_dev), nullptr, 0, C_alloc, pos, slot, drop, inv,
+    return launch_route_impl(s, idx, src, const_cast<locmoe_capacity_t*>(cap_dev), nullptr, nullptr, 0, C_alloc, pos, slot, drop, inv,
                              counts, kept, send_counts, load, locality, status, ws, st);
 }
 
@@ -656,8 +687,21 @@ int launch_capacity_route(const locmoe_shape_t& s, const int32_t* idx, const flo
                             status, ws, st);
     }
     const FusedCapacity f{cos_sim, rule, delta_e, theta_e};
-    return launch_route_impl(s, idx, src, cap_dev, &f, early_init, C_alloc, pos, slot, drop, inv, counts, kept, send_counts, load,
-                             locality, status, ws, st);
+    return launch_route_impl(s, idx, src, cap_dev, &f, nullptr, early_init, C_alloc, pos, slot, drop, inv, counts, kept, send_counts,
+                             load, locality, status, ws, st);
+}
+
+// Gate, capacity and route as one chain: fill -> gate (which also takes the route stage's first pass over the
+// tokens and the cosine minima) -> scatter passes.  Any number of experts (the minima live in global memory).
+int launch_gate_route(const locmoe_shape_t& s, const void* x, const float* eps, const int32_t* src,
+                      const locmoe_capacity_rule_t& rule, int32_t* idx, float* gate_w, float* cos_sim, float* delta_e,
+                      float* theta_e, locmoe_capacity_t* cap_dev, int32_t C_alloc, int32_t* pos, int32_t* slot, uint8_t* drop,
+                      int32_t* inv, int32_t* counts, int32_t* kept, int32_t* send_counts, int32_t* load, int64_t* locality,
+                      int32_t* status, int early_init, void* ws, cudaStream_t st) {
+    const FusedCapacity f{cos_sim, rule, delta_e, theta_e};
+    const FusedGate g{x, eps, idx, gate_w, cos_sim};
+    return launch_route_impl(s, idx, src, cap_dev, &f, &g, early_init, C_alloc, pos, slot, drop, inv, counts, kept, send_counts,
+                             load, locality, status, ws, st);
 }
 
 }  // namespace locmoe

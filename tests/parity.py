@@ -184,7 +184,8 @@ def check_combine_sampled(y, shape, st, ref_route, gate_info, tokens_sample):
 def run_staged(w: W.Workload, capacity_factor=1.0, min_mult=None, layout=B.LAYOUT_SEND, delta_override=-1.0,
                bound_form=B.BOUND_BETA, C_alloc=None, full=True, n_sample=512, y_random=False, eps=None, seed=0,
                fused=True):
-    """Runs the five calls on the workload and compares every stage; returns a small report."""
+    """Runs the path on the workload (``fused``: "gate" = locmoe_gate_route, True = gate + locmoe_capacity_route, False =
+    the separate calls) and compares every stage; returns a small report."""
     dev = torch.device("cuda:0")
     x = W.make_tokens(w, dev)
     src = W.make_src(w, dev)

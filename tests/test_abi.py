@@ -76,6 +76,7 @@ def test_null_pointers_are_rejected_before_any_launch(B):
     assert lib.locmoe_cos_hist(C.byref(sh), None, None, 0, 1, 8, -1.0, 1.0, None, None, None, None) == -1
     rule = B.CapacityRule(1.0, 1.0, -1.0, 0, 0)
     assert lib.locmoe_capacity(C.byref(sh), None, None, C.byref(rule), None, None, None, None, 0, None) == -1
+    assert lib.locmoe_gate_route(C.byref(sh), None, None, None, C.byref(rule), *([None] * 6), 4, *([None] * 10), 0, None, 0, None) == -1
     assert lib.locmoe_route(C.byref(sh), None, None, None, 4, *([None] * 10), None, 0, None) == -1
     assert lib.locmoe_capacity_route(C.byref(sh), None, None, None, C.byref(rule), None, None, None, 4, *([None] * 10),
                                      0, None, 0, None) == -1

@@ -116,6 +116,64 @@ def test_warp_per_row_dispatch_variant(P, monkeypatch):
     P.run_staged(P.W.CONFIGS[1], 1.0, layout=1, full=True)
 
 
+# ---- gate, capacity and route as ONE call chain (the gate kernel takes the route stage's first pass) ----
+
+@pytest.mark.parametrize("cfg,T", [(1, 4096), (2, 6000), (3, 8229), (4, 5003), (5, 7001)])
+@pytest.mark.parametrize("layout", [0, 1])
+def test_gate_route_call_configs(P, cfg, T, layout):
+    rep = P.run_staged(P.W.CONFIGS[cfg].scaled(T), 1.0, layout=layout, full=True, y_random=cfg == 4, fused="gate")
+    assert rep["status"] == 0
+
+
+@pytest.mark.parametrize("kw", [
+    dict(T=1, H=64, E=4, n_nodes=1, dev_per_node=2),
+    dict(T=31, H=64, E=1, n_nodes=1, dev_per_node=1),
+    dict(T=777, H=60, E=4, n_nodes=1, dev_per_node=4, dtype="f32"),     # general vector gate kernel
+    dict(T=777, H=36, E=4, n_nodes=2, dev_per_node=2),                  # scalar gate kernel
+    dict(T=513, H=1024, E=512, n_nodes=4, dev_per_node=8),
+    dict(T=3000, H=4096, E=2048, n_nodes=1, dev_per_node=1),
+    dict(T=4097, H=2048, E=2048, n_nodes=8, dev_per_node=8),            # three radix passes
+    dict(T=300, H=16384, E=16384, n_nodes=1, dev_per_node=1),           # > 8192 experts
+])
+def test_gate_route_call_shapes(P, kw):
+    P.run_staged(_wl(P, **kw), 1.0, layout=1, full=True, fused="gate")
+
+
+def test_gate_route_call_grid_path_and_full_size(P, monkeypatch):
+    rep = P.run_staged(P.W.CONFIGS[2], 1.0, full=False, n_sample=512, fused="gate")
+    assert rep["C_local"] == 16
+    rep = P.run_staged(P.W.CONFIGS[3], 1.0, full=False, n_sample=512, fused="gate")
+    assert rep["drop_frac"] > 0.3
+    monkeypatch.setenv("LOCMOE_PATH", "grid")
+    P.run_staged(P.W.CONFIGS[2].scaled(70001), 1.0, full=True, fused="gate")
+
+
+def test_gate_route_call_with_bias_bad_sources_and_clamp(P):
+    import numpy as np
+    W, B = P.W, P.B
+    w = _wl(P, T=2000, H=512, E=16, n_nodes=2, dev_per_node=4)
+    P.run_staged(w, 1.0, eps=np.linspace(-0.05, 0.05, 16).astype(np.float32), full=True, fused="gate")
+    rep = P.run_staged(P.W.CONFIGS[1], 2.0, C_alloc=40, full=True, fused="gate")
+    assert rep["status"] & 1
+    # a token with an impossible source device is dropped and flagged by the gate kernel's hook
+    dev = torch.device("cuda:0")
+    x, src = W.make_tokens(w, dev), W.make_src(w, dev).clone()
+    src[5] = 99
+    src[700] = -3
+    sh = B.make_shape(w.T, w.H, w.E, 2, 4, x.dtype)
+    st = B.make_router(sh, 20, B.CapacityRule(1.0, 1.0, -1.0, 0, 0), dev)
+    B.router_forward(st, x, src, fused="gate")
+    torch.cuda.synchronize()
+    ref = B.make_router(sh, 20, B.CapacityRule(1.0, 1.0, -1.0, 0, 0), dev)
+    B.router_forward(ref, x, src, fused=False)
+    torch.cuda.synchronize()
+    assert st.status.item() == ref.status.item() == 2
+    for name in ("pos", "slot", "drop", "inv", "counts", "kept", "send_counts", "load", "locality", "idx"):
+        assert torch.equal(getattr(st, name), getattr(ref, name)), name
+    assert torch.equal(st.out.view(torch.int16), ref.out.view(torch.int16))
+    assert st.slot[5].item() == -1 and st.slot[700].item() == -1
+
+
 # ---- capacity and route as two separate calls (the default path runs them as the one fused call) ----
 
 @pytest.mark.parametrize("cfg,T", [(1, 4096), (2, 6000), (3, 8229), (4, 5003), (5, 7001)])
