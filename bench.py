@@ -28,6 +28,7 @@ if ROOT not in sys.path:
 METRIC = "routed tokens/sec (gate+dispatch+combine) and achieved HBM GB/s vs B200 peak, 1 GPU"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0     # the nominal HBM3e figure the 70 % target is stated against
 
 
 def parse_args():
@@ -42,7 +43,11 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=48, help="end-to-end steps (the three-stream pipeline needs a few steps to fill)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
-    ap.add_argument("--event-every", type=int, default=8, help="carry per-stage CUDA events on every n-th timed step")
+    ap.add_argument("--stage-steps", type=int, default=24,
+                    help="eager steps with per-stage CUDA events after the timed region (median per stage; at least 20)")
+    ap.add_argument("--other-steps", type=int, default=20, help="timed steps of each of the other configurations")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the short runs of configurations 1, 3, 4 and 5 that the default line carries")
     ap.add_argument("--variant", choices=["router", "peer8", "topk2"], default="router",
                     help="router: the metric's path; peer8: dispatch / combine through a table of eight receive buffers "
                          "(the fused-exchange kernels, all buffers on this GPU); topk2: the top-2 variant")
@@ -70,6 +75,15 @@ def measured_tensor_peak():
             return float(json.load(f)["bf16_tflops_sustained"]), "measured (cuBLAS bf16 sustained, MEASURED_PEAKS.json)"
     except Exception:
         return 1400.0, "fallback"
+
+
+def measured_tensor_burst():
+    """cuBLAS bf16 rate of a kernel timed alone (burst), for context beside the sustained figure."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops"])
+    except Exception:
+        return 1590.0
 
 
 class ClockSampler(threading.Thread):
@@ -185,7 +199,7 @@ def run_reference(args):
         "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic", "impl": "reference",
-        "config": {**workload_config(w, args), "sample_tokens_per_step": n},
+        "config": workload_config(w, args), "sample_tokens_per_step": n,
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "host_cores": os.cpu_count(),
@@ -209,43 +223,27 @@ def workload_config(w, args, n_tokens=None):
     }
 
 
-def main():
-    args = parse_args()
-    if args.impl == "reference":
-        return run_reference(args)
+def median(v):
+    s = sorted(v)
+    n = len(s)
+    return float(s[n // 2] if n % 2 else 0.5 * (s[n // 2 - 1] + s[n // 2]))
 
+
+def measure(args, w, env, *, steps, warmup, stage_steps, use_ffn, variant, fuse_gate, fused, e2e_steps, cpu_baseline_s):
+    """Builds the workload on the device, times K steps of the whole path (CUDA events on the launching stream,
+    barrier + synchronize on both sides, max over ranks), then takes per-stage times from a separate pass of eager
+    steps with events between the stages (median).  Returns the pieces of the JSON line."""
     import numpy as np
     import torch
-    from paper_2401_13920_b200 import binding as B   # raises if the CUDA library cannot be built / loaded
+    from paper_2401_13920_b200 import binding as B
     from paper_2401_13920_b200 import sharding
     from paper_2401_13920_b200 import workloads as W
 
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=dev)
-
-    w = W.CONFIGS[args.config]
-    if args.tokens > 0:
-        w = w.scaled(args.tokens)
-    if world > 1:
-        # every rank routes its own batch: same shape, its own seed
-        w = W.Workload(**{**w.__dict__, "config": w.config + 10 * rank, "name": w.name})
-    use_ffn = (w.config % 10) == 5 and not args.no_ffn
-    variant = args.variant
-    if variant != "router":
-        use_ffn = False
+    dev, dist, world, rank, local_rank = env["dev"], env["dist"], env["world"], env["rank"], env["local_rank"]
+    layout_name = args.layout
     if use_ffn or variant == "peer8":
-        args.layout = "recv"      # the expert FFN and the peer kernels work on the receive-side layout
-    layout = B.LAYOUT_SEND if args.layout == "send" else B.LAYOUT_RECV
+        layout_name = "recv"      # the expert FFN and the peer kernels work on the receive-side layout
+    layout = B.LAYOUT_SEND if layout_name == "send" else B.LAYOUT_RECV
     x = W.make_tokens(w, dev)
     src = W.make_src(w, dev)
     shape = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, layout)
@@ -264,8 +262,6 @@ def main():
     ysrc = st.buf if y is None else y
 
     stream = torch.cuda.current_stream()
-    fused = not args.unfused
-    fuse_gate = args.fuse_gate and variant == "router"
     stages = (["gate_route"] if fuse_gate else ["gate"] + (["capacity_route"] if fused else ["capacity", "route"])) + \
              ["dispatch"] + (["ffn"] if use_ffn else []) + ["combine"]
 
@@ -339,15 +335,13 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    warmup = max(warmup, 3)
+    for _ in range(warmup):
         step()
     barrier()
 
-    # ---- timed region: exactly K steps, device-timed.  The step is captured once in a CUDA graph and replayed;
-    #      every EV-th step is launched eagerly instead, with CUDA events between its stages on the launching
-    #      stream (an event record costs ~2.5 us of stream time, so only a sample of the steps carries them) ----
-    K = args.steps
-    EV = max(1, args.event_every)
+    # ---- timed region: exactly K steps, device-timed; the step is captured once in a CUDA graph and replayed ----
+    K = steps
     graph = None
     if not args.no_graph:
         side = torch.cuda.Stream(dev)
@@ -363,27 +357,39 @@ def main():
             stream = stream_backup
         torch.cuda.current_stream().wait_stream(side)
         graph.replay()
-    n_ev = (K + EV - 1) // EV
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(n_ev)]
-    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler = ClockSampler(physical_gpu_index(local_rank), period_s=0.001)
     sampler.start()
     barrier()
     t_start = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     t_start.record(stream)
     for k in range(K):
-        if k % EV == 0 or graph is None:
-            step(evs[k // EV] if k % EV == 0 else None)
+        if graph is None:
+            step()
         else:
             graph.replay()
     t_end.record(stream)
     barrier()
-    clocks = sampler.stop()
+    n_timed = len(sampler.samples)
     total_ms = sharding.max_over_ranks(t_start.elapsed_time(t_end), dev)
     ms_per_step = total_ms / K
     value = world * w.T * K / (total_ms * 1e-3)
 
-    stage_ms = {s: float(np.mean([evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(n_ev)])) for i, s in enumerate(stages)}
+    # ---- per-stage times: a separate pass of eager steps with CUDA events between the stages on the launching
+    #      stream (an event record costs ~2.5 us of stream time, so the timed region above carries none); medians ----
+    S = max(int(stage_steps), 20)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(S)]
+    for k in range(S):
+        step(evs[k])
+    barrier()
+    clocks = sampler.stop()
+    clocks["samples_in_timed_region"] = n_timed
+    clocks["covers"] = "timed region and per-stage pass"
+    stage_ms = {s: median([evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(S)]) for i, s in enumerate(stages)}
+    flags = B.locmoe_device_flags()
+    if flags != 0:
+        raise RuntimeError("a kernel gave up a bounded wait during the bench (device flags %d): the timing is void" % flags)
+
     # ---- algorithmic bytes per launch (per token: see the per-kernel byte model in the design notes) ----
     slot_t = tk["slot"] if tk is not None else st.slot
     kept = int((slot_t >= 0).sum().item())            # kept assignments (tokens, or token-choice pairs for top-k)
@@ -403,23 +409,34 @@ def main():
     kernels = {}
     for s in hbm_stages:
         gbs = bytes_per_launch[s] / (stage_ms[s] * 1e-3) / 1e9
-        kernels[s] = {"ms": stage_ms[s], "bytes": bytes_per_launch[s], "achieved_gbs": gbs, "frac": gbs / peak}
+        kernels[s] = {"ms": stage_ms[s], "bytes": bytes_per_launch[s], "achieved_gbs": gbs, "frac": gbs / peak,
+                      "frac_nominal": gbs / NOMINAL_HBM_GBS}
     dominant = max(hbm_stages, key=lambda s: stage_ms[s])
     traffic = ncu_traffic(dominant, w, args.cf, args.tokens) if variant == "router" else None
+    path_bytes = sum(bytes_per_launch.values())
+    path_gbs = path_bytes / (ms_per_step * 1e-3) / 1e9
+    if use_ffn:     # the router path's bytes over the time of its own stages (the tensor-bound stage left out)
+        hbm_ms = sum(v for k, v in stage_ms.items() if k != "ffn")
+        path_gbs = path_bytes / (hbm_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["achieved_gbs"], "peak": peak,
                 "peak_kind": peak_kind + " (copy, MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
-                "unit": "GB/s", "frac": kernels[dominant]["frac"], "traffic": traffic,
-                "path_bytes": sum(bytes_per_launch.values()),
-                "path_frac": sum(bytes_per_launch.values()) / (ms_per_step * 1e-3) / 1e9 / peak,
-                "kernels": kernels, "stage_ms": stage_ms}
+                "unit": "GB/s", "frac": kernels[dominant]["frac"], "frac_nominal": kernels[dominant]["frac_nominal"],
+                "nominal_peak": NOMINAL_HBM_GBS, "traffic": traffic,
+                "traffic_source": None if traffic is None else
+                "ncu capture of this workload and launch configuration summarised in profiles/dram_traffic_config2.md; "
+                "not measured in this run",
+                "path_bytes": path_bytes, "path_frac": path_gbs / peak, "path_frac_nominal": path_gbs / NOMINAL_HBM_GBS,
+                "kernels": kernels, "stage_ms": stage_ms,
+                "stage_ms_how": "median of %d eager steps after the timed region, CUDA events between the stages" % S}
     if use_ffn:
         # the expert FFN dominates: two grouped GEMMs, 2 * 2 * rows * H * F flops, tensor-core bound
         flops = 4.0 * rows * w.H * F
         tf = flops / (stage_ms["ffn"] * 1e-3) / 1e12
         tpeak, tkind = measured_tensor_peak()
         roofline.update({"bound": "tensor", "kernel": "ffn_gemm_kernel (two launches)", "achieved": tf, "peak": tpeak,
-                         "peak_kind": tkind, "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None, "flops": flops,
-                         "hbm_kernels": kernels})
+                         "peak_kind": tkind, "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None, "traffic_source": None,
+                         "flops": flops, "frac_of_burst_peak": tf / measured_tensor_burst(), "hbm_kernels": kernels})
+        roofline.pop("frac_nominal", None)
 
     launches = B.locmoe_launch_counts(shape)
     if variant == "topk2":
@@ -434,12 +451,11 @@ def main():
         launches = {"gate": launches["gate"], "capacity_route": cr, "dispatch": launches["dispatch"], "combine": launches["combine"]}
     if use_ffn:
         launches["ffn"] = 2
-    launches_per_step = sum(launches.values())
     cap = B.locmoe_capacity_read(tk["cap_dev"] if tk is not None else st.cap_dev)
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
     e2e = None
-    if args.e2e_steps > 0 and not use_ffn and variant == "router":
+    if e2e_steps > 0 and not use_ffn and variant == "router":
         xh = torch.empty(x.shape, dtype=x.dtype, pin_memory=True)
         xh.copy_(x)
         srch = torch.empty(src.shape, dtype=src.dtype, pin_memory=True)
@@ -453,7 +469,7 @@ def main():
         a = torch.cuda.Event(enable_timing=True)
         b = torch.cuda.Event(enable_timing=True)
         a.record(hr.s_in)
-        for i in range(args.e2e_steps):
+        for i in range(e2e_steps):
             hr.forward(xh, srch, outh[i & 1], y=y)
         hr.s_out.wait_stream(hr.s_comp)
         hr.s_out.wait_stream(hr.s_in)
@@ -461,15 +477,16 @@ def main():
         hr.synchronize()
         barrier()
         ems = sharding.max_over_ranks(a.elapsed_time(b), dev)
-        e2e = {"value": world * w.T * args.e2e_steps / (ems * 1e-3), "unit": UNIT,
+        e2e = {"value": world * w.T * e2e_steps / (ems * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": xh.numel() * xh.element_size() + srch.numel() * 4,
-               "d2h_bytes_per_step": outh[0].numel() * outh[0].element_size(), "steps": args.e2e_steps,
+               "d2h_bytes_per_step": outh[0].numel() * outh[0].element_size(), "steps": e2e_steps,
                "api": "binding.HostRouter.forward on pinned host tensors (copy in, five C-ABI calls, copy out; "
                       "successive steps pipelined over three streams)"}
+        del hr, xh, outh
 
     # ---- CPU baseline: the oracle, as it stands, on the host cores (rank 0, N = 1 only) ----
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and cpu_baseline_s > 0:
         import oracle
         oracle.build()
         n = min(w.T, 65536)
@@ -481,23 +498,110 @@ def main():
             oracle_step(oracle, xs, ss, shape.x_dtype, sub, args.cf, layout)
             reps += 1
             dt = time.perf_counter() - t0
-            if dt >= 10.0 or reps >= 64:
+            if dt >= cpu_baseline_s or reps >= 64:
                 break
         cpu_baseline = {"value": n * reps / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
                         "sample": "first %d tokens of the workload, whole path %d times, single thread, gcc -O2 "
                                   "(host has %d cores)" % (n, reps, os.cpu_count())}
 
+    args_l = argparse.Namespace(**{**vars(args), "layout": layout_name, "no_ffn": not use_ffn, "variant": variant})
+    return {
+        "value": value, "ms_per_step": ms_per_step, "steps": K, "warmup": warmup, "config": workload_config(w, args_l),
+        "clocks": clocks, "e2e": e2e, "launches": launches, "graph": graph is not None,
+        "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "routing": {"kept_fraction": kept / w.T, "C_local": cap.C_local, "C_expert": cap.C_expert, "delta": cap.delta,
+                    "ec_min": cap.ec_min, "rows": rows, "kept_tokens_per_s": value * kept / w.T},
+    }
+
+
+def summary_of(m):
+    """Short record of one configuration for the `other_configs` object of the JSON line."""
+    r = m["roofline"]
+    ks = r.get("hbm_kernels", r["kernels"])
+    out = {
+        "workload": m["config"]["workload"], "expert_ffn": m["config"]["expert_ffn"], "steps": m["steps"], "warmup": m["warmup"],
+        "ms_per_step": m["ms_per_step"], "tokens_per_s": m["value"],
+        "kernels": {k: {"ms": v["ms"], "achieved_gbs": v["achieved_gbs"], "frac": v["frac"], "frac_nominal": v["frac_nominal"]}
+                    for k, v in ks.items()},
+        "stage_ms": r["stage_ms"], "path_frac": r["path_frac"], "path_frac_nominal": r["path_frac_nominal"],
+        "kept_fraction": m["routing"]["kept_fraction"], "C_local": m["routing"]["C_local"],
+        "clocks": {k: m["clocks"][k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples")},
+        "launches_per_step": sum(m["launches"].values()),
+    }
+    if m["config"]["expert_ffn"]:
+        out["ffn"] = {"ms": r["stage_ms"]["ffn"], "tflops": r["achieved"], "frac_of_sustained_peak": r["frac"],
+                      "frac_of_burst_peak": r["frac_of_burst_peak"], "peak_sustained": r["peak"]}
+    return out
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import gc
+    import torch
+    from paper_2401_13920_b200 import binding as B   # raises if the CUDA library cannot be built / loaded
+    from paper_2401_13920_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    env = {"dev": dev, "dist": dist, "world": world, "rank": rank, "local_rank": local_rank}
+
+    def workload(cfg, tokens=0):
+        w = W.CONFIGS[cfg]
+        if tokens > 0:
+            w = w.scaled(tokens)
+        if world > 1:
+            # every rank routes its own batch: same shape, its own seed
+            w = W.Workload(**{**w.__dict__, "config": w.config + 10 * rank, "name": w.name})
+        return w
+
+    w = workload(args.config, args.tokens)
+    variant = args.variant
+    use_ffn = (w.config % 10) == 5 and not args.no_ffn and variant == "router"
+    m = measure(args, w, env, steps=args.steps, warmup=args.warmup, stage_steps=args.stage_steps, use_ffn=use_ffn,
+                variant=variant, fuse_gate=args.fuse_gate and variant == "router", fused=not args.unfused,
+                e2e_steps=args.e2e_steps, cpu_baseline_s=0.0 if args.no_cpu_baseline else 10.0)
+
+    # ---- the other configurations, each a short run of the same bench (one GPU only; the headline stays above) ----
+    others = None
+    default_headline = args.config == 2 and args.tokens == 0 and variant == "router" and not args.fuse_gate and not args.unfused
+    if world == 1 and default_headline and not args.no_other_configs:
+        others = {}
+        for name, cfg, ffn in (("config1", 1, False), ("config3", 3, False), ("config4", 4, False),
+                               ("config5_router_only", 5, False), ("config5_with_ffn", 5, True)):
+            gc.collect()
+            torch.cuda.empty_cache()
+            try:
+                mo = measure(args, workload(cfg), env, steps=args.other_steps, warmup=5, stage_steps=args.stage_steps,
+                             use_ffn=ffn, variant="router", fuse_gate=False, fused=True, e2e_steps=0, cpu_baseline_s=0.0)
+                others[name] = summary_of(mo)
+                del mo
+            except Exception as exc:   # a configuration that cannot run here is reported, the headline is kept
+                others[name] = {"error": "%s: %s" % (type(exc).__name__, exc)}
+
     if rank == 0:
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic", "config": workload_config(w, args),
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "launches_per_step": launches,
-            "launch_mode": ("CUDA graph replay of the step; every %d-th step eager with per-stage events" % EV)
-                           if graph is not None else "eager",
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
-            "routing": {"kept_fraction": kept / w.T, "C_local": cap.C_local, "C_expert": cap.C_expert, "delta": cap.delta,
-                        "ec_min": cap.ec_min, "rows": rows, "kept_tokens_per_s": value * kept / w.T},
+            "metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": m["steps"], "warmup": m["warmup"],
+            "ms_per_step": m["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "config": m["config"],
+            "clocks": m["clocks"], "e2e": m["e2e"], "gpu_launches": sum(m["launches"].values()) * m["steps"],
+            "launches_per_step": m["launches"],
+            "launch_mode": "CUDA graph replay of the step in the timed region; per-stage times from a separate eager pass"
+                           if m["graph"] else "eager",
+            "roofline": m["roofline"], "cpu_baseline": m["cpu_baseline"], "routing": m["routing"],
+            "other_configs": others,
             "context": "the paper reports a 12.68%-22.24% per-epoch training-time reduction on 64-256 Ascend 910A NPUs; "
                        "it gives no number for this path",
         }

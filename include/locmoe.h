@@ -25,6 +25,20 @@
  *     failed launch.  Conditions met on the device (capacity clamped, a token
  *     with an impossible source device) set LOCMOE_WARN_* bits in the
  *     caller's int32 status word; no kernel traps or asserts.
+ *   - Environment variables, read at call time, select alternative kernels.
+ *     They are testing aids (every choice gives the same results) and no part
+ *     of the interface a program should rely on:
+ *       LOCMOE_PATH=grid|cluster    capacity / route: force the multi-kernel or
+ *                                   the one-cluster form regardless of size
+ *       LOCMOE_GATE=general         gate: the general kernel on shapes that have
+ *                                   a specialised one
+ *       LOCMOE_DISPATCH=tma|vec|flat  dispatch: bulk-copy, warp-per-row or flat
+ *                                   row-major kernel
+ *       LOCMOE_FFN=2|2s             expert FFN: the two-SM kernel (2s: with one
+ *                                   accumulator)
+ *       LOCMOE_PDL=0                plain launches instead of programmatic
+ *                                   dependent launches (read once per process)
+ *       LOCMOE_DEBUG=1              print the CUDA error behind LOCMOE_ERR_CUDA
  *   - Row-major, densely packed arrays.  T tokens, H hidden size (the paper's
  *     d), E experts (n), g = H / E group width.  Logical devices
  *     D = n_nodes * dev_per_node; E % D == 0; expert e lives on device
@@ -161,7 +175,12 @@ int locmoe_capacity(const locmoe_shape_t *shape, const int32_t *idx, const float
  *     ordered by the caller;
  *   - the first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current) and caches it; make
- *     that first call outside of, and before, any stream capture.
+ *     that first call outside of, and before, any stream capture;
+ *   - the cached address is that of the device's primary context at the time
+ *     of the first call.  A cudaDeviceReset, or a switch to another context on
+ *     the same device, makes it stale: do not call this entry point afterwards
+ *     (the library cannot detect this, and kernels would write through a dead
+ *     address).
  */
 int locmoe_capacity_noalloc(const locmoe_shape_t *shape, const int32_t *idx, const float *cos_sim,
                             const locmoe_capacity_rule_t *rule, float *delta_e, float *theta_e,
@@ -423,6 +442,33 @@ typedef struct {
 int locmoe_moe_layer(const locmoe_shape_t *shape, const void *x, const int32_t *src_dev, const float *eps,
                      const locmoe_capacity_rule_t *rule, int32_t C_alloc, int32_t F, const void *w_in,
                      const void *w_out, const locmoe_layer_buffers_t *bufs, void *out, void *stream);
+
+/*
+ * Host-side helpers of the capacity rule and the buffer layout: plain arithmetic
+ * on host memory, nothing is launched.
+ *
+ * locmoe_conventional_capacity: the conventional term of the capacity rule,
+ *   ec = ceil(b_s * c_f / (ep * n)) of Sec. 3.2.3 with b_s = the batch's tokens
+ *   (rule->T_global if > 0, else shape->T), ep = D, at least 1 and at most b_s:
+ *   the row stride a caller allocates the buffer with (C_alloc) when Theorem 1's
+ *   minimum does not bind.  Rounded exactly as the device evaluates the rule.
+ *
+ * locmoe_batch_delta: the batch-wide cosine threshold from per-expert minima
+ *   (delta_e as written by locmoe_capacity, copied to HOST memory, possibly
+ *   already combined over ranks by an element-wise minimum): min over experts,
+ *   clamped to [0, 1] as the device clamps it -- a negative minimum becomes 0, so
+ *   that the value can be passed on as rule->delta_override, where "< 0" would
+ *   mean "measure" (abstract; Lemma 3 uses delta^2).
+ *
+ * locmoe_dest_order: r(a, b) of the buffer layout, the position of logical
+ *   device b in device a's list of destinations -- a itself, then the rest of
+ *   a's node, then the other nodes cyclically (Sec. 3.2.4; abstract: inter-node
+ *   traffic turned into intra-node).  Returns r >= 0, or LOCMOE_ERR_SHAPE.
+ */
+int locmoe_conventional_capacity(const locmoe_shape_t *shape, const locmoe_capacity_rule_t *rule,
+                                 int32_t *C_alloc);
+int locmoe_batch_delta(const float *delta_e_host, int32_t E, double *delta_host);
+int locmoe_dest_order(const locmoe_shape_t *shape, int32_t a, int32_t b);
 
 /* Kernels launched per call of gate, capacity, route, dispatch, combine on this
  * shape (counts[5], host memory); a bookkeeping aid for benchmarks.  The paper

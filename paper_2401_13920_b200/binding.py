@@ -9,7 +9,6 @@ this module raises.
 from __future__ import annotations
 
 import ctypes as C
-import math
 from dataclasses import dataclass
 
 import torch
@@ -25,6 +24,7 @@ FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
     "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route", "locmoe_capacity_route", "locmoe_gate_route",
+    "locmoe_conventional_capacity", "locmoe_batch_delta", "locmoe_dest_order",
     "locmoe_dispatch", "locmoe_combine", "locmoe_dispatch_peer", "locmoe_combine_peer", "locmoe_topk_select", "locmoe_topk_fold", "locmoe_combine_topk", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
@@ -92,6 +92,9 @@ def _load() -> C.CDLL:
     lib.locmoe_topk_select.argtypes = [C.POINTER(Shape), vp, vp, vp, i32, vp, vp, vp]
     lib.locmoe_topk_fold.argtypes = [C.POINTER(Shape), i32, vp, vp]
     lib.locmoe_combine_topk.argtypes = [C.POINTER(Shape), i32, vp, i32, i32, vp, vp, vp, vp]
+    lib.locmoe_conventional_capacity.argtypes = [C.POINTER(Shape), C.POINTER(CapacityRule), C.POINTER(C.c_int32)]
+    lib.locmoe_batch_delta.argtypes = [vp, i32, C.POINTER(C.c_double)]
+    lib.locmoe_dest_order.argtypes = [C.POINTER(Shape), i32, i32]
     lib.locmoe_launch_counts.argtypes = [C.POINTER(Shape), C.POINTER(C.c_int32 * 5)]
     lib.locmoe_device_flags.argtypes = [C.POINTER(C.c_int32), vp]
     lib.locmoe_status_string.argtypes = [C.c_int]
@@ -409,8 +412,28 @@ def locmoe_moe_layer(shape: Shape, x, src_dev, eps, rule: CapacityRule, C_alloc,
 
 
 def conventional_capacity(T: int, D: int, E: int, capacity_factor: float) -> int:
-    """Host-side row stride to allocate: ceil(c_f T / (D n)), at least 1 (Sec. 3.2.3)."""
-    return max(1, math.ceil(capacity_factor * T / (D * E)))
+    """Row stride to allocate the buffer with: the conventional term of the capacity rule for a batch of T tokens
+    (``locmoe_conventional_capacity``; Sec. 3.2.3), evaluated by the library exactly as the device evaluates it."""
+    shape = Shape(int(T), int(E), int(E), int(D), 1, F32, LAYOUT_SEND)      # only T, E and D enter the rule
+    rule = CapacityRule(float(capacity_factor), float(capacity_factor), -1.0, BOUND_BETA, 0)
+    out = C.c_int32(0)
+    _check("locmoe_conventional_capacity", _lib.locmoe_conventional_capacity(C.byref(shape), C.byref(rule), C.byref(out)))
+    return out.value
+
+
+def batch_delta(delta_e) -> float:
+    """Batch-wide cosine threshold from per-expert minima in HOST memory (``locmoe_batch_delta``): the minimum over
+    the experts, clamped to [0, 1] as the device clamps it."""
+    d = delta_e.detach().to("cpu", torch.float32).contiguous()
+    out = C.c_double(0.0)
+    _check("locmoe_batch_delta", _lib.locmoe_batch_delta(C.c_void_p(d.data_ptr()), int(d.numel()), C.byref(out)))
+    return out.value
+
+
+def dest_order(n_nodes: int, dev_per_node: int, a: int, b: int) -> int:
+    """r(a, b): position of logical device b in device a's destination list (``locmoe_dest_order``)."""
+    shape = Shape(1, 1, 1, int(n_nodes), int(dev_per_node), F32, LAYOUT_SEND)   # only the device map is read
+    return _check("locmoe_dest_order", _lib.locmoe_dest_order(C.byref(shape), int(a), int(b)))
 
 
 @dataclass

@@ -1,4 +1,5 @@
 // C-ABI front end: argument validation on the host, then the kernel launchers.
+#include <math.h>
 #include <stdlib.h>
 
 #include "common.cuh"
@@ -356,6 +357,47 @@ int locmoe_moe_layer(const locmoe_shape_t* shape, const void* x, const int32_t* 
     rc = locmoe_combine(shape, C_alloc, ysrc, ydt, b->slot, b->gate_w, out, 0, stream);
     if (rc < 0) return rc;
     return warn | rc;
+}
+
+int locmoe_conventional_capacity(const locmoe_shape_t* shape, const locmoe_capacity_rule_t* rule, int32_t* C_alloc) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!rule || !C_alloc) return LOCMOE_ERR_NULL;
+    if (rule->T_global < 0 || !(rule->capacity_factor >= 0.0)) return LOCMOE_ERR_SHAPE;
+    // the same sequence of individually rounded operations as the device's integer rule (host code is
+    // compiled without contraction of a * b / c into fused operations: these are separate statements)
+    const double dT = (double)(rule->T_global > 0 ? rule->T_global : shape->T);
+    const double dD = (double)shape->n_nodes * (double)shape->dev_per_node, n = (double)shape->E;
+    volatile double cfT = rule->capacity_factor * dT;
+    volatile double den = dD * n;
+    volatile double q = cfT / den;
+    double c = ceil(q);
+    c = c < 1.0 ? 1.0 : (c > dT ? dT : c);
+    *C_alloc = (int32_t)c;
+    return LOCMOE_OK;
+}
+
+int locmoe_batch_delta(const float* delta_e_host, int32_t E, double* delta_host) {
+    if (!delta_e_host || !delta_host) return LOCMOE_ERR_NULL;
+    if (E < 1) return LOCMOE_ERR_SHAPE;
+    float m = delta_e_host[0];
+    for (int32_t e = 0; e < E; ++e) {
+        const float v = delta_e_host[e];
+        if (v != v) return LOCMOE_ERR_SHAPE;   // a NaN cannot be a threshold
+        if (v < m) m = v;
+    }
+    const double d = (double)m;
+    *delta_host = d < 0.0 ? 0.0 : (d > 1.0 ? 1.0 : d);
+    return LOCMOE_OK;
+}
+
+int locmoe_dest_order(const locmoe_shape_t* shape, int32_t a, int32_t b) {
+    if (!shape) return LOCMOE_ERR_NULL;
+    const int N = shape->n_nodes, Dn = shape->dev_per_node;
+    if (N < 1 || Dn < 1 || (long long)N * Dn > 0x7fffffffll) return LOCMOE_ERR_SHAPE;
+    const int D = N * Dn;
+    if (a < 0 || a >= D || b < 0 || b >= D) return LOCMOE_ERR_SHAPE;
+    return dest_order(a, b, N, Dn);
 }
 
 int locmoe_launch_counts(const locmoe_shape_t* shape, int32_t counts[5]) {

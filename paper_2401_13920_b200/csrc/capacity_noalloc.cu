@@ -29,7 +29,10 @@ constexpr int kMaxDevices = 64;
 std::mutex g_setup_mutex;
 void* g_scratch_addr[kMaxDevices] = {nullptr};
 
-// Device address of the scratch on the CURRENT device; looked up once per device and cached.
+// Device address of the scratch on the CURRENT device; looked up once per device and cached.  The cached
+// address belongs to the device's primary context as it was at the first call: after cudaDeviceReset (or in
+// a process that switches to another context on the same device) it is stale, and the entry point must not
+// be used any more.
 int scratch_address(void** out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
@@ -65,6 +68,7 @@ extern "C" int locmoe_capacity_noalloc(const locmoe_shape_t* shape, const int32_
     if (D > shape->E || shape->E % D != 0) return LOCMOE_ERR_SHAPE;
     if (shape->E > kNoAllocMaxExperts) return LOCMOE_ERR_TOO_LARGE;  // beyond the built-in scratch
     if (rule->bound_form < LOCMOE_BOUND_BETA || rule->bound_form > LOCMOE_BOUND_EXP) return LOCMOE_ERR_DTYPE;
+    if (rule->T_global < 0) return LOCMOE_ERR_SHAPE;
     if (!(rule->min_mult >= 0.0) || !(rule->capacity_factor >= 0.0) || rule->delta_override != rule->delta_override)
         return LOCMOE_ERR_SHAPE;
     if ((uintptr_t)cap_dev % 8) return LOCMOE_ERR_ALIGN;

@@ -140,6 +140,14 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 #endif
 
+// r(a, b) of the buffer layout: position of logical device b in device a's destination list (a itself, the rest
+// of a's node, then the other nodes cyclically).  The one definition the kernels and the C ABI share.
+__host__ __device__ __forceinline__ int dest_order(int a, int b, int N, int Dn) {
+    int dn = b / Dn - a / Dn; if (dn < 0) dn += N;
+    int dl = b % Dn - a % Dn; if (dl < 0) dl += Dn;
+    return dn * Dn + dl;
+}
+
 // ---- small device helpers ----
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }

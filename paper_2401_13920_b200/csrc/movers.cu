@@ -320,7 +320,6 @@ __global__ void __launch_bounds__(kThreads) combine_scalar_kernel(const void* __
 int flat_grid(unsigned long long total, int per_thread) {
     unsigned long long want = (total + (unsigned long long)kThreads * per_thread * 2 - 1) / ((unsigned long long)kThreads * per_thread * 2);
     unsigned long long cap = 256ull * sm_count();
-    if (const char* g = getenv("LOCMOE_FLAT_GRID")) cap = (unsigned long long)atoi(g) * sm_count();
     if (want > cap) want = cap;
     return want < 1 ? 1 : (int)want;
 }

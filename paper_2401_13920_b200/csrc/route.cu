@@ -71,18 +71,12 @@ struct RouteArgs {
     locmoe_capacity_t* cap_out;
 };
 
-__device__ __forceinline__ int dest_rank(int a, int b, int N, int Dn) {
-    int dn = b / Dn - a / Dn; if (dn < 0) dn += N;
-    int dl = b % Dn - a % Dn; if (dl < 0) dl += Dn;
-    return dn * Dn + dl;
-}
-
 // Row base (in units of C_alloc rows) of key k = s * E + e in the chosen layout.
 __device__ __forceinline__ long long route_row_base(const RouteArgs& a, int k) {
     const int s = k / a.E, e = k - s * a.E;
     const int b = e / a.Ed, el = e - b * a.Ed;
-    if (a.layout == LOCMOE_LAYOUT_SEND) return ((long long)s * a.D + dest_rank(s, b, a.N, a.Dn)) * a.Ed + el;
-    return (long long)e * a.D + dest_rank(b, s, a.N, a.Dn);
+    if (a.layout == LOCMOE_LAYOUT_SEND) return ((long long)s * a.D + dest_order(s, b, a.N, a.Dn)) * a.Ed + el;
+    return (long long)e * a.D + dest_order(b, s, a.N, a.Dn);
 }
 
 // early != 0: nothing this kernel writes is touched by the kernel queued before it (the caller says so), so the

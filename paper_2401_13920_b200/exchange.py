@@ -14,11 +14,6 @@ import torch
 import torch.distributed as dist
 
 
-def dest_rank_order(a: int, b: int, n_nodes: int, dev_per_node: int) -> int:
-    """Position of device b in device a's destination list: a itself, the rest of a's node, then the other nodes."""
-    return ((b // dev_per_node - a // dev_per_node) % n_nodes) * dev_per_node + ((b % dev_per_node - a % dev_per_node) % dev_per_node)
-
-
 class ExchangePlan:
     """Cell permutations for one rank.  A cell is the block of C_alloc rows of one (source device, expert) pair."""
 
@@ -30,7 +25,8 @@ class ExchangePlan:
         a0 = rank * per
         self.D, self.Ed, self.per, self.world, self.rank = D, Ed, per, world, rank
         self.cells_local = per * D * Ed            # cells of this rank in either layout
-        r = lambda a, b: dest_rank_order(a, b, n_nodes, dev_per_node)
+        from . import binding
+        r = lambda a, b: binding.dest_order(n_nodes, dev_per_node, a, b)   # the layout's r(a, b), from the library
         # send order: destination rank q, then source device a (mine), then destination device b (q's), then local expert
         send = []
         for q in range(world):

@@ -58,13 +58,14 @@ def global_capacity_inputs(delta_e_local: torch.Tensor, T_local: int, group=None
 
     delta_e_local: float32[E], the per-expert minimum cosines of this rank's tokens as written by the capacity
     call (1.0 for an expert without tokens).  Returns (delta, T_global): the batch-wide minimum over experts and
-    ranks, clamped to [0, 1] exactly as the single-GPU call clamps it, and the total token count.  Pass them to
-    the capacity rule as ``delta_override`` and ``T_global``; every rank then derives the same capacities.
+    ranks, clamped to [0, 1] exactly as the single-GPU call clamps it (the library's ``locmoe_batch_delta`` does
+    that; this function only all-reduces), and the total token count.  Pass them to the capacity rule as
+    ``delta_override`` and ``T_global``; every rank then derives the same capacities.
     """
+    from . import binding
     d = delta_e_local.detach().to(torch.float32).clone()
     n = torch.tensor([int(T_local)], dtype=torch.int64, device=d.device)
     if dist.is_available() and dist.is_initialized():
         dist.all_reduce(d, op=dist.ReduceOp.MIN, group=group)
         dist.all_reduce(n, op=dist.ReduceOp.SUM, group=group)
-    delta = float(d.min().item())
-    return min(max(delta, 0.0), 1.0), int(n.item())
+    return binding.batch_delta(d), int(n.item())

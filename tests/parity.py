@@ -183,9 +183,13 @@ def check_combine_sampled(y, shape, st, ref_route, gate_info, tokens_sample):
 
 def run_staged(w: W.Workload, capacity_factor=1.0, min_mult=None, layout=B.LAYOUT_SEND, delta_override=-1.0,
                bound_form=B.BOUND_BETA, C_alloc=None, full=True, n_sample=512, y_random=False, eps=None, seed=0,
-               fused=True):
+               fused=True, allow_substitution=False):
     """Runs the path on the workload (``fused``: "gate" = locmoe_gate_route, True = gate + locmoe_capacity_route, False =
-    the separate calls) and compares every stage; returns a small report."""
+    the separate calls) and compares every stage; returns a small report.
+
+    Unless ``allow_substitution`` is set, the run fails if any expected value had to take a GPU choice as its input
+    (a near-tie picked differently, or an integer capacity moved by the last bit of the fp32 cosine minimum): on the
+    seeded workloads every expected value comes from the oracle's own chain, and the tests say so."""
     dev = torch.device("cuda:0")
     x = W.make_tokens(w, dev)
     src = W.make_src(w, dev)
@@ -209,7 +213,11 @@ def run_staged(w: W.Workload, capacity_factor=1.0, min_mult=None, layout=B.LAYOU
     rep.update(delta=cap.delta, ec_min=cap.ec_min, C_local=cap.C_local, C_expert=cap.C_expert)
     rr = check_route(shape, st, src, cap, gi, ref_cap)
     # True when every expected value below comes from the oracle's chain on the seeded inputs alone
-    rep["oracle_chain_only"] = (gi["n_differ"] == 0) and (ref_cap.C_local, ref_cap.C_expert) == (cap.C_local, cap.C_expert)
+    cap_same = (ref_cap.C_local, ref_cap.C_expert) == (cap.C_local, cap.C_expert)
+    rep["n_substituted"] = gi["n_differ"] + (0 if cap_same else 1)
+    rep["oracle_chain_only"] = rep["n_substituted"] == 0
+    assert allow_substitution or rep["oracle_chain_only"], \
+        "%d near-tie picks / capacities were taken from the GPU for the oracle's route input" % rep["n_substituted"]
     rep.update(drop_frac=float(rr.drop.mean()), status=rr.status)
     ysrc = st.buf if y is None else y
     rng = np.random.default_rng(seed)

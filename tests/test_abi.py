@@ -112,3 +112,75 @@ def test_header_is_plain_c_and_links_from_a_c_program(tmp_path):
     r = subprocess.run([str(exe)], capture_output=True, text=True)
     assert r.returncode == 0, r.stdout + r.stderr
     assert r.stdout.split()[0] == "0" and "invalid shape" in r.stdout
+
+
+def _readme_example():
+    """The indented C example of README.md (the block that starts at the shape initialiser)."""
+    lines = open(os.path.join(ROOT, "README.md")).read().splitlines()
+    start = next(i for i, l in enumerate(lines) if l.startswith("    locmoe_shape_t s ="))
+    block = []
+    for l in lines[start:]:
+        if l.strip() and not l.startswith("    "):
+            break
+        block.append(l)
+    return "\n".join(block)
+
+
+def test_readme_example_compiles_against_the_header(tmp_path):
+    # the README's call sequence, wrapped in a function whose parameters are the names it uses: it must compile as
+    # C99 against include/locmoe.h with every warning on (a missing argument would not)
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if not gcc:
+        pytest.skip("no host compiler")
+    body = _readme_example()
+    assert "locmoe_capacity_route" in body and "locmoe_combine" in body
+    src = tmp_path / "readme_example.c"
+    src.write_text(
+        '#include "locmoe.h"\n'
+        "void example(int32_t T, int32_t H, int32_t E, int32_t n_nodes, int32_t dev_per_node, const void *x, const int32_t *src_dev,\n"
+        "             int32_t *idx, float *gate_w, float *cos_sim, float *delta_e, float *theta_e, locmoe_capacity_t *cap,\n"
+        "             int32_t *pos, int32_t *slot, uint8_t *drop, int32_t *inv, int32_t *counts, int32_t *kept,\n"
+        "             int32_t *send_counts, int32_t *load, int64_t *locality, int32_t *status, void *ws, void *buf,\n"
+        "             const void *y, void *out, void *stream) {\n"
+        "    int32_t C_alloc = 0; size_t ws_bytes = 0;\n" + body + "\n}\n")
+    subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-Werror", "-I", os.path.join(ROOT, "include"), "-c", str(src),
+                    "-o", str(tmp_path / "readme_example.o")], check=True)
+
+
+def test_host_helpers_of_the_rule_and_the_layout(B, oracle_mod):
+    import numpy as np
+    from paper_2401_13920_b200 import workloads as W
+    # the conventional term against the oracle's integer rule on the five configurations (its minimum does not bind
+    # at delta = 0) and the three multipliers
+    for w in W.CONFIGS.values():
+        for cf in (1.0, 1.25, 2.0):
+            idx = np.arange(w.T, dtype=np.int32) % w.E
+            ref = oracle_mod.capacity(idx, np.zeros(w.T), w.E, w.H, w.D, min_mult=cf, capacity_factor=cf, delta_override=0.0)
+            assert B.conventional_capacity(w.T, w.D, w.E, cf) == ref.C_local
+    assert B.conventional_capacity(5, 4, 8, 1.0) == 1 and B.conventional_capacity(100, 2, 2, 0.0) == 1
+    sh, rule, out = B.make_shape(100, 64, 8, 2, 2, B.F32), B.CapacityRule(1.0, 1.0, -1.0, 0, 1000), C.c_int32()
+    assert B._lib.locmoe_conventional_capacity(C.byref(sh), C.byref(rule), C.byref(out)) == 0 and out.value == 32   # T_global
+    rule.T_global = -1
+    assert B._lib.locmoe_conventional_capacity(C.byref(sh), C.byref(rule), C.byref(out)) == -2
+    # the batch-wide threshold: minimum over experts, clamped to [0, 1]; a negative minimum must not read as "measure"
+    import torch
+    assert B.batch_delta(torch.tensor([0.5, 0.25, 1.0])) == 0.25
+    assert B.batch_delta(torch.tensor([0.5, -0.125, 1.0])) == 0.0
+    assert B.batch_delta(torch.tensor([1.0, 1.0])) == 1.0
+    assert B.batch_delta(torch.tensor([0.1], dtype=torch.float32)) == float(np.float32(0.1))
+    d = C.c_double()
+    assert B._lib.locmoe_batch_delta(None, 3, C.byref(d)) == -1
+    nan = (C.c_float * 2)(0.5, float("nan"))
+    assert B._lib.locmoe_batch_delta(C.cast(nan, C.c_void_p), 2, C.byref(d)) == -2
+    # r(a, b) against the oracle's destination orders
+    for N, Dn in ((2, 2), (1, 4), (4, 8), (3, 1)):
+        r = oracle_mod.dest_order(N, Dn)              # r[a][b]
+        D = N * Dn
+        for a in range(D):
+            for b in range(D):
+                assert B.dest_order(N, Dn, a, b) == int(r[a][b])
+    # device 1 of a 2 x 2 map lists itself, its node neighbour 0, then the other node's 3 and 2
+    assert [B.dest_order(2, 2, 1, b) for b in (1, 0, 3, 2)] == [0, 1, 2, 3]
+    assert B._lib.locmoe_dest_order(C.byref(B.make_shape(1, 1, 1, 2, 2, B.F32)), 0, 4) == -2

@@ -120,6 +120,49 @@ def test_full_layer_config5_scaled(P, monkeypatch, kernel):
     P.check_combine_sampled(y, sh, st, rr, gi, toks)
 
 
+def test_full_layer_config5_full_size(P):
+    # config 5 at its full size (T = 65536, 2048 rows per expert, F = 10240: 20480 tiles per GEMM) through the one
+    # layer call, default (one-SM) kernel: router stages against the oracle, sampled expert-output rows (occupied and
+    # empty) and sampled combined tokens against the fp64 oracle
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    w = W.CONFIGS[5]
+    F = 10240
+    x = W.make_tokens(w, dev)
+    src = W.make_src(w, dev)
+    w_in, w_out = W.make_expert_weights(w, F, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, B.LAYOUT_RECV)
+    rule = B.CapacityRule(1.0, 1.0, -1.0, 0, 0)
+    Ca = B.conventional_capacity(w.T, sh.D, w.E, 1.0)
+    assert Ca == 64
+    st = B.make_router(sh, Ca, rule, dev)
+    h1 = torch.empty(st.rows, F, dtype=torch.bfloat16, device=dev)
+    y = torch.full((st.rows, w.H), 7.0, dtype=torch.bfloat16, device=dev)
+    B.locmoe_moe_layer(sh, x, src, None, rule, Ca, F, w_in, w_out, B.layer_buffers(st, h1, y), st.out)
+    torch.cuda.synchronize()
+    assert B.locmoe_device_flags() == 0
+    gi = P.check_gate(x, sh, st)
+    assert gi["n_differ"] == 0
+    cap, ref_cap = P.check_capacity(sh, st, rule, gi)
+    assert (ref_cap.C_local, ref_cap.C_expert) == (cap.C_local, cap.C_expert) == (64, 2048)
+    rr = P.check_route(sh, st, src, cap, gi, ref_cap)
+    rng = np.random.default_rng(11)
+    P.check_dispatch_sampled(x, sh, st, rr, np.unique(rng.integers(0, st.rows, 1024)))
+    occ = np.nonzero(rr.inv >= 0)[0]
+    emp = np.nonzero(rr.inv < 0)[0]
+    assert len(emp) >= 2
+    M = st.rows // w.E
+    # rows from the first and last tile of an expert, the first and last expert, and random ones in between
+    picks = [occ[0], occ[-1], occ[occ >= 17 * M][0], occ[occ < 18 * M][-1]]
+    picks += list(rng.choice(occ, 14, replace=False)) + [emp[0], emp[-1]]
+    _check_rows(P, st.buf, w_in, w_out, y, w.E, M, [int(r) for r in picks])
+    assert not y[int(emp[0])].any().item() and not y[int(emp[-1])].any().item()
+    toks = np.unique(np.concatenate([rng.integers(0, w.T, 256), [0, w.T - 1], np.nonzero(rr.drop)[0][:16]]))
+    P.check_combine_sampled(y, sh, st, rr, gi, toks)
+    del h1, y, w_in, w_out, st
+    torch.cuda.empty_cache()
+
+
 def test_layer_call_with_identity_experts_equals_the_five_calls(P):
     W, B = P.W, P.B
     dev = torch.device("cuda:0")

@@ -60,10 +60,19 @@ def test_configs_full_size_sampled(P, cfg):
         assert 0.03 < rep["drop_frac"] < 0.15
 
 
-def test_config4_full_size_sampled(P):
+@pytest.mark.parametrize("mult,C_local", [(1.0, 16), (1.25, 20), (2.0, 32)])
+def test_config4_full_size_sampled(P, mult, C_local):
+    # the capacity multipliers of the large-batch configuration at its full size (both knobs); up to 86 GB on the device
     w = P.W.CONFIGS[4]
-    rep = P.run_staged(w, 1.0, full=False, n_sample=1024, y_random=True)
-    assert rep["C_local"] == 16 and 0.05 < rep["drop_frac"] < 0.15
+    rep = P.run_staged(w, mult, full=False, n_sample=1024, y_random=True)
+    assert rep["C_local"] == C_local and rep["oracle_chain_only"]
+    if mult == 1.0:
+        assert 0.05 < rep["drop_frac"] < 0.15
+    elif mult == 1.25:
+        assert 0.005 < rep["drop_frac"] < 0.05
+    else:
+        assert rep["drop_frac"] < 1e-3
+    torch.cuda.empty_cache()
 
 
 # ---- the large-batch variants (multi-kernel capacity, prescanned route histograms) forced at small sizes ----
