@@ -382,6 +382,16 @@ def measure(args, w, env, *, steps, warmup, stage_steps, use_ffn, variant, fuse_
     for k in range(S):
         step(evs[k])
     barrier()
+    # the gate kernel launched back to back on its own (no other kernel's dirty lines to write back under it)
+    gate_alone_ms = None
+    if variant == "router" and not fuse_gate:
+        ga = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(S)]
+        for k in range(S):
+            ga[k][0].record(stream)
+            B.locmoe_gate(st.shape, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
+            ga[k][1].record(stream)
+        barrier()
+        gate_alone_ms = median([g[0].elapsed_time(g[1]) for g in ga])
     clocks = sampler.stop()
     clocks["samples_in_timed_region"] = n_timed
     clocks["covers"] = "timed region and per-stage pass"
@@ -411,6 +421,11 @@ def measure(args, w, env, *, steps, warmup, stage_steps, use_ffn, variant, fuse_
         gbs = bytes_per_launch[s] / (stage_ms[s] * 1e-3) / 1e9
         kernels[s] = {"ms": stage_ms[s], "bytes": bytes_per_launch[s], "achieved_gbs": gbs, "frac": gbs / peak,
                       "frac_nominal": gbs / NOMINAL_HBM_GBS}
+    if gate_alone_ms is not None:
+        g = bytes_per_launch["gate"] / (gate_alone_ms * 1e-3) / 1e9
+        kernels["gate"].update({"alone_ms": gate_alone_ms, "alone_gbs": g, "alone_frac": g / peak, "alone_frac_nominal": g / NOMINAL_HBM_GBS,
+                                "note": "ms / frac: inside the step, where the previous kernel's last ~55 MB of output are still dirty "
+                                        "in L2 and are written back under this kernel; alone_*: the same launch repeated back to back"})
     dominant = max(hbm_stages, key=lambda s: stage_ms[s])
     traffic = ncu_traffic(dominant, w, args.cf, args.tokens) if variant == "router" else None
     path_bytes = sum(bytes_per_launch.values())
@@ -521,8 +536,7 @@ def summary_of(m):
     out = {
         "workload": m["config"]["workload"], "expert_ffn": m["config"]["expert_ffn"], "steps": m["steps"], "warmup": m["warmup"],
         "ms_per_step": m["ms_per_step"], "tokens_per_s": m["value"],
-        "kernels": {k: {"ms": v["ms"], "achieved_gbs": v["achieved_gbs"], "frac": v["frac"], "frac_nominal": v["frac_nominal"]}
-                    for k, v in ks.items()},
+        "kernels": {k: {kk: vv for kk, vv in v.items() if kk not in ("bytes", "note")} for k, v in ks.items()},
         "stage_ms": r["stage_ms"], "path_frac": r["path_frac"], "path_frac_nominal": r["path_frac_nominal"],
         "kept_fraction": m["routing"]["kept_fraction"], "C_local": m["routing"]["C_local"],
         "clocks": {k: m["clocks"][k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples")},

@@ -94,10 +94,14 @@ class PeerBuffers:
             self._handle = symm.rendezvous(self.local, group=group if group is not None else dist.group.WORLD)
             self.pointers = [int(p) for p in self._handle.buffer_ptrs]
 
+    def synchronize(self, stream=None):
+        """Waits for the stream that ran this rank's kernels (before the host reads their results or meets its peers)."""
+        (stream or torch.cuda.current_stream()).synchronize()
+
     def barrier(self, stream=None):
         if self.world == 1:
             return
-        (stream or torch.cuda.current_stream()).synchronize()
+        self.synchronize(stream)
         dist.barrier(group=self.group)
 
 
@@ -112,6 +116,14 @@ def peer_layer_forward(B, sharding, shape_local, C_alloc, rule, x, src_dev, recv
     rank's experts ([E / world][F][H] and [E / world][H][F]).  Sequence: gate -> per-rank minima -> batch-wide
     capacity (All-Reduce MIN / SUM on the host side of ``sharding.global_capacity_inputs``) -> route -> peer-store
     dispatch -> barrier -> local experts -> barrier -> peer-load combine.  Only call sequencing lives here.
+
+    Ordering across ranks (no kernel waits on another GPU, so the host orders the steps): the first barrier ends
+    every rank's stores into the receive buffers before any expert reads them; the second ends every expert's
+    writes of ``y`` before any combine loads them.  A rank's next pass begins with kernels that touch only its own
+    memory and reaches its first barrier only after its own combine has completed, so with a separate ``y`` no
+    third barrier is needed: the experts of the next pass cannot overwrite ``y`` before every rank's combine is
+    done.  When ``y`` IS ``recv`` (identity experts), the next pass's peer stores would land in rows a slower rank's
+    combine is still loading; a trailing barrier closes that window.
     """
     world = recv.world
     rank = dist.get_rank(group) if world > 1 else 0
@@ -121,7 +133,7 @@ def peer_layer_forward(B, sharding, shape_local, C_alloc, rule, x, src_dev, recv
     B.locmoe_gate(shape_local, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
     B.locmoe_capacity(shape_local, st.idx, st.cos_sim, rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
     if world > 1:
-        (stream or torch.cuda.current_stream()).synchronize()
+        recv.synchronize(stream)      # the per-expert minima are read by the host-side reduction
     delta, T_global = sharding.global_capacity_inputs(st.delta_e, shape_local.T, group)
     rule_g = B.CapacityRule(rule.min_mult, rule.capacity_factor, delta if rule.delta_override < 0 else rule.delta_override,
                             rule.bound_form, T_global)
@@ -139,4 +151,6 @@ def peer_layer_forward(B, sharding, shape_local, C_alloc, rule, x, src_dev, recv
         B.locmoe_expert_ffn(sh_ffn, D * C_alloc, F, recv.local, w_in, w_out, h1, y.local, stream)
     y.barrier(stream)
     B.locmoe_combine_peer(shape_local, C_alloc, y.pointers, ydt, st.slot, st.gate_w, out, stream)
+    if world > 1 and (y is recv or y.local.data_ptr() == recv.local.data_ptr()):
+        y.barrier(stream)   # the next pass's peer stores must not overtake a slower rank's loads of the same rows
     return out
