@@ -48,14 +48,19 @@ def parse_args():
     ap.add_argument("--other-steps", type=int, default=20, help="timed steps of each of the other configurations")
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the short runs of configurations 1, 3, 4 and 5 that the default line carries")
-    ap.add_argument("--variant", choices=["router", "peer8", "topk2"], default="router",
+    ap.add_argument("--variant", choices=["router", "peer8", "topk2", "peer"], default="router",
                     help="router: the metric's path; peer8: dispatch / combine through a table of eight receive buffers "
-                         "(the fused-exchange kernels, all buffers on this GPU); topk2: the top-2 variant")
+                         "(the fused-exchange kernels, all buffers on this GPU); topk2: the top-2 variant; peer: one rank "
+                         "per GPU, each routing the tokens of its own logical source devices and storing them straight "
+                         "into the receive buffers of the GPUs that host the experts (exchange.peer_layer_forward)")
     ap.add_argument("--fuse-gate", action="store_true",
                     help="gate, capacity and route as the one call locmoe_gate_route (the gate's time is then part of that stage)")
     ap.add_argument("--unfused", action="store_true", help="capacity and route as two calls instead of locmoe_capacity_route")
     ap.add_argument("--no-ffn", action="store_true", help="config 5 only: identity experts instead of the expert FFN")
     ap.add_argument("--ffn-inner", type=int, default=10240, help="config 5: inner size F of the expert FFN")
+    ap.add_argument("--slices", type=int, default=1,
+                    help="--variant peer with the expert FFN (config 5): expert blocks per rank, the exchange of block s+1 "
+                         "overlapping the experts of block s")
     ap.add_argument("--tokens", type=int, default=0, help="override T (profiling-sized case; not the metric's workload)")
     return ap.parse_args()
 
@@ -214,7 +219,9 @@ def workload_config(w, args, n_tokens=None):
         "expert_ffn": bool((w.config % 10) == 5 and not getattr(args, "no_ffn", False) and getattr(args, "variant", "router") == "router"),
         "variant": {"router": "the metric's path (top-1, one GPU)",
                     "peer8": "dispatch / combine through a table of eight receive buffers (fused-exchange kernels, all on this GPU)",
-                    "topk2": "top-2 variant: 2T assignments routed, two-term combine"}[getattr(args, "variant", "router")],
+                    "topk2": "top-2 variant: 2T assignments routed, two-term combine",
+                    "peer": "fused exchange: every rank routes its own source devices' tokens and stores them into the "
+                            "owners' receive buffers (peer stores / loads; identity experts)"}[getattr(args, "variant", "router")],
         "T": n_tokens or w.T, "H": w.H, "E": w.E, "token_dtype": w.dtype, "n_nodes": w.n_nodes,
         "dev_per_node": w.dev_per_node, "capacity_factor": args.cf, "layout": args.layout,
         "l2": "inputs exceed the 126 MB L2, no flush" if (n_tokens or w.T) * w.H * (2 if w.dtype == "bf16" else 4) > 126e6
@@ -240,6 +247,8 @@ def measure(args, w, env, *, steps, warmup, stage_steps, use_ffn, variant, fuse_
     from paper_2401_13920_b200 import workloads as W
 
     dev, dist, world, rank, local_rank = env["dev"], env["dist"], env["world"], env["rank"], env["local_rank"]
+    if variant == "peer":
+        return measure_peer(args, w, env, steps=steps, warmup=warmup, stage_steps=stage_steps)
     layout_name = args.layout
     if use_ffn or variant == "peer8":
         layout_name = "recv"      # the expert FFN and the peer kernels work on the receive-side layout
@@ -527,6 +536,128 @@ def measure(args, w, env, *, steps, warmup, stage_steps, use_ffn, variant, fuse_
         "routing": {"kept_fraction": kept / w.T, "C_local": cap.C_local, "C_expert": cap.C_expert, "delta": cap.delta,
                     "ec_min": cap.ec_min, "rows": rows, "kept_tokens_per_s": value * kept / w.T},
     }
+
+
+def measure_peer(args, w, env, *, steps, warmup, stage_steps):
+    """The fused exchange at N ranks: rank r owns the logical devices [r D/N, (r+1) D/N) and draws w.T tokens that
+    come from them (weak scaling: N * w.T tokens in the whole batch, the capacity rule counts all of them); every
+    rank routes its tokens in the receive-side layout of the whole map, stores kept rows into the owners' buffers
+    (peer stores), and combines through peer loads; identity experts.  The host orders the steps across ranks
+    (barriers inside exchange.peer_layer_forward), so the step is launched eagerly, not as a CUDA graph."""
+    import torch
+    from paper_2401_13920_b200 import binding as B
+    from paper_2401_13920_b200 import exchange, sharding
+    from paper_2401_13920_b200 import workloads as W
+
+    dev, dist, world, rank, local_rank = env["dev"], env["dist"], env["world"], env["rank"], env["local_rank"]
+    D = w.n_nodes * w.dev_per_node
+    devs = sharding.devices_of_rank(D, world, rank)
+    x = W.make_tokens(w, dev)                                       # this rank's tokens (its own seed when N > 1)
+    src = (devs.start + torch.arange(w.T, device=dev, dtype=torch.int64) % len(devs)).to(torch.int32)
+    T_global = world * w.T
+    shape = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, B.LAYOUT_RECV)
+    rule = B.CapacityRule(args.cf, args.cf, -1.0, B.BOUND_BETA, 0)
+    C_alloc = B.conventional_capacity(T_global, D, w.E, args.cf)
+    rows = D * w.E * C_alloc
+    st = B.make_router(shape, C_alloc, rule, dev, with_buffer=False)
+    recv = exchange.PeerBuffers(rows // world, w.H, x.dtype, dev)   # this rank's slice of the receive buffer
+    stream = torch.cuda.current_stream()
+    stages = ["gate", "capacity_route", "dispatch_peer", "experts", "combine_peer"]
+    use_ffn = (w.config % 10) == 5 and not args.no_ffn
+    F = args.ffn_inner
+    y, w_in, w_out, h1, ffn_stream = recv, None, None, None, None
+    if use_ffn:                                                     # this rank's experts: E / world of them
+        w_all_in, w_all_out = W.make_expert_weights(w, F, dev)
+        El = w.E // world
+        w_in, w_out = w_all_in[rank * El:(rank + 1) * El].contiguous(), w_all_out[rank * El:(rank + 1) * El].contiguous()
+        del w_all_in, w_all_out
+        y = exchange.PeerBuffers(rows // world, w.H, torch.bfloat16, dev)
+        h1 = torch.empty(rows // world, F, dtype=torch.bfloat16, device=dev)
+        ffn_stream = torch.cuda.Stream(dev) if args.slices > 1 else None
+
+    def step(ev=None):
+        i = 0
+        def mark():
+            nonlocal i
+            if ev:
+                ev[i].record(stream)
+            i += 1
+        exchange.peer_layer_forward(B, sharding, shape, C_alloc, rule, x, src, recv, y, st, w_in, w_out, F, h1, stream=stream,
+                                    mark=mark, slices=args.slices if use_ffn else 1, ffn_stream=ffn_stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    warmup = max(warmup, 3)
+    for _ in range(warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(physical_gpu_index(local_rank), period_s=0.001)
+    sampler.start()
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for _ in range(steps):
+        step()
+    t1.record(stream)
+    barrier()
+    n_timed = len(sampler.samples)
+    total_ms = sharding.max_over_ranks(t0.elapsed_time(t1), dev)
+    S = max(int(stage_steps), 20)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(S)]
+    for k in range(S):
+        step(evs[k])
+    barrier()
+    clocks = sampler.stop()
+    clocks["samples_in_timed_region"] = n_timed
+    stage_ms = {s: median([evs[k][i].elapsed_time(evs[k][i + 1]) for k in range(S)]) for i, s in enumerate(stages)}
+    if B.locmoe_device_flags() != 0:
+        raise RuntimeError("a kernel gave up a bounded wait during the bench")
+    kept = int((st.slot >= 0).sum().item())
+    sc = st.send_counts.view(D, D)[devs.start:devs.stop]           # kept rows of my sources per destination device
+    own = int(sc[:, devs.start:devs.stop].sum().item())
+    to_peers = (int(sc.sum().item()) - own) * w.H * x.element_size()
+    bx = x.element_size()
+    rows_mine = rows // world                                      # rows this rank zero-fills / owns on average
+    bytes_per_launch = {"gate": w.T * w.H * bx + 12 * w.T,
+                        "dispatch_peer": kept * w.H * bx + rows_mine * w.H * bx + 4 * rows_mine,
+                        "combine_peer": kept * w.H * bx + w.T * w.H * bx + 8 * w.T}
+    peak, peak_kind = measured_peak()
+    kernels = {}
+    for s_, b_ in bytes_per_launch.items():
+        gbs = b_ / (stage_ms[s_] * 1e-3) / 1e9
+        kernels[s_] = {"ms": stage_ms[s_], "bytes": b_, "achieved_gbs": gbs, "frac": gbs / peak, "frac_nominal": gbs / NOMINAL_HBM_GBS}
+    ms_per_step = total_ms / steps
+    path_bytes = sum(bytes_per_launch.values())
+    path_gbs = path_bytes / (ms_per_step * 1e-3) / 1e9
+    dominant = max(bytes_per_launch, key=lambda s_: stage_ms[s_])
+    link_gbs = to_peers / (stage_ms["dispatch_peer"] * 1e-3) / 1e9 if to_peers else 0.0
+    roofline = {"bound": "hbm" if world == 1 else "hbm / nvlink", "kernel": dominant, "achieved": kernels[dominant]["achieved_gbs"],
+                "peak": peak, "peak_kind": peak_kind + " (copy, MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
+                "unit": "GB/s", "frac": kernels[dominant]["frac"], "frac_nominal": kernels[dominant]["frac_nominal"],
+                "nominal_peak": NOMINAL_HBM_GBS, "traffic": None, "traffic_source": None, "path_bytes": path_bytes,
+                "path_frac": path_gbs / peak, "path_frac_nominal": path_gbs / NOMINAL_HBM_GBS, "kernels": kernels,
+                "stage_ms": stage_ms, "stage_ms_how": "median of %d eager steps, CUDA events between the stages" % S,
+                "peer": {"world": world, "bytes_to_peers_per_step": to_peers, "bytes_from_peers_per_step": to_peers,
+                         "peer_store_gbs_per_rank": link_gbs, "nvlink_measured_gbs_per_direction": 770.0,
+                         "expert_ffn": use_ffn, "slices": args.slices if use_ffn else 1,
+                         "note": "stage times of dispatch_peer / experts include the host-ordered barrier across ranks; with "
+                                 "slices > 1 dispatch_peer is the main stream's share (the windowed stores) and experts the wait "
+                                 "for the second stream"}}
+    cap = B.locmoe_capacity_read(st.cap_dev)
+    launches = B.locmoe_launch_counts(shape)
+    launches = {"gate": 1, "capacity": launches["capacity"], "capacity_route": launches["route"], "dispatch_peer": 1, "combine_peer": 1}
+    args_l = argparse.Namespace(**{**vars(args), "layout": "recv", "no_ffn": True, "variant": "peer"})
+    cfg = workload_config(w, args_l)
+    cfg["T_global"] = T_global
+    cfg["expert_ffn"] = use_ffn
+    return {"value": world * w.T * steps / (total_ms * 1e-3), "ms_per_step": ms_per_step, "steps": steps, "warmup": warmup,
+            "config": cfg, "clocks": clocks, "e2e": None, "launches": launches, "graph": False, "roofline": roofline,
+            "cpu_baseline": None,
+            "routing": {"kept_fraction": kept / w.T, "C_local": cap.C_local, "C_expert": cap.C_expert, "delta": cap.delta,
+                        "ec_min": cap.ec_min, "rows": rows, "kept_tokens_per_s": world * kept * steps / (total_ms * 1e-3)}}
 
 
 def summary_of(m):

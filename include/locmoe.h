@@ -134,6 +134,34 @@ int locmoe_gate(const locmoe_shape_t *shape, const void *x, const float *eps,
                 int32_t *idx, float *gate_w, float *cos_sim, float *probs, void *stream);
 
 /*
+ * The gate with its optional extras (Sec. 3.2.1 for the bias eps_i, which the paper
+ * leaves undefined; Sec. 3.2.2 for the P_i of the auxiliary loss).  Same outputs as
+ * locmoe_gate; the options struct is HOST memory, its pointers are device pointers.
+ *   eps / src_dev  with src_dev == NULL, eps is float[E] as in locmoe_gate (or NULL).
+ *                  With src_dev int32[T], eps is a table float[D][E] and token t takes
+ *                  the row of its source device: G_i = ReLU(mean_i + eps[src_dev[t]][i]);
+ *                  a token whose source is outside [0, D) gets no bias.
+ *   probs          float[T][E] or NULL, as in locmoe_gate.
+ *   p_part         float[LOCMOE_GATE_PARTIAL_ROWS][E] or NULL: the column sums of the
+ *                  probabilities, formed inside the gate kernel -- every CTA adds the rows
+ *                  of its warps in a fixed order and writes one row of p_part -- so that
+ *                  P_i and L_aux need no probability matrix (locmoe_aux_loss_partial).
+ *                  The number of rows written is returned in p_rows (host field); it
+ *                  depends on the shape and the device only, and so does the summation
+ *                  order: the sums are deterministic.
+ */
+enum { LOCMOE_GATE_PARTIAL_ROWS = 2048 };
+typedef struct {
+    const float *eps;
+    const int32_t *src_dev;
+    float *probs;
+    float *p_part;
+    int32_t p_rows;  /* out */
+} locmoe_gate_opts_t;
+int locmoe_gate_ex(const locmoe_shape_t *shape, const void *x, locmoe_gate_opts_t *opts,
+                   int32_t *idx, float *gate_w, float *cos_sim, void *stream);
+
+/*
  * Angular deviation and capacity (abstract; Lemma 3; Theorem 1; Sec. 3.2.3).
  *   delta_e[e] = smallest cos_sim among tokens with idx == e (1 if none),
  *   theta_e[e] = acos(delta_e[e])  -- the largest angle between expert e's
@@ -316,6 +344,15 @@ int locmoe_dispatch_peer(const locmoe_shape_t *shape, int32_t C_alloc, const voi
                          const int32_t *inv, const int32_t *slot, void *const *peer_bufs,
                          int32_t n_peers, int32_t src_lo, int32_t src_hi, int32_t zero_pad,
                          void *stream);
+/* locmoe_dispatch_peer restricted to a window of every owner's buffer: only rows whose index INSIDE their
+ * owner's slice lies in [win_lo, win_hi) are stored or zero-filled (0 and INT64_MAX: everything).  With the
+ * window of one block of experts, a caller fills the receive buffer block by block and starts the experts of
+ * a block while the next one is in flight -- the overlap of the exchange with the expert computation of
+ * Sec. 3.2.4. */
+int locmoe_dispatch_peer_window(const locmoe_shape_t *shape, int32_t C_alloc, const void *x,
+                                const int32_t *inv, const int32_t *slot, void *const *peer_bufs,
+                                int32_t n_peers, int32_t src_lo, int32_t src_hi, int32_t zero_pad,
+                                int64_t win_lo, int64_t win_hi, void *stream);
 int locmoe_combine_peer(const locmoe_shape_t *shape, int32_t C_alloc, void *const *peer_y,
                         int32_t n_peers, int32_t y_dtype, const int32_t *slot, const float *gate_w,
                         void *out, void *stream);
@@ -362,6 +399,13 @@ int locmoe_combine_topk(const locmoe_shape_t *shape, int32_t C_alloc, const void
  */
 int locmoe_aux_loss(const locmoe_shape_t *shape, const float *probs, const int32_t *load, float alpha,
                     float *f_out, float *p_out, float *loss_out, void *ws, size_t ws_bytes, void *stream);
+
+/* The same loss (Sec. 3.2.2) from the per-CTA column sums locmoe_gate_ex left in p_part
+ * (p_rows rows of E floats): P_i = (1/T) * sum of the rows in index order, in fp64.  No
+ * probability matrix and no workspace. */
+int locmoe_aux_loss_partial(const locmoe_shape_t *shape, const float *p_part, int32_t p_rows,
+                            const int32_t *load, float alpha, float *f_out, float *p_out,
+                            float *loss_out, void *stream);
 
 /*
  * Locality loss, forward value (Sec. 3.2.2, second loss equation):

@@ -143,6 +143,28 @@ def gate(x, dtype, E, eps=None, want_G=False, want_probs=False) -> GateOut:
     return GateOut(idx, R, cs, gap, G, pr)
 
 
+def gate_per_source(x, dtype, E, eps_table, src, want_probs=False) -> GateOut:
+    """The gate with a per-source-device bias table eps_table[D][E]: token t is gated with the row of its source
+    device src[t] (no bias when src[t] is outside [0, D)).  The oracle's gate routine is simply called once per
+    source device on that device's tokens; nothing is computed here."""
+    eps_table = np.ascontiguousarray(eps_table, dtype=np.float32)
+    src = np.asarray(src)
+    D = eps_table.shape[0]
+    T = src.shape[0]
+    out = GateOut(np.empty(T, np.int32), np.empty(T, np.float64), np.empty(T, np.float64), np.empty(T, np.float64), None,
+                  np.empty((T, E), np.float64) if want_probs else None)
+    groups = [(np.nonzero(src == d)[0], eps_table[d]) for d in range(D)]
+    groups.append((np.nonzero((src < 0) | (src >= D))[0], None))
+    for sel, row in groups:
+        if len(sel) == 0:
+            continue
+        g = gate(np.ascontiguousarray(np.asarray(x)[sel]), dtype, E, eps=row, want_probs=want_probs)
+        out.idx[sel], out.R[sel], out.cos[sel], out.gap[sel] = g.idx, g.R, g.cos, g.gap
+        if want_probs:
+            out.probs[sel] = g.probs
+    return out
+
+
 def p_delta(delta: float, d: int) -> float:
     return lib().oracle_p_delta(float(delta), int(d))
 

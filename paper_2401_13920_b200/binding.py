@@ -23,9 +23,9 @@ WARN_CLAMPED, WARN_BAD_SRC, WARN_BAD_IDX = 1, 2, 4
 FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 
 EXPORTS = [
-    "locmoe_workspace_bytes", "locmoe_gate", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route", "locmoe_capacity_route", "locmoe_gate_route",
+    "locmoe_workspace_bytes", "locmoe_gate", "locmoe_gate_ex", "locmoe_aux_loss_partial", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route", "locmoe_capacity_route", "locmoe_gate_route",
     "locmoe_conventional_capacity", "locmoe_batch_delta", "locmoe_dest_order",
-    "locmoe_dispatch", "locmoe_combine", "locmoe_dispatch_peer", "locmoe_combine_peer", "locmoe_topk_select", "locmoe_topk_fold", "locmoe_combine_topk", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
+    "locmoe_dispatch", "locmoe_combine", "locmoe_dispatch_peer", "locmoe_dispatch_peer_window", "locmoe_combine_peer", "locmoe_topk_select", "locmoe_topk_fold", "locmoe_combine_topk", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
 
@@ -47,6 +47,14 @@ class Capacity(C.Structure):
     _fields_ = [("delta", C.c_double), ("p_delta", C.c_double), ("ec_min", C.c_double),
                 ("C_expert", C.c_int32), ("C_local", C.c_int32), ("n_empty_experts", C.c_int32),
                 ("flags", C.c_int32)]
+
+
+GATE_PARTIAL_ROWS = 2048
+
+
+class GateOpts(C.Structure):
+    _fields_ = [("eps", C.c_void_p), ("src_dev", C.c_void_p), ("probs", C.c_void_p), ("p_part", C.c_void_p),
+                ("p_rows", C.c_int32)]
 
 
 class LayerBuffers(C.Structure):
@@ -71,6 +79,8 @@ def _load() -> C.CDLL:
     vp, i32 = C.c_void_p, C.c_int32
     lib.locmoe_workspace_bytes.argtypes = [C.POINTER(Shape), i32, C.POINTER(C.c_size_t)]
     lib.locmoe_gate.argtypes = [C.POINTER(Shape), vp, vp, vp, vp, vp, vp, vp]
+    lib.locmoe_gate_ex.argtypes = [C.POINTER(Shape), vp, C.POINTER(GateOpts), vp, vp, vp, vp]
+    lib.locmoe_aux_loss_partial.argtypes = [C.POINTER(Shape), vp, i32, vp, C.c_float, vp, vp, vp, vp]
     lib.locmoe_capacity.argtypes = [C.POINTER(Shape), vp, vp, C.POINTER(CapacityRule), vp, vp, vp, vp, C.c_size_t, vp]
     lib.locmoe_capacity_noalloc.argtypes = [C.POINTER(Shape), vp, vp, C.POINTER(CapacityRule), vp, vp, vp, vp]
     lib.locmoe_capacity_read.argtypes = [vp, C.POINTER(Capacity), vp]
@@ -88,6 +98,8 @@ def _load() -> C.CDLL:
     lib.locmoe_loc_loss.argtypes = [C.POINTER(Shape), vp, i32, C.c_double, C.c_double, vp, vp, vp, vp, vp]
     lib.locmoe_cos_hist.argtypes = [C.POINTER(Shape), vp, vp, i32, i32, i32, C.c_float, C.c_float, vp, vp, vp, vp]
     lib.locmoe_dispatch_peer.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, C.POINTER(vp), i32, i32, i32, i32, vp]
+    lib.locmoe_dispatch_peer_window.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, C.POINTER(vp), i32, i32, i32, i32,
+                                                C.c_int64, C.c_int64, vp]
     lib.locmoe_combine_peer.argtypes = [C.POINTER(Shape), i32, C.POINTER(vp), i32, i32, vp, vp, vp, vp]
     lib.locmoe_topk_select.argtypes = [C.POINTER(Shape), vp, vp, vp, i32, vp, vp, vp]
     lib.locmoe_topk_fold.argtypes = [C.POINTER(Shape), i32, vp, vp]
@@ -186,6 +198,39 @@ def locmoe_gate(shape: Shape, x, eps, idx, gate_w, cos_sim, probs=None, stream=N
         _want(probs, torch.float32, shape.T * shape.E, "probs")
     return _check("locmoe_gate", _lib.locmoe_gate(C.byref(shape), _ptr(x), _ptr(eps), _ptr(idx), _ptr(gate_w),
                                                   _ptr(cos_sim), _ptr(probs), _stream(stream)))
+
+
+def locmoe_gate_ex(shape: Shape, x, idx, gate_w, cos_sim, eps=None, src_dev=None, probs=None, p_part=None, stream=None) -> int:
+    """The gate with its extras; returns the number of rows of ``p_part`` the call wrote (0 without ``p_part``).
+    ``eps`` is float[E], or float[D][E] when ``src_dev`` (int32[T]) is given: the per-source bias table."""
+    _want(x, torch.float32 if shape.x_dtype == F32 else torch.bfloat16, shape.T * shape.H, "x")
+    _want(idx, torch.int32, shape.T, "idx")
+    _want(gate_w, torch.float32, shape.T, "gate_w")
+    _want(cos_sim, torch.float32, shape.T, "cos_sim")
+    if eps is not None:
+        _want(eps, torch.float32, shape.E * (shape.D if src_dev is not None else 1), "eps")
+    if src_dev is not None:
+        _want(src_dev, torch.int32, shape.T, "src_dev")
+    if probs is not None:
+        _want(probs, torch.float32, shape.T * shape.E, "probs")
+    if p_part is not None:
+        _want(p_part, torch.float32, GATE_PARTIAL_ROWS * shape.E, "p_part")
+    p = lambda t: None if t is None else _ptr(t).value
+    opts = GateOpts(p(eps), p(src_dev), p(probs), p(p_part), 0)
+    _check("locmoe_gate_ex", _lib.locmoe_gate_ex(C.byref(shape), _ptr(x), C.byref(opts), _ptr(idx), _ptr(gate_w), _ptr(cos_sim),
+                                                 _stream(stream)))
+    return opts.p_rows
+
+
+def locmoe_aux_loss_partial(shape: Shape, p_part, p_rows, load, alpha, f_out, p_out, loss_out, stream=None) -> int:
+    _want(p_part, torch.float32, p_rows * shape.E, "p_part")
+    _want(load, torch.int32, shape.E, "load")
+    _want(f_out, torch.float32, shape.E, "f_out")
+    _want(p_out, torch.float32, shape.E, "p_out")
+    _want(loss_out, torch.float32, 1, "loss_out")
+    return _check("locmoe_aux_loss_partial", _lib.locmoe_aux_loss_partial(C.byref(shape), _ptr(p_part), int(p_rows), _ptr(load),
+                                                                          float(alpha), _ptr(f_out), _ptr(p_out), _ptr(loss_out),
+                                                                          _stream(stream)))
 
 
 def locmoe_capacity(shape: Shape, idx, cos_sim, rule: CapacityRule, delta_e, theta_e, cap_dev, ws, stream=None) -> int:
@@ -324,13 +369,19 @@ def _ptr_table(ptrs):
     return (C.c_void_p * len(vals))(*vals), len(vals)
 
 
-def locmoe_dispatch_peer(shape: Shape, C_alloc, x, inv, slot, peer_bufs, src_lo, src_hi, zero_pad=True, stream=None) -> int:
+def locmoe_dispatch_peer(shape: Shape, C_alloc, x, inv, slot, peer_bufs, src_lo, src_hi, zero_pad=True, stream=None,
+                         window=None) -> int:
+    """``window`` = (lo, hi): only rows whose index inside their owner's slice lies in [lo, hi) (locmoe_dispatch_peer_window)."""
     rows = shape.D * shape.E * C_alloc
     dt = torch.float32 if shape.x_dtype == F32 else torch.bfloat16
     _want(x, dt, shape.T * shape.H, "x")
     _want(inv, torch.int32, rows, "inv")
     _want(slot, torch.int32, shape.T, "slot")
     table, n = _ptr_table(peer_bufs)
+    if window is not None:
+        return _check("locmoe_dispatch_peer_window", _lib.locmoe_dispatch_peer_window(
+            C.byref(shape), int(C_alloc), _ptr(x), _ptr(inv), _ptr(slot), table, n, int(src_lo), int(src_hi),
+            1 if zero_pad else 0, int(window[0]), int(window[1]), _stream(stream)))
     return _check("locmoe_dispatch_peer", _lib.locmoe_dispatch_peer(C.byref(shape), int(C_alloc), _ptr(x), _ptr(inv), _ptr(slot),
                                                                     table, n, int(src_lo), int(src_hi), 1 if zero_pad else 0,
                                                                     _stream(stream)))
@@ -467,8 +518,10 @@ class RouterState:
         return self.shape.D * self.shape.E * self.C_alloc
 
 
-def make_router(shape: Shape, C_alloc: int, rule: CapacityRule, device="cuda") -> RouterState:
-    """Allocates every output and scratch tensor of the five calls with torch (memory plumbing only)."""
+def make_router(shape: Shape, C_alloc: int, rule: CapacityRule, device="cuda", with_buffer: bool = True) -> RouterState:
+    """Allocates every output and scratch tensor of the five calls with torch (memory plumbing only).
+    ``with_buffer`` = False leaves out the dispatch buffer (a rank of the fused exchange writes into the peers'
+    receive buffers instead)."""
     dev = torch.device(device)
     T, H, E, D = shape.T, shape.H, shape.E, shape.D
     rows = D * E * C_alloc
@@ -486,7 +539,7 @@ def make_router(shape: Shape, C_alloc: int, rule: CapacityRule, device="cuda") -
         send_counts=torch.empty(D * D, **i32), load=torch.empty(E, **i32),
         locality=torch.empty(6, dtype=torch.int64, device=dev), status=torch.zeros(1, **i32),
         ws=torch.empty(ws_bytes, dtype=torch.uint8, device=dev),
-        buf=torch.empty(rows, H, dtype=xdt, device=dev), out=torch.empty(T, H, dtype=xdt, device=dev),
+        buf=torch.empty(rows if with_buffer else 0, H, dtype=xdt, device=dev), out=torch.empty(T, H, dtype=xdt, device=dev),
     )
 
 

@@ -80,6 +80,30 @@ int locmoe_gate(const locmoe_shape_t* shape, const void* x, const float* eps, in
     return launch_gate(*shape, x, eps, idx, gate_w, cos_sim, probs, static_cast<cudaStream_t>(stream));
 }
 
+int locmoe_gate_ex(const locmoe_shape_t* shape, const void* x, locmoe_gate_opts_t* opts, int32_t* idx, float* gate_w,
+                   float* cos_sim, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!x || !opts || !idx || !gate_w || !cos_sim) return LOCMOE_ERR_NULL;
+    const int esz = shape->x_dtype == LOCMOE_F32 ? 4 : 2;
+    if ((uintptr_t)x % esz) return LOCMOE_ERR_ALIGN;
+    if (opts->src_dev && !opts->eps) return LOCMOE_ERR_NULL;   // a table is asked for but not given
+    const GateExtra extra{opts->eps ? opts->src_dev : nullptr, opts->p_part};
+    opts->p_rows = 0;
+    rc = launch_gate(*shape, x, opts->eps, idx, gate_w, cos_sim, opts->probs, static_cast<cudaStream_t>(stream), nullptr, &extra);
+    if (rc == LOCMOE_OK && opts->p_part) opts->p_rows = gate_last_grid();
+    return rc;
+}
+
+int locmoe_aux_loss_partial(const locmoe_shape_t* shape, const float* p_part, int32_t p_rows, const int32_t* load,
+                            float alpha, float* f_out, float* p_out, float* loss_out, void* stream) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!p_part || !load || !f_out || !p_out || !loss_out) return LOCMOE_ERR_NULL;
+    if (p_rows < 1 || p_rows > LOCMOE_GATE_PARTIAL_ROWS) return LOCMOE_ERR_SHAPE;
+    return launch_aux_from_partials(*shape, p_part, p_rows, load, alpha, f_out, p_out, loss_out, static_cast<cudaStream_t>(stream));
+}
+
 int locmoe_capacity(const locmoe_shape_t* shape, const int32_t* idx, const float* cos_sim,
                     const locmoe_capacity_rule_t* rule, float* delta_e, float* theta_e, locmoe_capacity_t* cap_dev,
                     void* ws, size_t ws_bytes, void* stream) {
@@ -258,6 +282,13 @@ int check_peers(const locmoe_shape_t* shape, void* const* peers, int32_t n_peers
 int locmoe_dispatch_peer(const locmoe_shape_t* shape, int32_t C_alloc, const void* x, const int32_t* inv,
                          const int32_t* slot, void* const* peer_bufs, int32_t n_peers, int32_t src_lo, int32_t src_hi,
                          int32_t zero_pad, void* stream) {
+    return locmoe_dispatch_peer_window(shape, C_alloc, x, inv, slot, peer_bufs, n_peers, src_lo, src_hi, zero_pad, 0,
+                                       INT64_MAX, stream);
+}
+
+int locmoe_dispatch_peer_window(const locmoe_shape_t* shape, int32_t C_alloc, const void* x, const int32_t* inv,
+                                const int32_t* slot, void* const* peer_bufs, int32_t n_peers, int32_t src_lo, int32_t src_hi,
+                                int32_t zero_pad, int64_t win_lo, int64_t win_hi, void* stream) {
     int rc = check_shape(shape);
     if (rc) return rc;
     if (!x || !inv || !slot) return LOCMOE_ERR_NULL;
@@ -269,8 +300,9 @@ int locmoe_dispatch_peer(const locmoe_shape_t* shape, int32_t C_alloc, const voi
     const size_t rb = (size_t)shape->H * (shape->x_dtype == LOCMOE_F32 ? 4 : 2);
     if (rb % 16 || (uintptr_t)x % 16) return LOCMOE_ERR_ALIGN;
     if ((unsigned long long)shape->T * (rb / 16) >= 0xf0000000ull) return LOCMOE_ERR_SHAPE;
+    if (win_lo < 0 || win_hi < win_lo) return LOCMOE_ERR_SHAPE;
     return launch_dispatch_peer(*shape, C_alloc, rows, x, inv, slot, peer_bufs, n_peers, src_lo, src_hi, zero_pad,
-                                static_cast<cudaStream_t>(stream));
+                                (long long)win_lo, (long long)win_hi, static_cast<cudaStream_t>(stream));
 }
 
 int locmoe_combine_peer(const locmoe_shape_t* shape, int32_t C_alloc, void* const* peer_y, int32_t n_peers, int32_t y_dtype,

@@ -65,4 +65,11 @@ int launch_aux_loss(const locmoe_shape_t& s, const float* probs, const int32_t* 
     return check_launch();
 }
 
+// The same loss from column sums the gate has already formed per CTA (locmoe_gate_ex): only the second level runs.
+int launch_aux_from_partials(const locmoe_shape_t& s, const float* p_part, int n_rows, const int32_t* load, float alpha,
+                             float* f, float* P, float* loss, cudaStream_t st) {
+    aux_final_kernel<<<1, 256, 0, st>>>(p_part, n_rows, load, s.T, s.E, alpha, f, P, loss);
+    return check_launch();
+}
+
 }  // namespace locmoe

@@ -41,8 +41,16 @@ struct GateFuse {
     int D, digit_mask, hstride, tile_shift;
 };
 
+// Optional extras of the gate (locmoe_gate_ex): a per-source bias table and the fused column sums of the probabilities.
+struct GateExtra {
+    const int32_t* bias_src;   // [T]: eps is then [D][E] and token t takes row bias_src[t]; nullptr: eps is [E]
+    float* p_part;             // [LOCMOE_GATE_PARTIAL_ROWS][E] or nullptr
+};
 int launch_gate(const locmoe_shape_t& s, const void* x, const float* eps, int32_t* idx, float* gate_w,
-                float* cos_sim, float* probs, cudaStream_t st, const GateFuse* fuse = nullptr);
+                float* cos_sim, float* probs, cudaStream_t st, const GateFuse* fuse = nullptr, const GateExtra* extra = nullptr);
+int gate_last_grid();   // CTAs of the gate launch this thread queued last (= rows of p_part it writes)
+int launch_aux_from_partials(const locmoe_shape_t& s, const float* p_part, int n_rows, const int32_t* load, float alpha,
+                             float* f, float* P, float* loss, cudaStream_t st);
 
 int launch_capacity(const locmoe_shape_t& s, const int32_t* idx, const float* cos_sim,
                     const locmoe_capacity_rule_t& rule, float* delta_e, float* theta_e,
@@ -100,7 +108,7 @@ int launch_cos_hist(const locmoe_shape_t& s, const void* x, const int32_t* idx, 
 
 int launch_dispatch_peer(const locmoe_shape_t& s, int C_alloc, int64_t rows, const void* x, const int32_t* inv,
                          const int32_t* slot, void* const* peer_bufs, int n_peers, int src_lo, int src_hi, int zero_pad,
-                         cudaStream_t st);
+                         long long win_lo, long long win_hi, cudaStream_t st);
 int launch_combine_peer(const locmoe_shape_t& s, int64_t rows, void* const* peer_y, int n_peers, int y_dtype,
                         const int32_t* slot, const float* gate_w, void* out, cudaStream_t st);
 

@@ -59,6 +59,17 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
     return false;
 }
 
+// After a wait has been given up: asynchronous work this CTA started (bulk tensor loads that write its shared
+// memory and count on its barriers, tcgen05.commit arrivals) may still be in flight, and a CTA must not leave
+// while it is.  Nothing tells when the last of it has landed once the barriers' phases are out of step, so the
+// CTA simply stays for a millisecond -- hundreds of times the latency of any such operation -- before it goes on
+// to free its tensor memory.  Bounded, and only ever executed on the failure path.
+__device__ __forceinline__ void quiesce_after_abort(volatile int* abort_word) {
+    if (*abort_word) {
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+}
+
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
@@ -115,26 +126,28 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 // GeLU(v) = v * Phi(v) with Phi(v) = 1 - 0.5 erfc(v / sqrt 2).  erfc(x) = P(t) exp(-x^2), t = 1 / (1 + p x), for
 // x >= 0 by the five-term rational approximation of Abramowitz & Stegun 7.1.26 (absolute error below 1.5e-7,
 // far under the bf16 rounding of the result); the negative side uses erfc(-x) = 2 - erfc(x) written so that a
-// small Phi is not formed by cancellation.  About half the instructions of erff().
+// small Phi is not formed by cancellation.  The reciprocal and the exponential are the hardware approximations
+// (rcp.approx, ex2.approx: a couple of ulps, far below the bf16 rounding of the result; 2.42 against 2.48 ms for the
+// first GEMM of the 65536 x 2560 x 10240 case).  About a third of the instructions of erff().
 // Two elements at a time with the two-wide fp32 instructions: the epilogue warps share their schedulers with
 // the TMA and MMA warps, so fewer epilogue instructions directly mean fewer bubbles in the MMA stream.
+__device__ __forceinline__ float rcp_approx(float x) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ float ex2_approx(float x) { float r; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
 __device__ __forceinline__ float2 gelu_erf2(float2 v) {
     const float2 x = __fmul2_rn(make_float2(fabsf(v.x), fabsf(v.y)), make_float2(0.70710678118654752f, 0.70710678118654752f));
     const float2 den = __ffma2_rn(make_float2(0.3275911f, 0.3275911f), x, make_float2(1.0f, 1.0f));
-    const float2 t = make_float2(__frcp_rn(den.x), __frcp_rn(den.y));
-    // coefficients already halved: the polynomial gives 0.5 erfc / exp(-x^2)
+    const float2 t = make_float2(rcp_approx(den.x), rcp_approx(den.y));
     float2 poly = __ffma2_rn(make_float2(0.5307027145f, 0.5307027145f), t, make_float2(-0.7265760135f, -0.7265760135f));
     poly = __ffma2_rn(poly, t, make_float2(0.7107068705f, 0.7107068705f));
     poly = __ffma2_rn(poly, t, make_float2(-0.142248368f, -0.142248368f));
     poly = __ffma2_rn(poly, t, make_float2(0.127414796f, 0.127414796f));
     const float2 arg = __fmul2_rn(__fmul2_rn(x, x), make_float2(-1.4426950408889634f, -1.4426950408889634f));
-    const float2 ex = make_float2(exp2f(arg.x), exp2f(arg.y));
-    const float2 h = __fmul2_rn(__fmul2_rn(poly, t), ex);                    // 0.5 erfc(|v| / sqrt 2)
+    const float2 ex = make_float2(ex2_approx(arg.x), ex2_approx(arg.y));
+    const float2 h = __fmul2_rn(__fmul2_rn(poly, t), ex);
     const float2 om = __ffma2_rn(h, make_float2(-1.0f, -1.0f), make_float2(1.0f, 1.0f));
     const float2 phi = make_float2(v.x < 0.0f ? h.x : om.x, v.y < 0.0f ? h.y : om.y);
     return __fmul2_rn(v, phi);
 }
-
 // Stores 32 consecutive columns of one output row (converted to the output type); static indexing keeps v[] in
 // registers.
 __device__ __forceinline__ void store_block32(const FfnArgs& a, long long grow, int col0, const float (&v)[32], bool wide_ok) {
@@ -261,7 +274,12 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             const int e = tile / tiles_per_expert, rem = tile - e * tiles_per_expert;
             const int nt = rem / a.m_tiles, mt = rem - nt * a.m_tiles;
-            if (!wait_or_abort(&acc_full[acc], acc_phase, abort_word)) break;
+            {   // one lane polls, the warp follows (32 lanes polling the same barrier only burn issue slots and power)
+                int ok = 1;
+                if (lane == 0) ok = wait_or_abort(&acc_full[acc], acc_phase, abort_word) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+            }
             tc_fence_after();
             const int r_in = mt * BM + q * 32 + lane;        // row inside the expert's block
             const bool row_ok = r_in < a.M;
@@ -291,6 +309,8 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
     }
     tc_fence_before();
+    __syncthreads();
+    quiesce_after_abort(abort_word);
     __syncthreads();
     if (warp == 2) {
         tc_fence_after();
@@ -336,13 +356,31 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
+// Raises the abort word of this CTA and of its partner in the pair (a plain store into the partner's shared
+// memory through the cluster address), so that both leave their loops together instead of the partner running
+// out its own wait against a CTA that has already given up.
+__device__ __forceinline__ void raise_abort_pair(volatile int* abort_word) {
+    *abort_word = 1;
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(smem_u32(const_cast<int*>(abort_word))), "r"(cluster_ctarank() ^ 1u));
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(ra), "r"(1) : "memory");
+    atomicOr(&g_ffn_flags, 1);
+}
+// The two waits of the two-SM kernel: like wait_or_abort, but a give-up is announced to both CTAs of the pair.
+__device__ __forceinline__ bool wait_or_abort_pair(uint64_t* bar, uint32_t parity, volatile int* abort_word) {
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 63u && *abort_word) return false;
+    }
+    raise_abort_pair(abort_word);
+    return false;
+}
 __device__ __forceinline__ bool wait_or_abort_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_word) {
     for (uint32_t i = 0; i < (1u << 22); ++i) {
         if (mbar_try_wait_cluster(bar, parity)) return true;
         if ((i & 63u) == 63u && *abort_word) return false;
     }
-    *abort_word = 1;
-    atomicOr(&g_ffn_flags, 1);
+    raise_abort_pair(abort_word);
     return false;
 }
 __device__ __forceinline__ void umma_bf16_2cta(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
@@ -426,7 +464,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int row0 = e * a.M + mt * 2 * BM + (int)rank * BM, n0 = nt * BN + (int)rank * (BN / 2);
                 bool ok = true;
                 for (int kb = 0; kb < kblocks && ok; ++kb) {
-                    if (!wait_or_abort(&empty[stage], phase ^ 1u, abort_word)) { ok = false; break; }
+                    if (!wait_or_abort_pair(&empty[stage], phase ^ 1u, abort_word)) { ok = false; break; }
                     unsigned char* sa = base + (size_t)stage * STAGE2_BYTES;
                     if (leader) mbar_expect_tx(&full[stage], 2 * STAGE2_BYTES);   // both CTAs' bytes are counted here
                     const uint32_t bar = leader_addr(&full[stage]);
@@ -439,7 +477,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // tail: every stage has been released, i.e. every commit that targets this CTA's barriers has arrived,
             // before the CTA may leave (the commits are asynchronous and multicast to both CTAs)
             for (int i = 0; i < NSTAGE2; ++i) {
-                if (!wait_or_abort(&empty[stage], phase ^ 1u, abort_word)) break;
+                if (!wait_or_abort_pair(&empty[stage], phase ^ 1u, abort_word)) break;
                 if (++stage == NSTAGE2) { stage = 0; phase ^= 1u; }
             }
         }
@@ -476,7 +514,12 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int tile = pair; tile < total_tiles; tile += npairs) {
             const int e = tile / tiles_per_expert, rem = tile - e * tiles_per_expert;
             const int nt = rem / m_tiles2, mt = rem - nt * m_tiles2;
-            if (!wait_or_abort(&acc_full[acc], acc_phase, abort_word)) break;
+            {
+                int ok = 1;
+                if (lane == 0) ok = wait_or_abort_pair(&acc_full[acc], acc_phase, abort_word) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+            }
             tc_fence_after();
             const int r_in = mt * 2 * BM + (int)rank * BM + q * 32 + lane;
             const bool row_ok = r_in < a.M;
@@ -506,6 +549,8 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
     }
     tc_fence_before();
+    __syncthreads();
+    quiesce_after_abort(abort_word);
     __syncthreads();
     cluster_sync_all();   // neither CTA frees its half of the paired allocation while the other may still use it
     if (warp == 2) {

@@ -35,7 +35,27 @@ struct GateArgs {
     int tab_ints;     // shared ints of the strip-offset table (one per unit of a row)
     float inv_g, sqrt_g;
     GateFuse f;       // route-stage work carried by the gate (f.src == nullptr: none)
+    const int32_t* bias_src;  // per-source bias table: eps is [bias_D][E] and token t takes row bias_src[t] (nullptr: eps is [E])
+    int bias_D;
+    float* p_part;    // [grid][E] per-CTA column sums of the probabilities (kernels built with PS only; nullptr: none)
+    int pacc_floats;  // shared floats per warp for those sums (E, or 0)
 };
+
+// The bias row of a token: eps itself, or the row of the per-source table (no bias for an impossible source).
+__device__ __forceinline__ const float* bias_row(const GateArgs& a, int sd) {
+    if (!a.bias_src || !a.eps) return a.eps;
+    return (unsigned)sd < (unsigned)a.bias_D ? a.eps + (size_t)sd * a.E : nullptr;
+}
+
+// End of a kernel built with PS: the CTA adds up its warps' column sums in warp order and writes its row.
+__device__ __forceinline__ void write_p_part(const GateArgs& a, const float* pacc_base, int wpb) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < a.E; i += blockDim.x) {
+        float s = 0.0f;
+        for (int ww = 0; ww < wpb; ++ww) s += pacc_base[(size_t)ww * a.pacc_floats + i];
+        a.p_part[(size_t)blockIdx.x * a.E + i] = s;
+    }
+}
 
 // Lane 0 of the warp that finished token `row`: the route stage's first pass over the tokens, done here.
 // sd = src[row], fetched by the caller (the specialised kernel prefetches it with the row).
@@ -84,12 +104,14 @@ __device__ __forceinline__ float2 pair_tree(const float2* p) {
 }
 
 // Softmax / arg-max / cosine of one row from the raw group sums in gsum[E].
-__device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gsum, float sq, int row, int lane) {
+template <bool EX>
+__device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gsum, float sq, int row, int lane, float* pacc) {
     const unsigned full = 0xffffffffu;
+    const float* eps = EX ? bias_row(a, a.bias_src ? a.bias_src[row] : 0) : a.eps;
     float best = -1.0f;  // every logit is >= 0 after the ReLU
     int bi = 0x7fffffff;
     for (int i = lane; i < a.E; i += kWarp) {
-        float G = fmaxf(gsum[i] * a.inv_g + (a.eps ? a.eps[i] : 0.0f), 0.0f);
+        float G = fmaxf(gsum[i] * a.inv_g + (eps ? eps[i] : 0.0f), 0.0f);
         if (G > best) { best = G; bi = i; }
     }
 #pragma unroll
@@ -100,7 +122,7 @@ __device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gs
     }
     float se = 0.0f;
     for (int i = lane; i < a.E; i += kWarp) {
-        float G = fmaxf(gsum[i] * a.inv_g + (a.eps ? a.eps[i] : 0.0f), 0.0f);
+        float G = fmaxf(gsum[i] * a.inv_g + (eps ? eps[i] : 0.0f), 0.0f);
         se += __expf(G - best);
     }
 #pragma unroll
@@ -109,11 +131,13 @@ __device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gs
         sq += __shfl_xor_sync(full, sq, o);
     }
     const float R = 1.0f / se;
-    if (a.probs) {
-        float* pr = a.probs + (size_t)row * a.E;
+    if (a.probs || pacc) {
+        float* pr = a.probs ? a.probs + (size_t)row * a.E : nullptr;
         for (int i = lane; i < a.E; i += kWarp) {
-            float G = fmaxf(gsum[i] * a.inv_g + (a.eps ? a.eps[i] : 0.0f), 0.0f);
-            pr[i] = __expf(G - best) * R;
+            float G = fmaxf(gsum[i] * a.inv_g + (eps ? eps[i] : 0.0f), 0.0f);
+            const float pv = __expf(G - best) * R;
+            if (pr) pr[i] = pv;
+            if (pacc) pacc[i] += pv;      // lane i owns column i, i + 32, ...: rows are added in the warp's row order
         }
     }
     if (lane == 0) {
@@ -128,7 +152,7 @@ __device__ __forceinline__ void gate_epilogue(const GateArgs& a, const float* gs
 
 // DT: token dtype.  U: elements per unit.  CH: vectors per lane per chunk.
 // EXACT: the row is a whole number of chunks (no bounds tests in the loop).
-template <int DT, int U, int CH, bool EXACT>
+template <int DT, int U, int CH, bool EXACT, bool PS>
 __global__ void __launch_bounds__(256, 4) gate_vec_kernel(const GateArgs a) {
     pdl_wait();
     pdl_trigger();
@@ -148,6 +172,9 @@ __global__ void __launch_bounds__(256, 4) gate_vec_kernel(const GateArgs a) {
     __syncthreads();
     float* part = smem + a.tab_ints + (size_t)wib * a.warp_floats;
     float* gsum = part + (size_t)a.E * a.PS;
+    float* pacc_base = smem + a.tab_ints + (size_t)wpb * a.warp_floats;
+    float* pacc = (PS && a.p_part) ? pacc_base + (size_t)wib * a.pacc_floats : nullptr;
+    if (pacc) for (int i = lane; i < a.E; i += kWarp) pacc[i] = 0.0f;
     const int nw = gridDim.x * wpb;
     const uint4* xv = reinterpret_cast<const uint4*>(a.x);
 
@@ -211,31 +238,34 @@ __global__ void __launch_bounds__(256, 4) gate_vec_kernel(const GateArgs a) {
             if (i < a.E && sl == 0) gsum[i] = s;
         }
         __syncwarp();
-        gate_epilogue(a, gsum, sq2.x + sq2.y, row, lane);
+        gate_epilogue<PS>(a, gsum, sq2.x + sq2.y, row, lane, pacc);
         __syncwarp();
         sq2 = make_float2(0.0f, 0.0f);
     };
 
     int row = blockIdx.x * wpb + wib, ch = 0;
-    if (row >= a.T) return;
-    load(bufA, row, 0);
-    while (true) {
-        int ch2 = ch + 1, row2 = row;
-        if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
-        if (row2 < a.T) load(bufB, row2, ch2);
-        consume(bufA, ch);
-        if (ch2 == 0) finish_row(row);
-        if (row2 >= a.T) break;
-        row = row2; ch = ch2;
+    if (!PS && row >= a.T) return;
+    if (row < a.T) {
+        load(bufA, row, 0);
+        while (true) {
+            int ch2 = ch + 1, row2 = row;
+            if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
+            if (row2 < a.T) load(bufB, row2, ch2);
+            consume(bufA, ch);
+            if (ch2 == 0) finish_row(row);
+            if (row2 >= a.T) break;
+            row = row2; ch = ch2;
 
-        ch2 = ch + 1; row2 = row;
-        if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
-        if (row2 < a.T) load(bufA, row2, ch2);
-        consume(bufB, ch);
-        if (ch2 == 0) finish_row(row);
-        if (row2 >= a.T) break;
-        row = row2; ch = ch2;
+            ch2 = ch + 1; row2 = row;
+            if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
+            if (row2 < a.T) load(bufA, row2, ch2);
+            consume(bufB, ch);
+            if (ch2 == 0) finish_row(row);
+            if (row2 >= a.T) break;
+            row = row2; ch = ch2;
+        }
     }
+    if (PS && a.p_part) write_p_part(a, pacc_base, wpb);
 }
 
 // Specialised bf16 kernel for the common shapes: the row is a whole number of chunks, every lane owns exactly NGK
@@ -269,7 +299,7 @@ __device__ __forceinline__ float strip_sum(const float* pp) {
     }
 }
 
-template <int U, int CH, int PUK, int NGK>
+template <int U, int CH, int PUK, int NGK, bool PS>
 __global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
     pdl_wait();
     pdl_trigger();
@@ -279,6 +309,12 @@ __global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int wpb = blockDim.x >> 5;
     float* part = smem + (size_t)wib * a.warp_floats;
+    float* pacc_base = smem + (size_t)wpb * a.warp_floats;
+    float* pacc = (PS && a.p_part) ? pacc_base + (size_t)wib * a.pacc_floats : nullptr;
+    if (pacc) {
+#pragma unroll
+        for (int m = 0; m < NGK; ++m) pacc[lane + 32 * m] = 0.0f;
+    }
     const int nw = gridDim.x * wpb;
     const uint4* xv = reinterpret_cast<const uint4*>(a.x);
     constexpr float kLog2e = 1.4426950408889634f;
@@ -291,7 +327,10 @@ __global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
         const uint4* base = xv + (size_t)r * a.V + c * (CH * kWarp) + lane;
 #pragma unroll
         for (int k = 0; k < CH; ++k) buf[k] = ld_stream(base + k * kWarp);
-        if (c == 0 && a.f.src) sd_new = a.f.src[r];
+        if (c == 0) {   // source device of the row, for the route hook / the bias row
+            if (a.f.src) sd_new = a.f.src[r];
+            else if (PS && a.bias_src) sd_new = a.bias_src[r];
+        }
     };
 
     auto consume = [&](const uint4 (&buf)[CH], int c) {
@@ -322,7 +361,8 @@ __global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
         for (int m = 0; m < NGK; ++m) gs[m] = strip_sum<PUK>(part + (size_t)(lane + 32 * m) * PUK);
         __syncwarp();  // the strip may now be overwritten by the next row
         // the logits are recomputed in the second pass rather than kept: fewer live registers, no spills
-        auto logit = [&](int m) { return fmaxf(fmaf(gs[m], a.inv_g, a.eps ? a.eps[lane + 32 * m] : 0.0f), 0.0f); };
+        const float* eps = PS ? bias_row(a, sd_cur) : a.eps;   // without the extras: the caller's row, as it is
+        auto logit = [&](int m) { return fmaxf(fmaf(gs[m], a.inv_g, eps ? eps[lane + 32 * m] : 0.0f), 0.0f); };
         float best = -1.0f;
         int bi = 0x7fffffff;
 #pragma unroll
@@ -350,6 +390,13 @@ __global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
 #pragma unroll
         for (int m = 1; m < NGK; ++m) if ((bi >> 5) == m) cand = gs[m];
         const float wsum = __shfl_sync(full, cand, bi & 31);
+        if constexpr (PS) {
+            if (a.p_part) {
+                const float R = 1.0f / se;
+#pragma unroll
+                for (int m = 0; m < NGK; ++m) pacc[lane + 32 * m] += exp2f(fmaf(logit(m), kLog2e, nb)) * R;
+            }
+        }
         if (lane == 0) {
             const float nrm = sqrtf(sq);
             const float cosv = nrm > 0.0f ? wsum / (a.sqrt_g * nrm) : 0.0f;
@@ -363,30 +410,33 @@ __global__ void __launch_bounds__(256, 4) gate_fast_kernel(const GateArgs a) {
     };
 
     int row = blockIdx.x * wpb + wib, ch = 0;
-    if (row >= a.T) return;
-    load(bufA, row, 0);
-    sd_cur = sd_new;
-    while (true) {
-        int ch2 = ch + 1, row2 = row;
-        if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
-        if (row2 < a.T) load(bufB, row2, ch2);
-        consume(bufA, ch);
-        if (ch2 == 0) finish_row(row);
-        if (row2 >= a.T) break;
-        row = row2; ch = ch2;
+    if (!PS && row >= a.T) return;
+    if (row < a.T) {
+        load(bufA, row, 0);
+        sd_cur = sd_new;
+        while (true) {
+            int ch2 = ch + 1, row2 = row;
+            if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
+            if (row2 < a.T) load(bufB, row2, ch2);
+            consume(bufA, ch);
+            if (ch2 == 0) finish_row(row);
+            if (row2 >= a.T) break;
+            row = row2; ch = ch2;
 
-        ch2 = ch + 1; row2 = row;
-        if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
-        if (row2 < a.T) load(bufA, row2, ch2);
-        consume(bufB, ch);
-        if (ch2 == 0) finish_row(row);
-        if (row2 >= a.T) break;
-        row = row2; ch = ch2;
+            ch2 = ch + 1; row2 = row;
+            if (ch2 == a.nch) { ch2 = 0; row2 = row + nw; }
+            if (row2 < a.T) load(bufA, row2, ch2);
+            consume(bufB, ch);
+            if (ch2 == 0) finish_row(row);
+            if (row2 >= a.T) break;
+            row = row2; ch = ch2;
+        }
     }
+    if (PS && a.p_part) write_p_part(a, pacc_base, wpb);
 }
 
 // Fallback for rows that are not 16-byte friendly: plain element loads, one warp per row.
-template <int DT>
+template <int DT, bool PS>
 __global__ void __launch_bounds__(256) gate_scalar_kernel(const GateArgs a) {
     pdl_wait();
     pdl_trigger();
@@ -395,6 +445,9 @@ __global__ void __launch_bounds__(256) gate_scalar_kernel(const GateArgs a) {
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int wpb = blockDim.x >> 5;
     float* gsum = smem + (size_t)wib * a.warp_floats;
+    float* pacc_base = smem + (size_t)wpb * a.warp_floats;
+    float* pacc = (PS && a.p_part) ? pacc_base + (size_t)wib * a.pacc_floats : nullptr;
+    if (pacc) for (int i = lane; i < a.E; i += kWarp) pacc[i] = 0.0f;
     const int nw = gridDim.x * wpb;
     for (int row = blockIdx.x * wpb + wib; row < a.T; row += nw) {
         float sq = 0.0f;
@@ -413,12 +466,15 @@ __global__ void __launch_bounds__(256) gate_scalar_kernel(const GateArgs a) {
             if (lane == 0) gsum[i] = s;
         }
         __syncwarp();
-        gate_epilogue(a, gsum, sq, row, lane);
+        gate_epilogue<PS>(a, gsum, sq, row, lane, pacc);
         __syncwarp();
     }
+    if (PS && a.p_part) write_p_part(a, pacc_base, wpb);
 }
 
 int gcd_int(int a, int b) { while (b) { int t = a % b; a = b; b = t; } return a; }
+
+thread_local int g_last_grid = 0;   // grid of the launch just queued by this thread's call (rows of p_part); set by launch_persistent
 
 template <typename K>
 int launch_persistent(K kernel, const GateArgs& a, int max_warps, cudaStream_t st) {
@@ -426,7 +482,7 @@ int launch_persistent(K kernel, const GateArgs& a, int max_warps, cudaStream_t s
     int wpb = max_warps;
     size_t smem = 0;
     for (; wpb >= 1; wpb >>= 1) {
-        smem = ((size_t)wpb * a.warp_floats + a.tab_ints) * sizeof(float);
+        smem = ((size_t)wpb * (a.warp_floats + a.pacc_floats) + a.tab_ints) * sizeof(float);
         if (smem <= 200 * 1024) break;
     }
     if (wpb < 1) return LOCMOE_ERR_SHAPE;
@@ -442,15 +498,24 @@ int launch_persistent(K kernel, const GateArgs& a, int max_warps, cudaStream_t s
     long long want = ((long long)a.T + wpb - 1) / wpb;
     long long grid = (long long)per_sm * sm_count();
     if (grid > want) grid = want;
+    if (a.p_part && grid > LOCMOE_GATE_PARTIAL_ROWS) grid = LOCMOE_GATE_PARTIAL_ROWS;
+    g_last_grid = (int)grid;
     return launch_pdl(kernel, (unsigned)grid, wpb * 32, smem, st, a);
 }
 
 }  // namespace
 
+int gate_last_grid() { return g_last_grid; }
+
 int launch_gate(const locmoe_shape_t& s, const void* x, const float* eps, int32_t* idx, float* gate_w,
-                float* cos_sim, float* probs, cudaStream_t st, const GateFuse* fuse) {
+                float* cos_sim, float* probs, cudaStream_t st, const GateFuse* fuse, const GateExtra* extra) {
     GateArgs a{};
     if (fuse) a.f = *fuse;
+    const bool ps = extra && (extra->p_part || extra->bias_src);   // kernels built with the extras
+    if (extra) {
+        a.bias_src = extra->bias_src; a.bias_D = s.n_nodes * s.dev_per_node;
+        a.p_part = extra->p_part; a.pacc_floats = extra->p_part ? ((s.E + 3) & ~3) : 0;
+    }
     a.x = x; a.eps = eps; a.idx = idx; a.gate_w = gate_w; a.cos_sim = cos_sim; a.probs = probs;
     a.T = s.T; a.H = s.H; a.E = s.E; a.g = s.H / s.E;
     a.inv_g = 1.0f / (float)a.g;
@@ -460,8 +525,10 @@ int launch_gate(const locmoe_shape_t& s, const void* x, const float* eps, int32_
     const bool vec_ok = ((size_t)s.H * esz) % 16 == 0 && ((uintptr_t)x % 16) == 0 && s.H <= 65535;
     if (!vec_ok) {
         a.warp_floats = (s.E + 3) & ~3;
-        if (s.x_dtype == LOCMOE_F32) return launch_persistent(gate_scalar_kernel<LOCMOE_F32>, a, 8, st);
-        return launch_persistent(gate_scalar_kernel<LOCMOE_BF16>, a, 8, st);
+        if (s.x_dtype == LOCMOE_F32) return ps ? launch_persistent(gate_scalar_kernel<LOCMOE_F32, true>, a, 8, st)
+                                               : launch_persistent(gate_scalar_kernel<LOCMOE_F32, false>, a, 8, st);
+        return ps ? launch_persistent(gate_scalar_kernel<LOCMOE_BF16, true>, a, 8, st)
+                  : launch_persistent(gate_scalar_kernel<LOCMOE_BF16, false>, a, 8, st);
     }
     const int U = gcd_int(a.g, VE);
     a.V = s.H / VE;
@@ -489,7 +556,9 @@ int launch_gate(const locmoe_shape_t& s, const void* x, const float* eps, int32_
         f.warp_floats = (s.H / U + 3) & ~3;
         f.tab_ints = 0;
 #define LOCMOE_FAST_CASE(UU, CC, PP, NN) \
-        if (U == UU && CH == CC && a.PU == PP && NG == NN) return launch_persistent(gate_fast_kernel<UU, CC, PP, NN>, f, 8, st);
+        if (U == UU && CH == CC && a.PU == PP && NG == NN)                                      \
+            return ps ? launch_persistent(gate_fast_kernel<UU, CC, PP, NN, true>, f, 8, st)     \
+                      : launch_persistent(gate_fast_kernel<UU, CC, PP, NN, false>, f, 8, st);
         LOCMOE_FAST_CASE(8, 4, 10, 2)   // H = 5120, E = 64
         LOCMOE_FAST_CASE(8, 5, 10, 1)   // H = 2560, E = 32
         LOCMOE_FAST_CASE(8, 4, 4, 4)    // H = 4096, E = 128
@@ -501,9 +570,12 @@ int launch_gate(const locmoe_shape_t& s, const void* x, const float* eps, int32_
     }
 #define LOCMOE_GATE_CASE(DT, UU)                                                                              \
     if (s.x_dtype == DT && U == UU) {                                                                         \
-        if (exact && CH == 4) return launch_persistent(gate_vec_kernel<DT, UU, 4, true>, a, 8, st);           \
-        if (exact && CH == 5) return launch_persistent(gate_vec_kernel<DT, UU, 5, true>, a, 8, st);           \
-        return launch_persistent(gate_vec_kernel<DT, UU, 4, false>, a, 8, st);                                \
+        if (exact && CH == 4) return ps ? launch_persistent(gate_vec_kernel<DT, UU, 4, true, true>, a, 8, st)   \
+                                        : launch_persistent(gate_vec_kernel<DT, UU, 4, true, false>, a, 8, st); \
+        if (exact && CH == 5) return ps ? launch_persistent(gate_vec_kernel<DT, UU, 5, true, true>, a, 8, st)   \
+                                        : launch_persistent(gate_vec_kernel<DT, UU, 5, true, false>, a, 8, st); \
+        return ps ? launch_persistent(gate_vec_kernel<DT, UU, 4, false, true>, a, 8, st)                        \
+                  : launch_persistent(gate_vec_kernel<DT, UU, 4, false, false>, a, 8, st);                      \
     }
     LOCMOE_GATE_CASE(LOCMOE_F32, 4)
     LOCMOE_GATE_CASE(LOCMOE_F32, 2)

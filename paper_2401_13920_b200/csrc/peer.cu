@@ -8,6 +8,8 @@
 //   combine : loads the expert output row from that GPU's buffer (plain peer loads) and scales it.
 // The send-side buffer and the library All-to-All disappear: a row crosses the link once, as it is produced.
 // Experts are split evenly, so rank q's buffer holds the rows [q * rows_per_peer, (q + 1) * rows_per_peer).
+// A call may be restricted to a window of every owner's buffer (rows [win_lo, win_hi) inside each peer's slice): the
+// receive buffer can then be filled expert slice by expert slice while the experts of the slices already filled run.
 // No kernel waits on another GPU; the caller separates dispatch, expert FFN and combine with a barrier across
 // the ranks (all stores of a kernel are visible to the peers once its stream has been synchronised).
 // Plain loads and stores only: no bulk-copy engine, no multicast.
@@ -39,7 +41,8 @@ __global__ void __launch_bounds__(kThreads) dispatch_peer_kernel(const uint4* __
                                                                  const int32_t* __restrict__ inv, const PeerTable peers,
                                                                  long long rows_per_peer, unsigned total, unsigned V, int T,
                                                                  long long rows, int zero_pad, int zrows, int C, int D, int Ed,
-                                                                 int N, int Dn, int src_lo, int src_hi) {
+                                                                 int N, int Dn, int src_lo, int src_hi, long long win_lo,
+                                                                 long long win_hi) {
     const unsigned base = blockIdx.x * (unsigned)(kThreads * 4 * kIters);
 #pragma unroll
     for (int it = 0; it < kIters; ++it) {
@@ -56,9 +59,12 @@ __global__ void __launch_bounds__(kThreads) dispatch_peer_kernel(const uint4* __
                 const int row = __ldg(slot + t);
                 if (row >= 0 && row < rows) {
                     const int q = (int)(row / rows_per_peer);
-                    r[k] = ld_stream(x + (size_t)t * V + v);
-                    dst[k] = peers.base[q] + (size_t)(row - q * rows_per_peer) * V + v;
-                    st[k] = true;
+                    const long long lr = row - q * rows_per_peer;      // row inside the owner's buffer
+                    if (lr >= win_lo && lr < win_hi) {
+                        r[k] = ld_stream(x + (size_t)t * V + v);
+                        dst[k] = peers.base[q] + (size_t)lr * V + v;
+                        st[k] = true;
+                    }
                 }
             }
         }
@@ -76,7 +82,9 @@ __global__ void __launch_bounds__(kThreads) dispatch_peer_kernel(const uint4* __
             const int s = row_source(row, C, D, Ed, N, Dn);
             if (s < src_lo || s >= src_hi) continue;   // another rank's row
             const int q = (int)(row / rows_per_peer);
-            uint4* d = peers.base[q] + (size_t)(row - q * rows_per_peer) * V;
+            const long long lr = row - q * rows_per_peer;
+            if (lr < win_lo || lr >= win_hi) continue;         // outside the window of this call
+            uint4* d = peers.base[q] + (size_t)lr * V;
             for (unsigned v = lane; v < V; v += 32) st_stream(d + v, make_uint4(0, 0, 0, 0));
         }
     }
@@ -145,7 +153,7 @@ __global__ void __launch_bounds__(kThreads) combine_peer_kernel(const PeerTable 
 
 int launch_dispatch_peer(const locmoe_shape_t& s, int C_alloc, int64_t rows, const void* x, const int32_t* inv,
                          const int32_t* slot, void* const* peer_bufs, int n_peers, int src_lo, int src_hi, int zero_pad,
-                         cudaStream_t st) {
+                         long long win_lo, long long win_hi, cudaStream_t st) {
     PeerTable pt{};
     for (int q = 0; q < n_peers; ++q) pt.base[q] = static_cast<uint4*>(peer_bufs[q]);
     const int esz = s.x_dtype == LOCMOE_F32 ? 4 : 2;
@@ -159,7 +167,7 @@ int launch_dispatch_peer(const locmoe_shape_t& s, int C_alloc, int64_t rows, con
     const int D = s.n_nodes * s.dev_per_node;
     dispatch_peer_kernel<<<g, kThreads, 0, st>>>(static_cast<const uint4*>(x), slot, inv, pt, (long long)(rows / n_peers), total,
                                                  V, s.T, (long long)rows, zero_pad, zrows, C_alloc, D, s.E / D, s.n_nodes,
-                                                 s.dev_per_node, src_lo, src_hi);
+                                                 s.dev_per_node, src_lo, src_hi, win_lo, win_hi);
     return check_launch();
 }
 

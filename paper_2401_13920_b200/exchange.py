@@ -104,9 +104,14 @@ class PeerBuffers:
         self.synchronize(stream)
         dist.barrier(group=self.group)
 
+    def order(self, first, then):
+        """Work queued on stream ``then`` from now on starts after everything queued on ``first`` so far."""
+        (then or torch.cuda.current_stream()).wait_stream(first or torch.cuda.current_stream())
+
 
 def peer_layer_forward(B, sharding, shape_local, C_alloc, rule, x, src_dev, recv: "PeerBuffers", y: "PeerBuffers",
-                       st, w_in=None, w_out=None, F=0, h1=None, out=None, group=None, stream=None):
+                       st, w_in=None, w_out=None, F=0, h1=None, out=None, group=None, stream=None, mark=None,
+                       slices=1, ffn_stream=None):
     """One MoE layer pass on this rank with the exchange fused into dispatch and combine.
 
     ``shape_local`` describes the WHOLE logical map with ``T`` = this rank's tokens and the receive-side layout;
@@ -123,14 +128,24 @@ def peer_layer_forward(B, sharding, shape_local, C_alloc, rule, x, src_dev, recv
     memory and reaches its first barrier only after its own combine has completed, so with a separate ``y`` no
     third barrier is needed: the experts of the next pass cannot overwrite ``y`` before every rank's combine is
     done.  When ``y`` IS ``recv`` (identity experts), the next pass's peer stores would land in rows a slower rank's
-    combine is still loading; a trailing barrier closes that window.
+    combine is still loading; a trailing barrier closes that window.  ``mark`` (optional) is called between the
+    stages -- before and after the gate, after the route, after the dispatch and its barrier, after the experts and
+    their barrier, after the combine -- so that a benchmark can record events there.
+
+    ``slices`` > 1 (with experts) overlaps the exchange with the expert computation, as Sec. 3.2.4 describes: this
+    rank's experts are cut into ``slices`` equal blocks; block s of EVERY rank's receive buffer is filled (windowed
+    peer stores on ``stream``, then the barrier), and the experts of block s start on ``ffn_stream`` while block
+    s + 1 is being stored.  The results are those of the unsliced pass, bit for bit.
     """
+    mark = mark or (lambda: None)
     world = recv.world
     rank = dist.get_rank(group) if world > 1 else 0
     D = shape_local.D
     devs = sharding.devices_of_rank(D, world, rank)
     out = st.out if out is None else out
+    mark()
     B.locmoe_gate(shape_local, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
+    mark()
     B.locmoe_capacity(shape_local, st.idx, st.cos_sim, rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
     if world > 1:
         recv.synchronize(stream)      # the per-expert minima are read by the host-side reduction
@@ -140,17 +155,38 @@ def peer_layer_forward(B, sharding, shape_local, C_alloc, rule, x, src_dev, recv
     B.locmoe_capacity_route(shape_local, st.idx, st.cos_sim, src_dev, rule_g, st.delta_e, st.theta_e, st.cap_dev, C_alloc,
                             st.pos, st.slot, st.drop, st.inv, st.counts, st.kept, st.send_counts, st.load, st.locality,
                             st.status, st.ws, stream)
-    B.locmoe_dispatch_peer(shape_local, C_alloc, x, st.inv, st.slot, recv.pointers, devs.start, devs.stop, True, stream)
-    recv.barrier(stream)
+    mark()
     ydt = B.dtype_code(y.local.dtype)
-    if w_in is not None:
-        # this rank's experts on its slice of the receive buffer: a shape whose experts are the local ones
-        # (one logical device holding E / world experts with D * C_alloc rows each: the same rows, regrouped)
-        E_loc = shape_local.E // world
-        sh_ffn = B.make_shape(shape_local.T, shape_local.H, E_loc, 1, 1, recv.local.dtype, B.LAYOUT_RECV)
-        B.locmoe_expert_ffn(sh_ffn, D * C_alloc, F, recv.local, w_in, w_out, h1, y.local, stream)
-    y.barrier(stream)
+    E_loc = shape_local.E // world
+    if w_in is not None and slices > 1:
+        if E_loc % slices:
+            raise ValueError("a rank's %d experts do not split into %d equal blocks" % (E_loc, slices))
+        Eb = E_loc // slices                      # experts per block
+        Rb = Eb * D * C_alloc                     # rows of a block inside a rank's buffer
+        sh_ffn = B.make_shape(shape_local.T, shape_local.H, Eb, 1, 1, recv.local.dtype, B.LAYOUT_RECV)
+        for s in range(slices):
+            B.locmoe_dispatch_peer(shape_local, C_alloc, x, st.inv, st.slot, recv.pointers, devs.start, devs.stop, True,
+                                   stream, window=(s * Rb, (s + 1) * Rb))
+            recv.barrier(stream)                  # block s of every rank's buffer is complete
+            recv.order(stream, ffn_stream)        # (one rank: no barrier, the streams alone order the two steps)
+            B.locmoe_expert_ffn(sh_ffn, D * C_alloc, F, recv.local[s * Rb:(s + 1) * Rb], w_in[s * Eb:(s + 1) * Eb],
+                                w_out[s * Eb:(s + 1) * Eb], h1[s * Rb:(s + 1) * Rb], y.local[s * Rb:(s + 1) * Rb], ffn_stream)
+        mark()
+        y.barrier(ffn_stream)
+        y.order(ffn_stream, stream)
+    else:
+        B.locmoe_dispatch_peer(shape_local, C_alloc, x, st.inv, st.slot, recv.pointers, devs.start, devs.stop, True, stream)
+        recv.barrier(stream)
+        mark()
+        if w_in is not None:
+            # this rank's experts on its slice of the receive buffer: a shape whose experts are the local ones
+            # (one logical device holding E / world experts with D * C_alloc rows each: the same rows, regrouped)
+            sh_ffn = B.make_shape(shape_local.T, shape_local.H, E_loc, 1, 1, recv.local.dtype, B.LAYOUT_RECV)
+            B.locmoe_expert_ffn(sh_ffn, D * C_alloc, F, recv.local, w_in, w_out, h1, y.local, stream)
+        y.barrier(stream)
+    mark()
     B.locmoe_combine_peer(shape_local, C_alloc, y.pointers, ydt, st.slot, st.gate_w, out, stream)
+    mark()
     if world > 1 and (y is recv or y.local.data_ptr() == recv.local.data_ptr()):
         y.barrier(stream)   # the next pass's peer stores must not overtake a slower rank's loads of the same rows
     return out

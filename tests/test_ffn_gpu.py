@@ -8,11 +8,18 @@ the oracle) the deviation from the fp64 oracle is bounded, with wide margin, by
   + 2^-8 * |y_i|               (final bf16 rounding, half an ulp is at most |y| / 256)
   + 1e-6 * sum-scale           (fp32 accumulation).
 """
+import os
+
 import numpy as np
 import pytest
 import torch
 
 pytestmark = pytest.mark.gpu
+
+# The two-SM kernel is opt-in in the library (LOCMOE_FFN=2) and therefore in the tests as well: its launches failed
+# under multi-metric profiler captures for a reason that has not been found, so a default test run leaves it alone.
+# LOCMOE_TEST_FFN2=1 runs its cases.
+two_sm = pytest.mark.skipif(os.environ.get("LOCMOE_TEST_FFN2") != "1", reason="two-SM FFN kernel is opt-in (LOCMOE_TEST_FFN2=1)")
 
 
 @pytest.fixture(scope="module")
@@ -48,7 +55,7 @@ def _check_rows(P, buf, w_in, w_out, y, E, M, rows, y_is_bf16=True):
     (4, 2, 2, 70, 264, 520, torch.float32),
     (8, 1, 8, 40, 512, 1024, torch.bfloat16),    # M = 320, several k-blocks and n-tiles
 ])
-@pytest.mark.parametrize("kernel", ["one_sm", "two_sm_single_acc", "two_sm"])
+@pytest.mark.parametrize("kernel", ["one_sm", pytest.param("two_sm_single_acc", marks=two_sm), pytest.param("two_sm", marks=two_sm)])
 def test_expert_ffn_small_shapes_all_rows(P, monkeypatch, kernel, E, N, Dn, C, H, F, ydt):
     # LOCMOE_FFN=2 selects the two-SM kernel (cluster of two CTAs, tcgen05 cta_group::2), 2s its one-accumulator form
     if kernel != "one_sm":
@@ -83,7 +90,7 @@ def test_expert_ffn_rejects_send_layout_and_bad_sizes(P):
     assert B._lib.locmoe_expert_ffn(C.byref(sh), 4, 64, C.c_void_p(8), one, one, one, one, B.BF16, None) == -4
 
 
-@pytest.mark.parametrize("kernel", ["one_sm", "two_sm"])
+@pytest.mark.parametrize("kernel", ["one_sm", pytest.param("two_sm", marks=two_sm)])
 def test_full_layer_config5_scaled(P, monkeypatch, kernel):
     # config 5: router + dispatch (RECV layout), expert FFN with random-init weights, combine; one C-ABI call
     if kernel == "two_sm":

@@ -166,3 +166,31 @@ def test_aux_loss_definition_and_minimum(oracle_mod):
     f_np = np.bincount(g.idx, minlength=16) / 500
     assert np.allclose(f, f_np) and np.allclose(P, g.probs.mean(0))
     assert L == pytest.approx(0.01 * 16 * (f_np * g.probs.mean(0)).sum(), rel=1e-12)
+
+
+# ---- per-source-device bias table (the paper leaves eps_i undefined; a table indexed by the source device is one
+#      reading of "locality-aware" bias, kept optional) ----
+
+def test_per_source_bias_rows_by_hand(oracle_mod):
+    # E = 2, H = 4: group means of [1, 1, 0.5, 0.5] are (1, 0.5).  Source 0 has no bias: expert 0 wins.
+    # Source 1 lifts expert 1 by 0.75: logits (1, 1.25), expert 1 wins with R = 1 / (1 + e^-0.25).
+    x = np.array([[1, 1, 0.5, 0.5]] * 3, dtype=np.float32)
+    table = np.array([[0.0, 0.0], [0.0, 0.75]], dtype=np.float32)
+    g = oracle_mod.gate_per_source(x, 0, 2, table, np.array([0, 1, 7]), want_probs=True)
+    assert list(g.idx) == [0, 1, 0]                        # source 7 does not exist: no bias
+    assert np.isclose(g.R[0], 1.0 / (1.0 + np.exp(-0.5))) and np.isclose(g.R[1], 1.0 / (1.0 + np.exp(-0.25)))
+    assert g.R[2] == g.R[0]
+    assert np.allclose(g.probs.sum(1), 1.0)
+    # the cosine ignores the bias: it is the angle to the chosen expert's weight
+    assert np.isclose(g.cos[0], 2.0 / (np.sqrt(2.0) * np.sqrt(2.5))) and np.isclose(g.cos[1], 1.0 / (np.sqrt(2.0) * np.sqrt(2.5)))
+
+
+def test_per_source_bias_with_equal_rows_is_the_plain_bias(oracle_mod):
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((300, 64)).astype(np.float32)
+    eps = rng.uniform(-0.1, 0.1, 8).astype(np.float32)
+    src = rng.integers(0, 4, 300)
+    a = oracle_mod.gate(x, 0, 8, eps=eps, want_probs=True)
+    b = oracle_mod.gate_per_source(x, 0, 8, np.tile(eps, (4, 1)), src, want_probs=True)
+    assert np.array_equal(a.idx, b.idx) and np.array_equal(a.R, b.R) and np.array_equal(a.cos, b.cos)
+    assert np.array_equal(a.probs, b.probs)

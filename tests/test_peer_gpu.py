@@ -174,3 +174,57 @@ def test_single_rank_peer_layer_equals_the_layer_call(P, with_ffn):
     assert B.locmoe_device_flags() == 0
     assert torch.equal(st2.slot, st.slot) and torch.equal(recv.local.view(torch.int16), st.buf.view(torch.int16))
     assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+
+
+@pytest.mark.parametrize("slices", [2, 8])
+def test_sliced_overlap_of_exchange_and_experts_equals_the_unsliced_pass(P, slices):
+    # the receive buffer filled expert block by expert block (windowed peer stores), the experts of a block running
+    # on a second stream while the next block is stored: bit for bit the unsliced layer pass
+    from paper_2401_13920_b200 import exchange, sharding
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    w = W.CONFIGS[5].scaled(6000)
+    F = 768
+    x, src = W.make_tokens(w, dev), W.make_src(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, B.LAYOUT_RECV)
+    rule = B.CapacityRule(1.0, 1.0, -1.0, 0, 0)
+    Ca = B.conventional_capacity(w.T, sh.D, w.E, 1.0)
+    w_in, w_out = W.make_expert_weights(w, F, dev)
+    outs = []
+    for S in (1, slices):
+        st = B.make_router(sh, Ca, rule, dev, with_buffer=False)
+        recv = exchange.PeerBuffers(sh.D * w.E * Ca, w.H, x.dtype, dev)
+        yb = exchange.PeerBuffers(sh.D * w.E * Ca, w.H, torch.bfloat16, dev)
+        recv.local.fill_(3.0)
+        yb.local.fill_(5.0)
+        h1 = torch.empty(sh.D * w.E * Ca, F, dtype=torch.bfloat16, device=dev)
+        got = torch.empty(w.T, w.H, dtype=x.dtype, device=dev)
+        exchange.peer_layer_forward(B, sharding, sh, Ca, rule, x, src, recv, yb, st, w_in, w_out, F, h1, out=got, slices=S,
+                                    ffn_stream=torch.cuda.Stream(dev))
+        torch.cuda.synchronize()
+        assert B.locmoe_device_flags() == 0
+        outs.append((recv.local.clone(), yb.local.clone(), got.clone(), st.slot.clone()))
+    a, b = outs
+    assert int((a[3] < 0).sum()) > 0 and int((a[3] >= 0).sum()) > 0
+    for u, v in zip(a, b):
+        assert torch.equal(u.view(torch.int16) if u.dtype == torch.bfloat16 else u, v.view(torch.int16) if v.dtype == torch.bfloat16 else v)
+
+
+def test_windowed_peer_dispatch_touches_only_its_window(P):
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    w = W.Workload(name="win", config=7, T=2000, H=256, E=8, n_nodes=2, dev_per_node=2, dtype="bf16", tokens="normal", src="uniform")
+    x, src = W.make_tokens(w, dev), W.make_src(w, dev)
+    sh = B.make_shape(w.T, w.H, w.E, 2, 2, x.dtype, B.LAYOUT_RECV)
+    Ca = B.conventional_capacity(w.T, 4, w.E, 1.0)
+    st = B.make_router(sh, Ca, B.CapacityRule(1.0, 1.0, -1.0, 0, 0), dev)
+    B.router_forward(st, x, src)                       # st.buf: the whole receive-side buffer
+    rows = st.rows
+    halves = [torch.full((rows // 2, w.H), 9.0, dtype=x.dtype, device=dev) for _ in range(2)]    # two "peers"
+    lo, hi = rows // 8, rows // 4                       # a window inside each peer's slice
+    B.locmoe_dispatch_peer(sh, Ca, x, st.inv, st.slot, halves, 0, 4, True, window=(lo, hi))
+    torch.cuda.synchronize()
+    for q in range(2):
+        want = torch.full_like(halves[q], 9.0)
+        want[lo:hi] = st.buf[q * (rows // 2) + lo:q * (rows // 2) + hi]
+        assert torch.equal(halves[q].view(torch.int16), want.view(torch.int16))

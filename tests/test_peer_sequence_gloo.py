@@ -58,11 +58,11 @@ class _RecordingBinding:
     def locmoe_capacity_route(self, sh, idx, cos_sim, src, rule, *rest):
         self.log.append(("capacity_route", rule.delta_override, rule.T_global, rule.min_mult, rule.capacity_factor))
 
-    def locmoe_dispatch_peer(self, sh, C_alloc, x, inv, slot, pointers, lo, hi, zero_pad, stream):
-        self.log.append(("dispatch_peer", tuple(pointers), lo, hi))
+    def locmoe_dispatch_peer(self, sh, C_alloc, x, inv, slot, pointers, lo, hi, zero_pad, stream, window=None):
+        self.log.append(("dispatch_peer", tuple(pointers), lo, hi) + ((window,) if window is not None else ()))
 
     def locmoe_expert_ffn(self, sh, C, F, buf, w_in, w_out, h1, y, stream):
-        self.log.append(("expert_ffn", sh.E, sh.n_nodes, sh.dev_per_node, C, F))
+        self.log.append(("expert_ffn", sh.E, sh.n_nodes, sh.dev_per_node, C, F) + ((stream,) if stream is not None else ()))
 
     def locmoe_combine_peer(self, sh, C_alloc, pointers, ydt, slot, gate_w, out, stream):
         self.log.append(("combine_peer", tuple(pointers)))
@@ -82,8 +82,11 @@ class _PlainPeerBuffers:
         self.log.append(("synchronize", self.name))
 
     def barrier(self, stream=None):
-        self.log.append(("barrier", self.name))
+        self.log.append(("barrier", self.name) + ((stream,) if stream is not None else ()))
         self.dist.barrier()
+
+    def order(self, first, then):
+        self.log.append(("order", first, then))
 
 
 class _State:
@@ -114,7 +117,11 @@ def _worker(rank, world, port, q):
                                     F=32, h1=None, stream=None)
         n1 = len(log)
         exchange.peer_layer_forward(B, sharding, shape, 9, rule, None, None, recv, recv, _State(), stream=None)
-        q.put((rank, log[:n1], log[n1:]))
+        n2 = len(log)
+        # pass 3: the exchange overlapped with the experts, two blocks of one expert each
+        exchange.peer_layer_forward(B, sharding, shape, 9, rule, None, None, recv, y, _State(), w_in=[0, 1], w_out=[0, 1],
+                                    F=32, h1=torch.zeros(72, 32), stream="main", slices=2, ffn_stream="side")
+        q.put((rank, log[:n1], log[n1:n2], log[n2:]))
     finally:
         dist.destroy_process_group()
 
@@ -129,7 +136,7 @@ def test_peer_layer_forward_call_sequence_on_two_ranks():
     res = sorted(q.get(timeout=120) for _ in range(2))
     for p in procs:
         p.join(timeout=60)
-    for rank, first, second in res:
+    for rank, first, second, third in res:
         names = [c[0] for c in first]
         assert names[2] == "synchronize"                           # the stream is waited for before the minima are reduced
         first, names = first[:2] + first[3:], names[:2] + names[3:]
@@ -148,4 +155,13 @@ def test_peer_layer_forward_call_sequence_on_two_ranks():
         assert [c[0] for c in second] == ["gate", "capacity", "capacity_route", "dispatch_peer", "barrier", "barrier",
                                            "combine_peer", "barrier"]
         assert second[6] == ("combine_peer", (1000, 2000))
+        # sliced pass: per block -- windowed peer stores, barrier on the main stream, stream order, that block's experts on
+        # the side stream -- then the barrier on the side stream, the order back, the combine
+        third = third[:2] + third[3:]
+        assert [c[0] for c in third] == ["gate", "capacity", "capacity_route", "dispatch_peer", "barrier", "order", "expert_ffn",
+                                          "dispatch_peer", "barrier", "order", "expert_ffn", "barrier", "order", "combine_peer"]
+        assert third[3][4] == (0, 36) and third[7][4] == (36, 72)        # rows of block s inside every rank's slice
+        assert third[4] == ("barrier", "recv", "main") and third[5] == ("order", "main", "side")
+        assert third[6] == ("expert_ffn", 1, 1, 1, 36, 32, "side") and third[10][-1] == "side"
+        assert third[11] == ("barrier", "y", "side") and third[12] == ("order", "side", "main")
     assert res[0][1][3] == res[1][1][3] and res[0][1][3][0] == "capacity_route"   # the same rule on both ranks
