@@ -146,12 +146,15 @@ def peer_layer_forward(B, sharding, shape_local, C_alloc, rule, x, src_dev, recv
     mark()
     B.locmoe_gate(shape_local, x, None, st.idx, st.gate_w, st.cos_sim, None, stream)
     mark()
-    B.locmoe_capacity(shape_local, st.idx, st.cos_sim, rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
+    rule_g = rule
     if world > 1:
+        # the whole batch's rule: per-rank minima, then All-Reduce MIN / SUM across the ranks (host side)
+        B.locmoe_capacity(shape_local, st.idx, st.cos_sim, rule, st.delta_e, st.theta_e, st.cap_dev, st.ws, stream)
         recv.synchronize(stream)      # the per-expert minima are read by the host-side reduction
-    delta, T_global = sharding.global_capacity_inputs(st.delta_e, shape_local.T, group)
-    rule_g = B.CapacityRule(rule.min_mult, rule.capacity_factor, delta if rule.delta_override < 0 else rule.delta_override,
-                            rule.bound_form, T_global)
+        delta, T_global = sharding.global_capacity_inputs(st.delta_e, shape_local.T, group)
+        rule_g = B.CapacityRule(rule.min_mult, rule.capacity_factor, delta if rule.delta_override < 0 else rule.delta_override,
+                                rule.bound_form, T_global)
+    # (one rank: its tokens are the batch, the fused call measures delta itself and nothing is read back)
     B.locmoe_capacity_route(shape_local, st.idx, st.cos_sim, src_dev, rule_g, st.delta_e, st.theta_e, st.cap_dev, C_alloc,
                             st.pos, st.slot, st.drop, st.inv, st.counts, st.kept, st.send_counts, st.load, st.locality,
                             st.status, st.ws, stream)
