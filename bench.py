@@ -37,7 +37,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", type=int, default=2, help="workload 1..5 (default 2, the metric's configuration)")
-    ap.add_argument("--cf", type=float, default=1.0, help="capacity factor (both knobs)")
+    ap.add_argument("--cf", type=float, default=1.0,
+                    help="capacity factor (both knobs); 0 = the literal-minimum mode: Theorem 1's minimum alone (multiplier 1)")
     ap.add_argument("--layout", choices=["send", "recv"], default="send")
     ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -158,7 +159,7 @@ def oracle_step(oracle, xh, srch, dtype_code, w, cf, layout):
     """One pass of the whole path in the CPU oracle on host arrays; returns kept tokens."""
     T = xh.shape[0]
     g = oracle.gate(xh, dtype_code, w.E)
-    cap = oracle.capacity(g.idx, g.cos, w.E, w.H, w.D, min_mult=cf, capacity_factor=cf)
+    cap = oracle.capacity(g.idx, g.cos, w.E, w.H, w.D, min_mult=cf if cf > 0 else 1.0, capacity_factor=cf)
     C = cap.C_local
     r = oracle.route(g.idx, srch, w.E, w.n_nodes, w.dev_per_node, C, C, layout)
     rows = w.D * w.E * C
@@ -256,7 +257,7 @@ def measure(args, w, env, *, steps, warmup, stage_steps, use_ffn, variant, fuse_
     x = W.make_tokens(w, dev)
     src = W.make_src(w, dev)
     shape = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype, layout)
-    rule = B.CapacityRule(args.cf, args.cf, -1.0, B.BOUND_BETA, 0)
+    rule = B.CapacityRule(args.cf if args.cf > 0 else 1.0, args.cf, -1.0, B.BOUND_BETA, 0)   # c_f = 0: the minimum alone
     C_alloc = B.conventional_capacity(w.T, shape.D, w.E, args.cf)
     st = B.make_router(shape, C_alloc, rule, dev)
     y = None
@@ -724,12 +725,14 @@ def main():
     default_headline = args.config == 2 and args.tokens == 0 and variant == "router" and not args.fuse_gate and not args.unfused
     if world == 1 and default_headline and not args.no_other_configs:
         others = {}
-        for name, cfg, ffn in (("config1", 1, False), ("config3", 3, False), ("config4", 4, False),
-                               ("config5_router_only", 5, False), ("config5_with_ffn", 5, True)):
+        for name, cfg, ffn, cf in (("config1", 1, False, args.cf), ("config3", 3, False, args.cf), ("config4", 4, False, args.cf),
+                                   ("config5_router_only", 5, False, args.cf), ("config5_with_ffn", 5, True, args.cf),
+                                   ("config2_literal_minimum_capacity", 2, False, 0.0)):
             gc.collect()
             torch.cuda.empty_cache()
             try:
-                mo = measure(args, workload(cfg), env, steps=args.other_steps, warmup=5, stage_steps=args.stage_steps,
+                args_o = argparse.Namespace(**{**vars(args), "cf": cf})
+                mo = measure(args_o, workload(cfg), env, steps=args.other_steps, warmup=5, stage_steps=args.stage_steps,
                              use_ffn=ffn, variant="router", fuse_gate=False, fused=True, e2e_steps=0, cpu_baseline_s=0.0)
                 others[name] = summary_of(mo)
                 del mo
