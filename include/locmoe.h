@@ -126,6 +126,10 @@ int locmoe_workspace_bytes(const locmoe_shape_t *shape, int32_t C_alloc, size_t 
  *   gate_w[t] = softmax(G)[idx[t]]                   (Eq. "gating_score")
  *   cos_sim[t] = <w_idx, x_t> / (|w_idx| |x_t|)      (Lemma 1; 0 for a zero token)
  *   probs[t][i] = softmax(G)_i                       (optional, NULL to skip)
+ * Tokens are expected to be finite.  A token with an infinity or a NaN in it gets
+ * unspecified score and cosine (possibly NaN) and a valid expert index in [0, E);
+ * it does not disturb any other token's outputs, and nothing faults.  A NaN cosine
+ * may or may not enter its expert's minimum in locmoe_capacity.
  * x: [T][H] of shape->x_dtype.  The fast path needs x 16-byte aligned and
  * H * sizeof(element) a multiple of 16; other inputs take a slower scalar path.
  * idx int32[T], gate_w / cos_sim float[T], probs float[T][E], eps float[E].

@@ -291,6 +291,42 @@ def test_bad_source_device_is_dropped_and_flagged(P):
     assert not st.out[7].any().item()
 
 
+def test_non_finite_tokens_stay_local_to_their_rows(P):
+    # infinities / NaNs in a few tokens: every other token's outputs are bit for bit those of the clean batch, the
+    # poisoned tokens still get an expert index in range, and the routing stays a valid placement
+    W, B = P.W, P.B
+    dev = torch.device("cuda:0")
+    for kw in (dict(T=3000, H=5120, E=64, n_nodes=8, dev_per_node=8), dict(T=2000, H=60, E=4, n_nodes=1, dev_per_node=4, dtype="f32")):
+        w = _wl(P, **kw)
+        x, src = W.make_tokens(w, dev), W.make_src(w, dev)
+        sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype)
+        Ca = B.conventional_capacity(w.T, sh.D, w.E, 1.0)
+        rule = B.CapacityRule(1.0, 1.0, 0.01, 0, 0)          # a fixed threshold: the capacity must not depend on the poison
+        clean = B.make_router(sh, Ca, rule, dev)
+        B.router_forward(clean, x, src)
+        torch.cuda.synchronize()
+        xp = x.clone()
+        bad = [3, 700, w.T - 1]
+        xp[3, 5] = float("inf")
+        xp[700, 0] = float("nan")
+        xp[w.T - 1, w.H - 1] = float("-inf")
+        xp[w.T - 1, 1] = float("inf")
+        st = B.make_router(sh, Ca, rule, dev)
+        B.router_forward(st, xp, src)
+        torch.cuda.synchronize()
+        assert B.locmoe_device_flags() == 0
+        good = torch.ones(w.T, dtype=torch.bool, device=dev)
+        good[bad] = False
+        for name in ("idx", "gate_w", "cos_sim"):
+            assert torch.equal(getattr(st, name)[good], getattr(clean, name)[good]), name
+        assert int(st.idx.min()) >= 0 and int(st.idx.max()) < w.E
+        keep = st.slot >= 0
+        assert len(torch.unique(st.slot[keep])) == int(keep.sum())                 # all slots distinct
+        assert torch.equal(st.inv[st.slot[keep].long()], torch.nonzero(keep).flatten().to(torch.int32))
+        assert int(st.kept.max()) <= B.locmoe_capacity_read(st.cap_dev).C_local
+        assert int(st.kept.sum()) + int(st.drop.sum()) == w.T
+
+
 def test_accumulate_adds_to_the_output(P):
     W, B = P.W, P.B
     w = _wl(P, T=900, H=256, E=8, n_nodes=2, dev_per_node=2, dtype="f32")
