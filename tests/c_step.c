@@ -5,7 +5,11 @@
  * end-to-end figure of the benchmark stands for; tests/test_c_step_gpu.py builds it, feeds it a
  * seeded batch and compares its output bit for bit with the Python binding's path.
  *
- *   c_step T H E n_nodes dev_per_node c_f x.bin src.bin out.bin slot.bin      (bf16 tokens)
+ *   c_step T H E n_nodes dev_per_node c_f x.bin src.bin out.bin slot.bin [graph]     (bf16 tokens)
+ *
+ * With the word "graph" as the last argument the four library calls are first run once eagerly, then captured
+ * into a CUDA graph (the library allocates nothing and never synchronises, so its calls can be captured), the
+ * outputs are overwritten with garbage, and the graph is replayed twice; the files hold the replay's result.
  */
 #include <stdint.h>
 #include <stdio.h>
@@ -35,7 +39,8 @@ static int write_file(const char *path, const void *src, size_t bytes) {
 }
 
 int main(int argc, char **argv) {
-    if (argc != 11) return 1;
+    if (argc != 11 && argc != 12) return 1;
+    const int use_graph = argc == 12;
     locmoe_shape_t s = {atoi(argv[1]), atoi(argv[2]), atoi(argv[3]), atoi(argv[4]), atoi(argv[5]), LOCMOE_BF16, LOCMOE_LAYOUT_SEND};
     const double cf = atof(argv[6]);
     locmoe_capacity_rule_t rule = {cf, cf, -1.0, LOCMOE_BOUND_BETA, 0};
@@ -66,11 +71,29 @@ int main(int argc, char **argv) {
     CK(cudaStreamCreate(&st));
     CK(cudaMemcpyAsync(x, xh, xb, cudaMemcpyHostToDevice, st));
     CK(cudaMemcpyAsync(src, srch, T * 4, cudaMemcpyHostToDevice, st));
-    LM(locmoe_gate(&s, x, NULL, idx, gate_w, cos_sim, NULL, st));
-    LM(locmoe_capacity_route(&s, idx, cos_sim, src, &rule, delta_e, theta_e, cap, C_alloc, pos, slot, drop, inv, counts, kept,
-                             send_counts, load, locality, status, 0, ws, ws_bytes, st));
-    LM(locmoe_dispatch(&s, C_alloc, x, inv, slot, buf, 1, st));
-    LM(locmoe_combine(&s, C_alloc, buf, LOCMOE_BF16, slot, gate_w, out, 0, st));
+#define STEP() do { \
+    LM(locmoe_gate(&s, x, NULL, idx, gate_w, cos_sim, NULL, st)); \
+    LM(locmoe_capacity_route(&s, idx, cos_sim, src, &rule, delta_e, theta_e, cap, C_alloc, pos, slot, drop, inv, counts, kept, \
+                             send_counts, load, locality, status, 0, ws, ws_bytes, st)); \
+    LM(locmoe_dispatch(&s, C_alloc, x, inv, slot, buf, 1, st)); \
+    LM(locmoe_combine(&s, C_alloc, buf, LOCMOE_BF16, slot, gate_w, out, 0, st)); } while (0)
+    STEP();
+    if (use_graph) {
+        cudaGraph_t graph;
+        cudaGraphExec_t exec;
+        CK(cudaStreamSynchronize(st));
+        CK(cudaStreamBeginCapture(st, cudaStreamCaptureModeGlobal));
+        STEP();
+        CK(cudaStreamEndCapture(st, &graph));
+        CK(cudaGraphInstantiate(&exec, graph, 0));
+        CK(cudaMemsetAsync(out, 0x5a, xb, st));
+        CK(cudaMemsetAsync(slot, 0x5a, T * 4, st));
+        CK(cudaGraphLaunch(exec, st));
+        CK(cudaGraphLaunch(exec, st));
+        CK(cudaStreamSynchronize(st));
+        CK(cudaGraphExecDestroy(exec));
+        CK(cudaGraphDestroy(graph));
+    }
     CK(cudaMemcpyAsync(outh, out, xb, cudaMemcpyDeviceToHost, st));
     CK(cudaMemcpyAsync(sloth, slot, T * 4, cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));

@@ -23,8 +23,8 @@ def _build_c_step(tmp_path):
     return exe
 
 
-@pytest.mark.parametrize("cfg,T,cf", [(2, 6000, 1.0), (5, 7001, 1.25)])
-def test_c_program_step_equals_the_binding_path(tmp_path, cfg, T, cf):
+@pytest.mark.parametrize("cfg,T,cf,graph", [(2, 6000, 1.0, False), (5, 7001, 1.25, False), (2, 6000, 1.0, True), (5, 7001, 1.25, True)])
+def test_c_program_step_equals_the_binding_path(tmp_path, cfg, T, cf, graph):
     if not torch.cuda.is_available():
         pytest.fail("GPU tests need a CUDA device")
     from paper_2401_13920_b200 import binding as B
@@ -36,7 +36,8 @@ def test_c_program_step_equals_the_binding_path(tmp_path, cfg, T, cf):
     W.host_bits(x).tofile(tmp_path / "x.bin")
     src.cpu().numpy().tofile(tmp_path / "src.bin")
     r = subprocess.run([str(exe), str(w.T), str(w.H), str(w.E), str(w.n_nodes), str(w.dev_per_node), repr(cf),
-                        str(tmp_path / "x.bin"), str(tmp_path / "src.bin"), str(tmp_path / "out.bin"), str(tmp_path / "slot.bin")],
+                        str(tmp_path / "x.bin"), str(tmp_path / "src.bin"), str(tmp_path / "out.bin"), str(tmp_path / "slot.bin")]
+                       + (["graph"] if graph else []),
                        capture_output=True, text=True, timeout=300)
     assert r.returncode == 0 and r.stdout.startswith("ok"), r.stdout + r.stderr
     sh = B.make_shape(w.T, w.H, w.E, w.n_nodes, w.dev_per_node, x.dtype)
