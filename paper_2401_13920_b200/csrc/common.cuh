@@ -66,7 +66,8 @@ struct RoutePlan {
     int hstride;      // row stride of the histogram matrices: ntiles rounded up to a multiple of 4
     int launches;     // kernel launches of one route call
     int prescan;      // 1: histogram matrices are prefix-scanned by a launch of their own (large batches)
-    size_t off_keys[2], off_toks[2], off_hist[4], off_keystart, off_rowbase, off_rowtot, off_cap_part, total;
+    int nrep;         // replicas of the per-key demand counters that the first pass adds to (few keys: many adds per address)
+    size_t off_keys[2], off_toks[2], off_hist[4], off_keystart, off_rowbase, off_rowtot, off_cap_part, off_counts_rep, total;
 };
 int plan_route(const locmoe_shape_t& s, RoutePlan* p);
 size_t capacity_ws_bytes(const locmoe_shape_t& s);

@@ -52,6 +52,8 @@ struct RouteArgs {
     uint32_t* keys[2];
     int32_t* toks[2];
     int32_t* hist[kMaxPasses];  // [1 << bits[p]][hstride], digit major
+    int32_t* counts_rep;        // [nrep][K] replicas of the demand counters (nrep > 1), summed into counts by the extras
+    int nrep;
     int32_t* keystart;          // [K]
     int32_t* rowbase;           // [K] first buffer row of the key's class
     int hstride, tile_shift;    // row stride of the histogram matrices (a multiple of 4 >= ntiles); log2(tile)
@@ -89,6 +91,8 @@ __global__ void __launch_bounds__(kThreads) route_init_kernel(const RouteArgs a,
     const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     for (long long i = i0; i < a.rows; i += stride) a.inv[i] = -1;
     for (long long i = i0; i < a.K; i += stride) a.counts[i] = 0;
+    if (a.nrep > 1)
+        for (long long i = i0; i < (long long)a.nrep * a.K; i += stride) a.counts_rep[i] = 0;
     for (long long i = i0; i < (long long)a.D * a.D; i += stride) a.send_counts[i] = 0;
     for (long long i = i0; i < a.E; i += stride) a.load[i] = 0;
     for (int p = a.hist_by_gate ? 0 : 1; p < a.passes; ++p) {
@@ -140,7 +144,10 @@ __global__ void __launch_bounds__(kThreads) route_hist0_kernel(const RouteArgs a
                 continue;
             }
             const int key = sd[u] * a.E + e[u];
-            atomicAdd(&a.counts[key], 1);
+            // few keys mean many adds per address (64 per key with 1024 keys and 65536 tokens, 3 us of serialised L2
+            // atomics): the tiles spread theirs over nrep copies, which the first extra CTA adds up
+            if (a.nrep > 1) atomicAdd(&a.counts_rep[(size_t)(blockIdx.x & (a.nrep - 1)) * a.K + key], 1);
+            else atomicAdd(&a.counts[key], 1);
             atomicAdd(&sh[(uint32_t)key & mask], 1);
         }
     }
@@ -193,6 +200,14 @@ __device__ void block_exclusive_scan(const int32_t* in, int32_t* out, int n) {
 // per-tile minima and evaluates the capacity rule (dyn = the CTA's dynamic shared memory, at least E words).
 __device__ void route_extras_a(const RouteArgs& a, int x, int nx, int* dyn) {
     if (x == 0) {
+        if (a.nrep > 1 && !a.hist_by_gate) {   // the replicas' sums are the demand counts
+            for (int k = threadIdx.x; k < a.K; k += kThreads) {
+                int c = 0;
+                for (int r = 0; r < a.nrep; ++r) c += __ldcg(a.counts_rep + (size_t)r * a.K + k);
+                a.counts[k] = c;
+            }
+            __syncthreads();
+        }
         block_exclusive_scan(a.counts, a.keystart, a.K);
         return;
     }
@@ -543,6 +558,9 @@ int plan_route(const locmoe_shape_t& s, RoutePlan* p) {
     p->off_rowbase = off; off += align256((size_t)K * 4);
     p->off_rowtot = off; off += 1024;
     p->off_cap_part = off; off += align256((size_t)(p->ntiles > 64 ? p->ntiles : 64) * s.E * 4);
+    p->nrep = 1;   // enough copies to bring the adds per address down to 16 (config 2's level, where one copy is fastest)
+    while (p->nrep < 8 && (long long)p->nrep * 2 * K <= 8192 && (long long)s.T > 16ll * K * p->nrep) p->nrep *= 2;
+    p->off_counts_rep = off; off += p->nrep > 1 ? align256((size_t)p->nrep * K * 4) : 0;
     p->total = off;
     p->prescan = ((long long)p->ntiles << p->bits[0]) > 32768 ? 1 : 0;
     {   // testing aid: LOCMOE_PATH=grid forces the large-batch variants at any size
@@ -596,6 +614,8 @@ static int launch_route_impl(const locmoe_shape_t& s, const int32_t* idx, const 
         a.bits[i] = p.bits[i];
         a.hist[i] = reinterpret_cast<int32_t*>(w + p.off_hist[i]);
     }
+    a.counts_rep = reinterpret_cast<int32_t*>(w + p.off_counts_rep);
+    a.nrep = gate ? 1 : p.nrep;
     a.keystart = reinterpret_cast<int32_t*>(w + p.off_keystart);
     a.rowbase = reinterpret_cast<int32_t*>(w + p.off_rowbase);
     a.hstride = p.hstride;
