@@ -725,11 +725,14 @@ def main():
     default_headline = args.config == 2 and args.tokens == 0 and variant == "router" and not args.fuse_gate and not args.unfused
     if world == 1 and default_headline and not args.no_other_configs:
         others = {}
-        for name, cfg, ffn, cf in (("config1", 1, False, args.cf), ("config3", 3, False, args.cf), ("config4", 4, False, args.cf),
-                                   ("config5_router_only", 5, False, args.cf), ("config5_with_ffn", 5, True, args.cf),
-                                   ("config2_literal_minimum_capacity", 2, False, 0.0)):
+        # the light configurations first, the power-hungry ones (config 4's 10 ms steps, the FFN) last, and a pause
+        # before each so that none inherits the clocks the power cap left its predecessor with
+        for name, cfg, ffn, cf in (("config1", 1, False, args.cf), ("config5_router_only", 5, False, args.cf),
+                                   ("config2_literal_minimum_capacity", 2, False, 0.0), ("config3", 3, False, args.cf),
+                                   ("config4", 4, False, args.cf), ("config5_with_ffn", 5, True, args.cf)):
             gc.collect()
             torch.cuda.empty_cache()
+            time.sleep(1.0)
             try:
                 args_o = argparse.Namespace(**{**vars(args), "cf": cf})
                 mo = measure(args_o, workload(cfg), env, steps=args.other_steps, warmup=5, stage_steps=args.stage_steps,
