@@ -9,6 +9,13 @@ batch on its own GPU (the path needs no exchange step on one logical-device
 map), so the reported value is the aggregate and scaling is weak.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--cf F] [--impl reference]
+                    [--variant router|peer8|topk2|peer] [--slices S] [--no-other-configs]
+
+The timed region is exactly K replays of the step (a CUDA graph); per-stage times come from a separate
+pass of eager steps with CUDA events between the stages (medians), the gate also launched on its own.
+The default line (config 2) also carries short runs of the other configurations (`other_configs`).
+`--variant peer` is the form with one rank per GPU and the exchange fused into dispatch and combine
+(peer stores / loads; N = 1 works on one GPU).  `--impl reference` times the CPU oracle instead.
 
 Prints ONE JSON line on rank 0.
 """
