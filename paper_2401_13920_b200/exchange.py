@@ -94,6 +94,19 @@ class PeerBuffers:
             self._handle = symm.rendezvous(self.local, group=group if group is not None else dist.group.WORLD)
             self.pointers = [int(p) for p in self._handle.buffer_ptrs]
 
+    @classmethod
+    def from_mappings(cls, local: torch.Tensor, pointers, group=None):
+        """Buffers whose peer mappings the caller obtained some other way (CUDA IPC handles, a driver-level
+        mapping): ``local`` is this rank's slice, ``pointers[q]`` the address of rank q's slice as valid on THIS GPU
+        (``pointers[rank]`` = ``local.data_ptr()``).  Same barrier / ordering behaviour as the symmetric-memory form."""
+        self = cls.__new__(cls)
+        self.group = group
+        self.world = len(pointers)
+        self.local = local
+        self.pointers = [int(p) for p in pointers]
+        self._handle = None
+        return self
+
     def synchronize(self, stream=None):
         """Waits for the stream that ran this rank's kernels (before the host reads their results or meets its peers)."""
         (stream or torch.cuda.current_stream()).synchronize()
