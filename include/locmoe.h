@@ -34,8 +34,11 @@
  *                                   a specialised one
  *       LOCMOE_DISPATCH=tma|vec|flat  dispatch: bulk-copy, warp-per-row or flat
  *                                   row-major kernel
- *       LOCMOE_FFN=2|2s             expert FFN: the two-SM kernel (2s: with one
- *                                   accumulator)
+ *       LOCMOE_FFN=1|w|w1|w2|2|2s   expert FFN: the 128 x 256-tile kernel for both
+ *                                   GEMMs, the 256 x 256-tile kernel for both / the
+ *                                   first / the second (default: chosen per GEMM by
+ *                                   its reduction length), the two-SM kernel (2s:
+ *                                   with one accumulator)
  *       LOCMOE_PDL=0                plain launches instead of programmatic
  *                                   dependent launches (read once per process)
  *       LOCMOE_DEBUG=1              print the CUDA error behind LOCMOE_ERR_CUDA

@@ -315,6 +315,155 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 }
 
 // =====================================================================================================
+// Wide form of the same GEMM: one CTA works on a 256 x 256 output tile as two 128 x 256 halves that share the
+// weight tile.  Per k-block 32 KB of activations (256 rows) and 32 KB of weights come in, and eight MMAs use them:
+// 64 KB per 1024 tensor-pipe cycles instead of 48 KB per 512, a third less data pulled out of L2 per flop.  The two
+// accumulators take all 512 TMEM columns, so a tile's epilogue no longer hides behind the next tile's MMAs except
+// for half a tile's worth at either end (each half has its own pair of barriers and the epilogue drains the upper
+// half first); that is the better trade where K is long.  Three stages of 64 KB.
+constexpr int NSTAGE_W = 3;
+constexpr int kWideMinK = 6144;   // shortest reduction for which the wide kernel is chosen by default
+constexpr uint32_t AW_BYTES = 2 * A_BYTES, STAGE_W_BYTES = AW_BYTES + B_BYTES;
+constexpr size_t kFfnWideSmem = (size_t)NSTAGE_W * STAGE_W_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+
+__global__ void __launch_bounds__(kFfnThreads, 1)
+ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const FfnArgs a) {
+    extern __shared__ unsigned char smraw[];
+    unsigned char* base = reinterpret_cast<unsigned char*>(((uintptr_t)smraw + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base + (size_t)NSTAGE_W * STAGE_W_BYTES);
+    uint64_t* full = bars;                     // [NSTAGE_W]
+    uint64_t* empty = bars + NSTAGE_W;         // [NSTAGE_W]
+    uint64_t* acc_full = bars + 2 * NSTAGE_W;  // [2] one per 128-row half
+    uint64_t* acc_empty = acc_full + 2;        // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile int* abort_word = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NSTAGE_W; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kEpiWarps); }
+        *abort_word = 0;
+        mbar_init_fence();
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int tiles_per_expert = a.m_tiles * a.n_tiles;   // m_tiles counts 256-row tiles here
+    const int total_tiles = a.E * tiles_per_expert;
+    const int kblocks = (a.K + BK - 1) / BK;
+
+    if (warp == 0) {
+        if (lane == 0) {  // ---- TMA producer: one 256-row box of A and one of B per k-block ----
+            int stage = 0; uint32_t phase = 0;
+            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+                const int e = tile / tiles_per_expert, rem = tile - e * tiles_per_expert;
+                const int nt = rem / a.m_tiles, mt = rem - nt * a.m_tiles;
+                const int row0 = e * a.M + mt * 2 * BM, n0 = nt * BN;
+                bool ok = true;
+                for (int kb = 0; kb < kblocks && ok; ++kb) {
+                    if (!wait_or_abort(&empty[stage], phase ^ 1u, abort_word)) { ok = false; break; }
+                    unsigned char* sa = base + (size_t)stage * STAGE_W_BYTES;
+                    mbar_expect_tx(&full[stage], STAGE_W_BYTES);
+                    tma_load_2d(sa, &tmA, kb * BK, row0, &full[stage]);
+                    tma_load_3d(sa + AW_BYTES, &tmB, kb * BK, n0, e, &full[stage]);
+                    if (++stage == NSTAGE_W) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+            }
+            for (int i = 0; i < NSTAGE_W; ++i) {   // every commit to this CTA's stage barriers has arrived
+                if (!wait_or_abort(&empty[stage], phase ^ 1u, abort_word)) break;
+                if (++stage == NSTAGE_W) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {  // ---- MMA issuer ----
+            int stage = 0; uint32_t phase = 0;
+            uint32_t acc_phase = 0;
+            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+                bool ok = true;
+                for (int kb = 0; kb < kblocks && ok; ++kb) {
+                    if (!wait_or_abort(&full[stage], phase, abort_word)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(base + (size_t)stage * STAGE_W_BYTES);
+                    const uint32_t sb = sa + AW_BYTES;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (kb == 0) {   // this half's accumulator has been drained
+                            if (!wait_or_abort(&acc_empty[h], acc_phase ^ 1u, abort_word)) { ok = false; break; }
+                            tc_fence_after();
+                        }
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; ++k)
+                            umma_bf16(tmem_base + (uint32_t)h * BN, umma_desc_sw128(sa + h * A_BYTES + k * UMMA_K * 2),
+                                      umma_desc_sw128(sb + k * UMMA_K * 2), (kb > 0 || k > 0) ? 1u : 0u);
+                        if (kb == kblocks - 1) umma_commit(&acc_full[h]);
+                    }
+                    if (!ok) break;
+                    umma_commit(&empty[stage]);
+                    if (++stage == NSTAGE_W) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                acc_phase ^= 1u;
+            }
+        }
+    } else {  // ---- epilogue warps 2..9: TMEM lane quadrant = warp % 4, column half = (warp - 2) / 4, both row halves ----
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
+        uint32_t acc_phase = 0;
+        const bool wide_ok = (a.N % 16 == 0) && ((uintptr_t)a.out % 32 == 0);
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            const int e = tile / tiles_per_expert, rem = tile - e * tiles_per_expert;
+            const int nt = rem / a.m_tiles, mt = rem - nt * a.m_tiles;
+            const int n0 = nt * BN;
+            bool ok = true;
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+                if (!wait_or_abort(&acc_full[h], acc_phase, abort_word)) { ok = false; break; }
+                tc_fence_after();
+                const int r_in = mt * 2 * BM + h * BM + q * 32 + lane;
+                const bool row_ok = r_in < a.M;
+                const long long grow = (long long)e * a.M + r_in;
+#pragma unroll 1
+                for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
+                    __syncwarp();
+                    uint32_t r[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * BN + c * 32), r);
+                    const int col0 = n0 + c * 32;
+                    if (!row_ok || col0 >= a.N) continue;
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float2 pr = make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                        if (a.gelu) pr = gelu_erf2(pr);
+                        v[i] = pr.x; v[i + 1] = pr.y;
+                    }
+                    store_block32(a, grow, col0, v, wide_ok);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[h]);
+            }
+            if (!ok) break;
+            acc_phase ^= 1u;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    quiesce_after_abort(abort_word);
+    __syncthreads();
+    if (warp == 2) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// =====================================================================================================
 // Two-SM form of the same GEMM: a cluster of two CTAs works on a 256 x 256 output tile.  Each CTA loads its own
 // 128 rows of A and only HALF of the B tile (128 of the 256 weight rows); tcgen05.mma.cta_group::2, issued by the
 // leader CTA (cluster rank 0), multiplies the 256 x 64 A (both CTAs' shared memory) by the 256 x 64 B (both halves)
@@ -613,6 +762,34 @@ int launch_gemm(const void* A, const void* W, void* out, int out_f32, int gelu, 
     return check_launch();
 }
 
+// Wide kernel: 256 x 256 tiles, one CTA each.
+int launch_gemm_wide(const void* A, const void* W, void* out, int out_f32, int gelu, int E, int M, int N, int K,
+                     cudaStream_t st) {
+    CUtensorMap tmA, tmB;
+    const uint64_t da[2] = {(uint64_t)K, (uint64_t)E * M};
+    const uint64_t db[3] = {(uint64_t)K, (uint64_t)N, (uint64_t)E};
+    if (!make_map(&tmA, A, 2, da, 2 * BM) || !make_map(&tmB, W, 3, db, BN)) return LOCMOE_ERR_CUDA;
+    FfnArgs a{};
+    a.out = out; a.out_f32 = out_f32; a.gelu = gelu; a.E = E; a.M = M; a.N = N; a.K = K;
+    a.m_tiles = (M + 2 * BM - 1) / (2 * BM);
+    a.n_tiles = (N + BN - 1) / BN;
+    static bool attr_done_dev[64] = {false};   // the attribute is per device
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!attr_done_dev[dev & 63]) {
+        if (cudaFuncSetAttribute(ffn_gemm_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFfnWideSmem) != cudaSuccess) {
+            cudaGetLastError();
+            return LOCMOE_ERR_CUDA;
+        }
+        attr_done_dev[dev & 63] = true;
+    }
+    const long long tiles = (long long)E * a.m_tiles * a.n_tiles;
+    int grid = sm_count();
+    if (tiles < grid) grid = (int)tiles;
+    ffn_gemm_wide_kernel<<<grid, kFfnThreads, kFfnWideSmem, st>>>(tmA, tmB, a);
+    return check_launch();
+}
+
 // Two-SM kernel.  nacc = 2: two accumulators per CTA (all 512 TMEM columns); nacc = 1: one (256 columns, the
 // epilogue does not overlap the next tile's MMAs).
 int launch_gemm2(const void* A, const void* W, void* out, int out_f32, int gelu, int E, int M, int N, int K, int nacc,
@@ -651,10 +828,15 @@ int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* 
                       const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st) {
     const int E = s.E;
     const int M = (int)(rows / E);
-    // LOCMOE_FFN=2 selects the two-SM kernel (4.68 ms against 4.81 ms for the one-SM kernel on E = 32, M = 2048,
-    // H = 2560, F = 10240 at full clocks), 2s its single-accumulator form.  It is opt-in: it passes every test and
-    // runs clean in the bench, but launches of it failed under multi-metric profiler captures for a reason that
-    // reading the code has not shown, so the one-SM kernel stays the default.
+    // Which kernel runs a GEMM.  By default the wide kernel (256 x 256 tiles, a third less operand traffic, the
+    // epilogue mostly exposed) where the reduction is long enough for the exposed epilogue not to matter and the
+    // rows of an expert fill its taller tiles as well as they fill the 128-row ones, else the 128 x 256 kernel.
+    // On E = 32, M = 2048, H = 2560, F = 10240, back to back under the power cap: second GEMM (K = 10240) 2.63
+    // against 2.77 ms, first GEMM (K = 2560, GeLU) 2.98 against 2.84 ms.
+    // LOCMOE_FFN (a testing aid) overrides: 1 = 128 x 256 kernel for both, w = wide for both, w1 / w2 = wide for
+    // the first / second GEMM only, 2 = the two-SM kernel (2s: its single-accumulator form).  The two-SM kernel is
+    // opt-in only: it passes every test and runs clean in the bench, but launches of it failed under multi-metric
+    // profiler captures for a reason that reading the code has not shown.
     const char* mode = getenv("LOCMOE_FFN");
     if (mode && mode[0] == '2' && sm_count() >= 2) {
         const int nacc = mode[1] == 's' ? 1 : 2;
@@ -662,9 +844,14 @@ int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* 
         if (rc) return rc;
         return launch_gemm2(h1, w_out, y, y_dtype == LOCMOE_F32 ? 1 : 0, 0, E, M, s.H, F, nacc, st);
     }
-    int rc = launch_gemm(buf, w_in, h1, 0, 1, E, M, F, s.H, st);
+    const bool fills = (M + 2 * BM - 1) / (2 * BM) * 2 == (M + BM - 1) / BM;   // no extra empty half tile
+    bool wide1 = fills && s.H >= kWideMinK, wide2 = fills && F >= kWideMinK;
+    if (mode && mode[0] == '1') wide1 = wide2 = false;
+    if (mode && mode[0] == 'w') { wide1 = mode[1] != '2'; wide2 = mode[1] != '1'; }
+    const int y_f32 = y_dtype == LOCMOE_F32 ? 1 : 0;
+    int rc = wide1 ? launch_gemm_wide(buf, w_in, h1, 0, 1, E, M, F, s.H, st) : launch_gemm(buf, w_in, h1, 0, 1, E, M, F, s.H, st);
     if (rc) return rc;
-    return launch_gemm(h1, w_out, y, y_dtype == LOCMOE_F32 ? 1 : 0, 0, E, M, s.H, F, st);
+    return wide2 ? launch_gemm_wide(h1, w_out, y, y_f32, 0, E, M, s.H, F, st) : launch_gemm(h1, w_out, y, y_f32, 0, E, M, s.H, F, st);
 }
 
 int read_ffn_flags(int* out, cudaStream_t st) {

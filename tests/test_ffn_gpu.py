@@ -54,12 +54,13 @@ def _check_rows(P, buf, w_in, w_out, y, E, M, rows, y_is_bf16=True):
     (4, 2, 2, 70, 264, 520, torch.bfloat16),     # M = 280, K and N with ragged tails
     (4, 2, 2, 70, 264, 520, torch.float32),
     (8, 1, 8, 40, 512, 1024, torch.bfloat16),    # M = 320, several k-blocks and n-tiles
+    (2, 1, 2, 300, 320, 512, torch.bfloat16),    # M = 600: three 256-row tiles, the last one with an empty lower half
 ])
-@pytest.mark.parametrize("kernel", ["one_sm", pytest.param("two_sm_single_acc", marks=two_sm), pytest.param("two_sm", marks=two_sm)])
+@pytest.mark.parametrize("kernel", ["one_sm", "wide", pytest.param("two_sm_single_acc", marks=two_sm), pytest.param("two_sm", marks=two_sm)])
 def test_expert_ffn_small_shapes_all_rows(P, monkeypatch, kernel, E, N, Dn, C, H, F, ydt):
     # LOCMOE_FFN=2 selects the two-SM kernel (cluster of two CTAs, tcgen05 cta_group::2), 2s its one-accumulator form
-    if kernel != "one_sm":
-        monkeypatch.setenv("LOCMOE_FFN", "2s" if kernel == "two_sm_single_acc" else "2")
+    # and w the wide kernel (256 x 256 tiles, one CTA each) for both GEMMs
+    monkeypatch.setenv("LOCMOE_FFN", {"one_sm": "1", "wide": "w", "two_sm_single_acc": "2s", "two_sm": "2"}[kernel])
     B = P.B
     dev = torch.device("cuda:0")
     D = N * Dn
@@ -90,11 +91,10 @@ def test_expert_ffn_rejects_send_layout_and_bad_sizes(P):
     assert B._lib.locmoe_expert_ffn(C.byref(sh), 4, 64, C.c_void_p(8), one, one, one, one, B.BF16, None) == -4
 
 
-@pytest.mark.parametrize("kernel", ["one_sm", pytest.param("two_sm", marks=two_sm)])
+@pytest.mark.parametrize("kernel", ["one_sm", "wide", pytest.param("two_sm", marks=two_sm)])
 def test_full_layer_config5_scaled(P, monkeypatch, kernel):
     # config 5: router + dispatch (RECV layout), expert FFN with random-init weights, combine; one C-ABI call
-    if kernel == "two_sm":
-        monkeypatch.setenv("LOCMOE_FFN", "2")
+    monkeypatch.setenv("LOCMOE_FFN", {"one_sm": "1", "wide": "w", "two_sm": "2"}[kernel])
     W, B = P.W, P.B
     dev = torch.device("cuda:0")
     w = W.CONFIGS[5].scaled(8192)
