@@ -844,8 +844,14 @@ int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* 
         if (rc) return rc;
         return launch_gemm2(h1, w_out, y, y_dtype == LOCMOE_F32 ? 1 : 0, 0, E, M, s.H, F, nacc, st);
     }
-    const bool fills = (M + 2 * BM - 1) / (2 * BM) * 2 == (M + BM - 1) / BM;   // no extra empty half tile
-    bool wide1 = fills && s.H >= kWideMinK, wide2 = fills && F >= kWideMinK;
+    // ... and the last wave of its twice-as-long tiles does not cost more than the wide tiles save (about 5 %)
+    const long long m1 = (M + BM - 1) / BM, m2 = (M + 2 * BM - 1) / (2 * BM), G = sm_count() > 0 ? sm_count() : 1;
+    auto pays = [&](int N, int K) {
+        const long long n = (N + BN - 1) / BN;
+        const long long waves_narrow = (E * m1 * n + G - 1) / G, waves_wide = (E * m2 * n + G - 1) / G;
+        return K >= kWideMinK && m2 * 2 == m1 && waves_wide * 2 * 19 <= waves_narrow * 20;
+    };
+    bool wide1 = pays(F, s.H), wide2 = pays(s.H, F);
     if (mode && mode[0] == '1') wide1 = wide2 = false;
     if (mode && mode[0] == 'w') { wide1 = mode[1] != '2'; wide2 = mode[1] != '1'; }
     const int y_f32 = y_dtype == LOCMOE_F32 ? 1 : 0;
