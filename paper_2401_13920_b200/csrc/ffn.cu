@@ -43,6 +43,7 @@ struct FfnArgs {
     int gelu;             // apply GeLU in the epilogue
     int E, M, N, K;       // experts, rows per expert, output columns, reduction length
     int m_tiles, n_tiles;
+    int split_from;       // wide kernel: tiles from this index on are worked on as two half tiles (see there)
 };
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
@@ -326,6 +327,16 @@ constexpr int kWideMinK = 6144;   // shortest reduction for which the wide kerne
 constexpr uint32_t AW_BYTES = 2 * A_BYTES, STAGE_W_BYTES = AW_BYTES + B_BYTES;
 constexpr size_t kFfnWideSmem = (size_t)NSTAGE_W * STAGE_W_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
+// Work item w of the wide kernel: a whole 256 x 256 tile (halves = 3) below split_from, one 128-row half of a tile
+// above it.  The last, partly filled wave of tiles is split in this way when its halves fit one wave: 148 CTAs
+// then finish after one more 128-row tile instead of one more 256-row tile.
+struct WideItem { int tile, halves; };
+__device__ __forceinline__ WideItem wide_item(const FfnArgs& a, int w) {
+    if (w < a.split_from) return {w, 3};
+    const int u = w - a.split_from;
+    return {a.split_from + (u >> 1), 1 << (u & 1)};
+}
+
 __global__ void __launch_bounds__(kFfnThreads, 1)
 ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const FfnArgs a) {
     extern __shared__ unsigned char smraw[];
@@ -356,12 +367,14 @@ ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
     const int tiles_per_expert = a.m_tiles * a.n_tiles;   // m_tiles counts 256-row tiles here
     const int total_tiles = a.E * tiles_per_expert;
+    const int total_items = a.split_from + 2 * (total_tiles - a.split_from);
     const int kblocks = (a.K + BK - 1) / BK;
 
     if (warp == 0) {
         if (lane == 0) {  // ---- TMA producer: one 256-row box of A and one of B per k-block ----
             int stage = 0; uint32_t phase = 0;
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            for (int w = blockIdx.x; w < total_items; w += gridDim.x) {
+                const int tile = wide_item(a, w).tile;   // a half-tile item loads the whole boxes all the same
                 const int e = tile / tiles_per_expert, rem = tile - e * tiles_per_expert;
                 const int nt = rem / a.m_tiles, mt = rem - nt * a.m_tiles;
                 const int row0 = e * a.M + mt * 2 * BM, n0 = nt * BN;
@@ -384,8 +397,9 @@ ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     } else if (warp == 1) {
         if (lane == 0) {  // ---- MMA issuer ----
             int stage = 0; uint32_t phase = 0;
-            uint32_t acc_phase = 0;
-            for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            uint32_t acc_phase[2] = {0, 0};
+            for (int w = blockIdx.x; w < total_items; w += gridDim.x) {
+                const int halves = wide_item(a, w).halves;
                 bool ok = true;
                 for (int kb = 0; kb < kblocks && ok; ++kb) {
                     if (!wait_or_abort(&full[stage], phase, abort_word)) { ok = false; break; }
@@ -394,8 +408,9 @@ ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     const uint32_t sb = sa + AW_BYTES;
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
+                        if (!((halves >> h) & 1)) continue;
                         if (kb == 0) {   // this half's accumulator has been drained
-                            if (!wait_or_abort(&acc_empty[h], acc_phase ^ 1u, abort_word)) { ok = false; break; }
+                            if (!wait_or_abort(&acc_empty[h], acc_phase[h] ^ 1u, abort_word)) { ok = false; break; }
                             tc_fence_after();
                         }
 #pragma unroll
@@ -409,22 +424,26 @@ ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     if (++stage == NSTAGE_W) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                acc_phase ^= 1u;
+                acc_phase[0] ^= (uint32_t)(halves & 1);
+                acc_phase[1] ^= (uint32_t)(halves >> 1);
             }
         }
     } else {  // ---- epilogue warps 2..9: TMEM lane quadrant = warp % 4, column half = (warp - 2) / 4, both row halves ----
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
-        uint32_t acc_phase = 0;
+        uint32_t acc_phase[2] = {0, 0};
         const bool wide_ok = (a.N % 16 == 0) && ((uintptr_t)a.out % 32 == 0);
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        for (int w = blockIdx.x; w < total_items; w += gridDim.x) {
+            const WideItem it = wide_item(a, w);
+            const int tile = it.tile;
             const int e = tile / tiles_per_expert, rem = tile - e * tiles_per_expert;
             const int nt = rem / a.m_tiles, mt = rem - nt * a.m_tiles;
             const int n0 = nt * BN;
             bool ok = true;
 #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
-                if (!wait_or_abort(&acc_full[h], acc_phase, abort_word)) { ok = false; break; }
+                if (!((it.halves >> h) & 1)) continue;
+                if (!wait_or_abort(&acc_full[h], acc_phase[h], abort_word)) { ok = false; break; }
                 tc_fence_after();
                 const int r_in = mt * 2 * BM + h * BM + q * 32 + lane;
                 const bool row_ok = r_in < a.M;
@@ -448,9 +467,9 @@ ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[h]);
+                acc_phase[h] ^= 1u;
             }
             if (!ok) break;
-            acc_phase ^= 1u;
         }
     }
     tc_fence_before();
@@ -785,6 +804,8 @@ int launch_gemm_wide(const void* A, const void* W, void* out, int out_f32, int g
     }
     const long long tiles = (long long)E * a.m_tiles * a.n_tiles;
     int grid = sm_count();
+    const long long tail = tiles % grid;   // tiles of the last, partly filled wave
+    a.split_from = (int)(tiles >= grid && tail > 0 && 2 * tail <= grid ? tiles - tail : tiles);
     if (tiles < grid) grid = (int)tiles;
     ffn_gemm_wide_kernel<<<grid, kFfnThreads, kFfnWideSmem, st>>>(tmA, tmB, a);
     return check_launch();
@@ -848,8 +869,10 @@ int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* 
     const long long m1 = (M + BM - 1) / BM, m2 = (M + 2 * BM - 1) / (2 * BM), G = sm_count() > 0 ? sm_count() : 1;
     auto pays = [&](int N, int K) {
         const long long n = (N + BN - 1) / BN;
-        const long long waves_narrow = (E * m1 * n + G - 1) / G, waves_wide = (E * m2 * n + G - 1) / G;
-        return K >= kWideMinK && m2 * 2 == m1 && waves_wide * 2 * 19 <= waves_narrow * 20;
+        const long long tw = E * m2 * n, tail = tw % G;
+        const long long waves_narrow = (E * m1 * n + G - 1) / G;                      // in 128-row tiles
+        const long long waves_wide = tw / G * 2 + (tail == 0 ? 0 : (tw >= G && 2 * tail <= G) ? 1 : 2);   // the same unit
+        return K >= kWideMinK && m2 * 2 == m1 && waves_wide * 19 <= waves_narrow * 20;
     };
     bool wide1 = pays(F, s.H), wide2 = pays(s.H, F);
     if (mode && mode[0] == '1') wide1 = wide2 = false;
