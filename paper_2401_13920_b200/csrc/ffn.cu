@@ -185,6 +185,28 @@ __device__ __forceinline__ void store_block32(const FfnArgs& a, long long grow, 
     }
 }
 
+// Epilogue of one warp on one accumulator: column blocks [c_begin, c_end) of 32 columns each, one row per lane
+// (TMEM lane = row).  taddr = the accumulator's TMEM address at this warp's lane quadrant, column 0.
+__device__ __forceinline__ void drain_columns(const FfnArgs& a, uint32_t taddr, long long grow, bool row_ok, int n0,
+                                              int c_begin, int c_end, bool wide_ok) {
+#pragma unroll 1
+    for (int c = c_begin; c < c_end; ++c) {
+        __syncwarp();  // tcgen05.ld is warp-collective: reconverge after the masked stores
+        uint32_t r[32];
+        tmem_ld32(taddr + (uint32_t)(c * 32), r);
+        const int col0 = n0 + c * 32;
+        if (!row_ok || col0 >= a.N) continue;
+        float v[32];
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+            float2 pr = make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+            if (a.gelu) pr = gelu_erf2(pr);
+            v[i] = pr.x; v[i + 1] = pr.y;
+        }
+        store_block32(a, grow, col0, v, wide_ok);
+    }
+}
+
 __global__ void __launch_bounds__(kFfnThreads, 1)
 ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const FfnArgs a) {
     extern __shared__ unsigned char smraw[];
@@ -283,22 +305,8 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const long long grow = (long long)e * a.M + r_in;
             const int n0 = nt * BN;
             const bool wide_ok = (a.N % 16 == 0) && ((uintptr_t)a.out % 32 == 0);
-#pragma unroll 1
-            for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
-                __syncwarp();  // tcgen05.ld is warp-collective: reconverge after the masked stores
-                uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
-                const int col0 = n0 + c * 32;
-                if (!row_ok || col0 >= a.N) continue;
-                float v[32];
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float2 pr = make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                    if (a.gelu) pr = gelu_erf2(pr);
-                    v[i] = pr.x; v[i + 1] = pr.y;
-                }
-                store_block32(a, grow, col0, v, wide_ok);
-            }
+            drain_columns(a, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), grow, row_ok, n0,
+                          half * (BN / 64), (half + 1) * (BN / 64), wide_ok);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[acc]);
@@ -397,7 +405,7 @@ ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     } else if (warp == 1) {
         if (lane == 0) {  // ---- MMA issuer ----
             int stage = 0; uint32_t phase = 0;
-            uint32_t acc_phase[2] = {0, 0};
+            uint32_t acc_phase = 0;   // bit h: phase of half h's accumulator barriers
             for (int w = blockIdx.x; w < total_items; w += gridDim.x) {
                 const int halves = wide_item(a, w).halves;
                 bool ok = true;
@@ -410,7 +418,7 @@ ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     for (int h = 0; h < 2; ++h) {
                         if (!((halves >> h) & 1)) continue;
                         if (kb == 0) {   // this half's accumulator has been drained
-                            if (!wait_or_abort(&acc_empty[h], acc_phase[h] ^ 1u, abort_word)) { ok = false; break; }
+                            if (!wait_or_abort(&acc_empty[h], ((acc_phase >> h) & 1u) ^ 1u, abort_word)) { ok = false; break; }
                             tc_fence_after();
                         }
 #pragma unroll
@@ -424,14 +432,13 @@ ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     if (++stage == NSTAGE_W) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                acc_phase[0] ^= (uint32_t)(halves & 1);
-                acc_phase[1] ^= (uint32_t)(halves >> 1);
+                acc_phase ^= (uint32_t)halves;
             }
         }
     } else {  // ---- epilogue warps 2..9: TMEM lane quadrant = warp % 4, column half = (warp - 2) / 4, both row halves ----
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
-        uint32_t acc_phase[2] = {0, 0};
+        uint32_t acc_phase = 0;   // bit h: phase of half h's accumulator barriers
         const bool wide_ok = (a.N % 16 == 0) && ((uintptr_t)a.out % 32 == 0);
         for (int w = blockIdx.x; w < total_items; w += gridDim.x) {
             const WideItem it = wide_item(a, w);
@@ -443,31 +450,17 @@ ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
                 if (!((it.halves >> h) & 1)) continue;
-                if (!wait_or_abort(&acc_full[h], acc_phase[h], abort_word)) { ok = false; break; }
+                if (!wait_or_abort(&acc_full[h], (acc_phase >> h) & 1u, abort_word)) { ok = false; break; }
                 tc_fence_after();
                 const int r_in = mt * 2 * BM + h * BM + q * 32 + lane;
                 const bool row_ok = r_in < a.M;
                 const long long grow = (long long)e * a.M + r_in;
-#pragma unroll 1
-                for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
-                    __syncwarp();
-                    uint32_t r[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * BN + c * 32), r);
-                    const int col0 = n0 + c * 32;
-                    if (!row_ok || col0 >= a.N) continue;
-                    float v[32];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float2 pr = make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                        if (a.gelu) pr = gelu_erf2(pr);
-                        v[i] = pr.x; v[i + 1] = pr.y;
-                    }
-                    store_block32(a, grow, col0, v, wide_ok);
-                }
+                drain_columns(a, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * BN), grow, row_ok, n0,
+                              half * (BN / 64), (half + 1) * (BN / 64), wide_ok);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&acc_empty[h]);
-                acc_phase[h] ^= 1u;
+                acc_phase ^= 1u << h;
             }
             if (!ok) break;
         }
@@ -685,22 +678,8 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const long long grow = (long long)e * a.M + r_in;
             const int n0 = nt * BN;
             const bool wide_ok = (a.N % 16 == 0) && ((uintptr_t)a.out % 32 == 0);
-#pragma unroll 1
-            for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
-                __syncwarp();
-                uint32_t r[32];
-                tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
-                const int col0 = n0 + c * 32;
-                if (!row_ok || col0 >= a.N) continue;
-                float v[32];
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float2 pr = make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                    if (a.gelu) pr = gelu_erf2(pr);
-                    v[i] = pr.x; v[i + 1] = pr.y;
-                }
-                store_block32(a, grow, col0, v, wide_ok);
-            }
+            drain_columns(a, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN), grow, row_ok, n0,
+                          half * (BN / 64), (half + 1) * (BN / 64), wide_ok);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(&acc_empty[acc], 0);
