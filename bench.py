@@ -734,8 +734,12 @@ def main():
         others = {}
         # the light configurations first, the power-hungry ones (config 4's 10 ms steps, the FFN) last, and a pause
         # before each so that none inherits the clocks the power cap left its predecessor with
-        for name, cfg, ffn, cf in (("config1", 1, False, args.cf), ("config5_router_only", 5, False, args.cf),
+        for name, cfg, ffn, cf in (("config1", 1, False, args.cf), ("config1_literal_minimum_capacity", 1, False, 0.0),
+                                   ("config5_router_only", 5, False, args.cf),
+                                   ("config5_literal_minimum_capacity", 5, False, 0.0),
                                    ("config2_literal_minimum_capacity", 2, False, 0.0), ("config3", 3, False, args.cf),
+                                   ("config3_literal_minimum_capacity", 3, False, 0.0),
+                                   ("config4_literal_minimum_capacity", 4, False, 0.0),
                                    ("config4", 4, False, args.cf), ("config5_with_ffn", 5, True, args.cf)):
             gc.collect()
             torch.cuda.empty_cache()
