@@ -378,7 +378,11 @@ int launch_dispatch(const locmoe_shape_t& s, int64_t rows, const void* x, const 
         const int rc = launch_dispatch_tma(s, rows, rb, x, inv, buf, zero_pad, st);
         if (rc != 1) return rc;   // 1: the row size does not suit the bulk-copy kernel, fall through
     }
-    if (vec_ok && slot && !mode && (unsigned long long)s.T * (rb / 16) < 0xf0000000ull) {
+    // the token-major kernel walks all T tokens: only where the buffer can hold at least half of them (with one
+    // slot per (source, expert) pair, 4096 rows for 65536 tokens, its 20480 nearly empty CTAs took 80 us; the
+    // row-major kernel below walks the rows instead)
+    const bool dense = (unsigned long long)rows * 2 >= (unsigned long long)s.T;
+    if (vec_ok && slot && dense && !mode && (unsigned long long)s.T * (rb / 16) < 0xf0000000ull) {
         const unsigned total = (unsigned)((unsigned long long)s.T * (rb / 16));
         const unsigned per = (unsigned)(kThreads * 4 * kTokIters);
         const int g = (int)((total + per - 1) / per);
