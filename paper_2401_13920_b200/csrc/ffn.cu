@@ -387,12 +387,16 @@ ffn_gemm_wide_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 const int nt = rem / a.m_tiles, mt = rem - nt * a.m_tiles;
                 const int row0 = e * a.M + mt * 2 * BM, n0 = nt * BN;
                 bool ok = true;
+                // every other wave sweeps the reduction backwards: an expert whose tiles straddle two waves then
+                // finds the end of its operand panels, which the earlier wave read last, still in L2
+                const bool rev = ((w / (int)gridDim.x) & 1) != 0;
                 for (int kb = 0; kb < kblocks && ok; ++kb) {
                     if (!wait_or_abort(&empty[stage], phase ^ 1u, abort_word)) { ok = false; break; }
                     unsigned char* sa = base + (size_t)stage * STAGE_W_BYTES;
+                    const int k0 = (rev ? kblocks - 1 - kb : kb) * BK;
                     mbar_expect_tx(&full[stage], STAGE_W_BYTES);
-                    tma_load_2d(sa, &tmA, kb * BK, row0, &full[stage]);
-                    tma_load_3d(sa + AW_BYTES, &tmB, kb * BK, n0, e, &full[stage]);
+                    tma_load_2d(sa, &tmA, k0, row0, &full[stage]);
+                    tma_load_3d(sa + AW_BYTES, &tmB, k0, n0, e, &full[stage]);
                     if (++stage == NSTAGE_W) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
