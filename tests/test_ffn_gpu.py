@@ -81,6 +81,40 @@ def test_expert_ffn_small_shapes_all_rows(P, monkeypatch, kernel, E, N, Dn, C, H
     _check_rows(P, buf, w_in, w_out, y, E, M, range(rows), ydt == torch.bfloat16)
 
 
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(n):
+        Dn = int(rng.choice([1, 2, 4]))
+        E = Dn * int(rng.choice([1, 2, 3]))       # the experts divide evenly over the devices
+        C = int(rng.integers(1, 160))            # M = Dn * C rows per expert: from 1 to several tiles, any remainder
+        H = 8 * int(rng.integers(1, 60))          # rows of 16 bytes and more, reductions that end inside a k-block
+        F = 8 * int(rng.integers(1, 90))
+        out.append((E, Dn, C, H, F))
+    return out
+
+
+@pytest.mark.parametrize("E,Dn,C,H,F", _random_shapes(8, 20240113))
+@pytest.mark.parametrize("kernel", ["one_sm", "wide"])
+def test_expert_ffn_random_ragged_shapes(P, monkeypatch, kernel, E, Dn, C, H, F):
+    # seeded random shapes, every row checked: tiles cut by the rows of an expert, by N and by K in either kernel
+    monkeypatch.setenv("LOCMOE_FFN", {"one_sm": "1", "wide": "w"}[kernel])
+    B = P.B
+    dev = torch.device("cuda:0")
+    rows, M = Dn * E * C, Dn * C
+    g = torch.Generator(device=dev).manual_seed(E * 1000 + C)
+    buf = torch.randn(rows, H, generator=g, device=dev).to(torch.bfloat16)
+    w_in = (torch.randn(E, F, H, generator=g, device=dev) * 0.1).to(torch.bfloat16)
+    w_out = (torch.randn(E, H, F, generator=g, device=dev) * 0.1).to(torch.bfloat16)
+    sh = B.make_shape(rows, H, E, 1, Dn, torch.bfloat16, B.LAYOUT_RECV)
+    h1 = torch.full((rows, F), 3.0, dtype=torch.bfloat16, device=dev)
+    y = torch.full((rows, H), 7.0, dtype=torch.bfloat16, device=dev)
+    B.locmoe_expert_ffn(sh, C, F, buf, w_in, w_out, h1, y)
+    torch.cuda.synchronize()
+    assert B.locmoe_device_flags() == 0
+    _check_rows(P, buf, w_in, w_out, y, E, M, range(rows))
+
+
 def test_expert_ffn_rejects_send_layout_and_bad_sizes(P):
     B = P.B
     import ctypes as C
