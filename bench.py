@@ -465,7 +465,7 @@ def measure(args, w, env, *, steps, warmup, stage_steps, use_ffn, variant, fuse_
         flops = 4.0 * rows * w.H * F
         tf = flops / (stage_ms["ffn"] * 1e-3) / 1e12
         tpeak, tkind = measured_tensor_peak()
-        roofline.update({"bound": "tensor", "kernel": "ffn_gemm_kernel / ffn_gemm_wide_kernel (two launches; the library picks per GEMM)", "achieved": tf, "peak": tpeak,
+        roofline.update({"bound": "tensor", "kernel": " + ".join(B.FFN_KERNEL_NAMES[k] for k in B.locmoe_ffn_kernels(st.shape, st.C_alloc, F)) + " (the library's choice per GEMM)", "achieved": tf, "peak": tpeak,
                          "peak_kind": tkind, "unit": "TFLOP/s", "frac": tf / tpeak, "traffic": None, "traffic_source": None,
                          "flops": flops, "frac_of_burst_peak": tf / measured_tensor_burst(), "hbm_kernels": kernels})
         roofline.pop("frac_nominal", None)

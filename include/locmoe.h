@@ -471,6 +471,15 @@ int locmoe_expert_ffn(const locmoe_shape_t *shape, int32_t C_alloc, int32_t F, c
                       const void *w_in, const void *w_out, void *h1, void *y, int32_t y_dtype,
                       void *stream);
 
+/*
+ * Host only, launches nothing: which kernel locmoe_expert_ffn would run each of
+ * its two GEMMs with on the current device for this shape -- kernels[0] for
+ * x W_in^T (+ GeLU), kernels[1] for g W_out^T.  The results do not depend on the
+ * choice; a program may want to report it.
+ */
+enum { LOCMOE_FFN_TILE_128x256 = 0, LOCMOE_FFN_TILE_256x256 = 1, LOCMOE_FFN_TWO_SM = 2, LOCMOE_FFN_TWO_SM_SINGLE = 3 };
+int locmoe_ffn_kernels(const locmoe_shape_t *shape, int32_t C_alloc, int32_t F, int32_t *kernels /* [2], host */);
+
 /* Every device array of one MoE layer pass, for locmoe_moe_layer (host struct of device pointers;
  * sizes as documented at the individual calls). */
 typedef struct {

@@ -25,7 +25,7 @@ FLAG_DELTA_OVERRIDE, FLAG_MIN_SATURATED, FLAG_MIN_BINDS = 1, 2, 4
 EXPORTS = [
     "locmoe_workspace_bytes", "locmoe_gate", "locmoe_gate_ex", "locmoe_aux_loss_partial", "locmoe_capacity", "locmoe_capacity_noalloc", "locmoe_capacity_read", "locmoe_route", "locmoe_capacity_route", "locmoe_gate_route",
     "locmoe_conventional_capacity", "locmoe_batch_delta", "locmoe_dest_order",
-    "locmoe_dispatch", "locmoe_combine", "locmoe_dispatch_peer", "locmoe_dispatch_peer_window", "locmoe_combine_peer", "locmoe_topk_select", "locmoe_topk_fold", "locmoe_combine_topk", "locmoe_expert_ffn", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
+    "locmoe_dispatch", "locmoe_combine", "locmoe_dispatch_peer", "locmoe_dispatch_peer_window", "locmoe_combine_peer", "locmoe_topk_select", "locmoe_topk_fold", "locmoe_combine_topk", "locmoe_expert_ffn", "locmoe_ffn_kernels", "locmoe_moe_layer", "locmoe_aux_loss", "locmoe_loc_loss", "locmoe_cos_hist", "locmoe_launch_counts", "locmoe_device_flags", "locmoe_status_string",
 ]
 
 
@@ -92,6 +92,7 @@ def _load() -> C.CDLL:
     lib.locmoe_dispatch.argtypes = [C.POINTER(Shape), i32, vp, vp, vp, vp, i32, vp]
     lib.locmoe_combine.argtypes = [C.POINTER(Shape), i32, vp, i32, vp, vp, vp, i32, vp]
     lib.locmoe_expert_ffn.argtypes = [C.POINTER(Shape), i32, i32, vp, vp, vp, vp, vp, i32, vp]
+    lib.locmoe_ffn_kernels.argtypes = [C.POINTER(Shape), i32, i32, C.POINTER(i32 * 2)]
     lib.locmoe_moe_layer.argtypes = [C.POINTER(Shape), vp, vp, vp, C.POINTER(CapacityRule), i32, i32, vp, vp,
                                      C.POINTER(LayerBuffers), vp, vp]
     lib.locmoe_aux_loss.argtypes = [C.POINTER(Shape), vp, vp, C.c_float, vp, vp, vp, vp, C.c_size_t, vp]
@@ -338,6 +339,17 @@ def locmoe_combine(shape: Shape, C_alloc, y, slot, gate_w, out, accumulate=False
     return _check("locmoe_combine", _lib.locmoe_combine(C.byref(shape), int(C_alloc), _ptr(y), dtype_code(y.dtype),
                                                         _ptr(slot), _ptr(gate_w), _ptr(out), 1 if accumulate else 0,
                                                         _stream(stream)))
+
+
+FFN_KERNEL_NAMES = ("ffn_gemm_kernel (128 x 256 tiles)", "ffn_gemm_wide_kernel (256 x 256 tiles)",
+                    "ffn_gemm2_kernel (two SMs per tile)", "ffn_gemm2_kernel (two SMs per tile, one accumulator)")
+
+
+def locmoe_ffn_kernels(shape: Shape, C_alloc, F):
+    """Which kernel the library runs each of the two GEMMs of locmoe_expert_ffn with (host only): two codes."""
+    out = (C.c_int32 * 2)()
+    _check("locmoe_ffn_kernels", _lib.locmoe_ffn_kernels(C.byref(shape), int(C_alloc), int(F), C.byref(out)))
+    return int(out[0]), int(out[1])
 
 
 def locmoe_expert_ffn(shape: Shape, C_alloc, F, buf, w_in, w_out, h1, y, stream=None) -> int:

@@ -364,6 +364,20 @@ int locmoe_expert_ffn(const locmoe_shape_t* shape, int32_t C_alloc, int32_t F, c
     return launch_expert_ffn(*shape, rows, F, buf, w_in, w_out, h1, y, y_dtype, static_cast<cudaStream_t>(stream));
 }
 
+int locmoe_ffn_kernels(const locmoe_shape_t* shape, int32_t C_alloc, int32_t F, int32_t* kernels) {
+    int rc = check_shape(shape);
+    if (rc) return rc;
+    if (!kernels) return LOCMOE_ERR_NULL;
+    if (F < 8 || F % 8 != 0 || shape->H % 8 != 0) return LOCMOE_ERR_SHAPE;
+    const long long rows = buffer_rows(shape, C_alloc);
+    if (rows < 0) return LOCMOE_ERR_SHAPE;
+    int k[2];
+    plan_expert_ffn(*shape, rows, F, k);
+    kernels[0] = k[0];
+    kernels[1] = k[1];
+    return LOCMOE_OK;
+}
+
 int locmoe_moe_layer(const locmoe_shape_t* shape, const void* x, const int32_t* src_dev, const float* eps,
                      const locmoe_capacity_rule_t* rule, int32_t C_alloc, int32_t F, const void* w_in,
                      const void* w_out, const locmoe_layer_buffers_t* b, void* out, void* stream) {

@@ -122,6 +122,7 @@ int launch_combine_topk(const locmoe_shape_t& s, int64_t rows, const void* y, in
 int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* buf, const void* w_in,
                       const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st);
 int read_ffn_flags(int* out, cudaStream_t st);
+void plan_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, int kernels[2]);
 
 // Copies the device diagnostics word to host memory (synchronises the stream).
 int read_device_flags(int* out, cudaStream_t st);

@@ -828,27 +828,24 @@ int launch_gemm2(const void* A, const void* W, void* out, int out_f32, int gelu,
 
 }  // namespace
 
-int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* buf, const void* w_in,
-                      const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st) {
+// Which kernel runs each of the two GEMMs: 0 = 128 x 256 tiles, 1 = wide (256 x 256 tiles), 2 = two-SM, 3 = two-SM with
+// one accumulator.  By default the wide kernel where the reduction is long enough for its exposed epilogue not to
+// matter, the rows of an expert fill its taller tiles as well as they fill the 128-row ones, and the last wave of its
+// twice-as-long tiles does not cost more than the wide tiles save (about 5 %); else the 128 x 256 kernel.
+// On E = 32, M = 2048, H = 2560, F = 10240, back to back under the power cap: second GEMM (K = 10240) 2.63
+// against 2.77 ms, first GEMM (K = 2560, GeLU) 2.98 against 2.84 ms.
+// LOCMOE_FFN (a testing aid) overrides: 1 = 128 x 256 kernel for both, w = wide for both, w1 / w2 = wide for
+// the first / second GEMM only, 2 = the two-SM kernel (2s: its single-accumulator form).  The two-SM kernel is
+// opt-in only: it passes every test and runs clean in the bench, but launches of it failed under multi-metric
+// profiler captures for a reason that reading the code has not shown.
+void plan_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, int kernels[2]) {
     const int E = s.E;
     const int M = (int)(rows / E);
-    // Which kernel runs a GEMM.  By default the wide kernel (256 x 256 tiles, a third less operand traffic, the
-    // epilogue mostly exposed) where the reduction is long enough for the exposed epilogue not to matter and the
-    // rows of an expert fill its taller tiles as well as they fill the 128-row ones, else the 128 x 256 kernel.
-    // On E = 32, M = 2048, H = 2560, F = 10240, back to back under the power cap: second GEMM (K = 10240) 2.63
-    // against 2.77 ms, first GEMM (K = 2560, GeLU) 2.98 against 2.84 ms.
-    // LOCMOE_FFN (a testing aid) overrides: 1 = 128 x 256 kernel for both, w = wide for both, w1 / w2 = wide for
-    // the first / second GEMM only, 2 = the two-SM kernel (2s: its single-accumulator form).  The two-SM kernel is
-    // opt-in only: it passes every test and runs clean in the bench, but launches of it failed under multi-metric
-    // profiler captures for a reason that reading the code has not shown.
     const char* mode = getenv("LOCMOE_FFN");
     if (mode && mode[0] == '2' && sm_count() >= 2) {
-        const int nacc = mode[1] == 's' ? 1 : 2;
-        int rc = launch_gemm2(buf, w_in, h1, 0, 1, E, M, F, s.H, nacc, st);
-        if (rc) return rc;
-        return launch_gemm2(h1, w_out, y, y_dtype == LOCMOE_F32 ? 1 : 0, 0, E, M, s.H, F, nacc, st);
+        kernels[0] = kernels[1] = mode[1] == 's' ? 3 : 2;
+        return;
     }
-    // ... and the last wave of its twice-as-long tiles does not cost more than the wide tiles save (about 5 %)
     const long long m1 = (M + BM - 1) / BM, m2 = (M + 2 * BM - 1) / (2 * BM), G = sm_count() > 0 ? sm_count() : 1;
     auto pays = [&](int N, int K) {
         const long long n = (N + BN - 1) / BN;
@@ -860,10 +857,25 @@ int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* 
     bool wide1 = pays(F, s.H), wide2 = pays(s.H, F);
     if (mode && mode[0] == '1') wide1 = wide2 = false;
     if (mode && mode[0] == 'w') { wide1 = mode[1] != '2'; wide2 = mode[1] != '1'; }
+    kernels[0] = wide1 ? 1 : 0;
+    kernels[1] = wide2 ? 1 : 0;
+}
+
+int launch_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, const void* buf, const void* w_in,
+                      const void* w_out, void* h1, void* y, int y_dtype, cudaStream_t st) {
+    const int E = s.E;
+    const int M = (int)(rows / E);
     const int y_f32 = y_dtype == LOCMOE_F32 ? 1 : 0;
-    int rc = wide1 ? launch_gemm_wide(buf, w_in, h1, 0, 1, E, M, F, s.H, st) : launch_gemm(buf, w_in, h1, 0, 1, E, M, F, s.H, st);
+    int kernels[2];
+    plan_expert_ffn(s, rows, F, kernels);
+    auto run = [&](int kernel, const void* A, const void* W, void* out, int out_f32, int gelu, int N, int K) {
+        if (kernel >= 2) return launch_gemm2(A, W, out, out_f32, gelu, E, M, N, K, kernel == 3 ? 1 : 2, st);
+        if (kernel == 1) return launch_gemm_wide(A, W, out, out_f32, gelu, E, M, N, K, st);
+        return launch_gemm(A, W, out, out_f32, gelu, E, M, N, K, st);
+    };
+    const int rc = run(kernels[0], buf, w_in, h1, 0, 1, F, s.H);
     if (rc) return rc;
-    return wide2 ? launch_gemm_wide(h1, w_out, y, y_f32, 0, E, M, s.H, F, st) : launch_gemm(h1, w_out, y, y_f32, 0, E, M, s.H, F, st);
+    return run(kernels[1], h1, w_out, y, y_f32, 0, s.H, F);
 }
 
 int read_ffn_flags(int* out, cudaStream_t st) {

@@ -184,3 +184,28 @@ def test_host_helpers_of_the_rule_and_the_layout(B, oracle_mod):
     # device 1 of a 2 x 2 map lists itself, its node neighbour 0, then the other node's 3 and 2
     assert [B.dest_order(2, 2, 1, b) for b in (1, 0, 3, 2)] == [0, 1, 2, 3]
     assert B._lib.locmoe_dest_order(C.byref(B.make_shape(1, 1, 1, 2, 2, B.F32)), 0, 4) == -2
+
+
+def test_ffn_kernel_choice_is_a_host_side_query(B, monkeypatch):
+    # no launch, no device needed (the SM count falls back to a B200's 148): config 5's full size takes the wide kernel for
+    # the long reduction only; small batches and forced choices behave as documented
+    monkeypatch.delenv("LOCMOE_FFN", raising=False)
+    sh = B.make_shape(65536, 2560, 32, 4, 8, B.BF16, B.LAYOUT_RECV)
+    assert B.locmoe_ffn_kernels(sh, 64, 10240) == (0, 1)         # 2048 rows per expert
+    assert B.locmoe_ffn_kernels(sh, 8, 10240) == (0, 1)          # 256 rows per expert: 320 wide tiles, the last 24 as halves
+    assert B.locmoe_ffn_kernels(sh, 4, 10240) == (0, 0)          # 128 rows per expert: half of every 256-row tile would be empty
+    assert B.locmoe_ffn_kernels(sh, 32, 10240) == (0, 1)         # 1024 rows per expert
+    assert B.locmoe_ffn_kernels(sh, 64, 4096) == (0, 0)          # no reduction of 6144 or more
+    sh3 = B.make_shape(65536, 2560, 32, 4, 8, B.BF16, B.LAYOUT_RECV)
+    assert B.locmoe_ffn_kernels(sh3, 3, 10240) == (0, 0)         # 96 rows per expert: a 256-row tile would be mostly empty
+    monkeypatch.setenv("LOCMOE_FFN", "w")
+    assert B.locmoe_ffn_kernels(sh, 8, 10240) == (1, 1)
+    monkeypatch.setenv("LOCMOE_FFN", "w1")
+    assert B.locmoe_ffn_kernels(sh, 8, 10240) == (1, 0)
+    monkeypatch.setenv("LOCMOE_FFN", "1")
+    assert B.locmoe_ffn_kernels(sh, 64, 10240) == (0, 0)
+    monkeypatch.setenv("LOCMOE_FFN", "2s")
+    assert B.locmoe_ffn_kernels(sh, 64, 10240) == (3, 3)
+    import ctypes as C
+    assert B._lib.locmoe_ffn_kernels(C.byref(sh), 64, 10244, C.byref((C.c_int32 * 2)())) == -2
+    assert B._lib.locmoe_ffn_kernels(C.byref(sh), 64, 10240, None) == -1
