@@ -331,7 +331,10 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 // for half a tile's worth at either end (each half has its own pair of barriers and the epilogue drains the upper
 // half first); that is the better trade where K is long.  Three stages of 64 KB.
 constexpr int NSTAGE_W = 3;
-constexpr int kWideMinK = 6144;   // shortest reduction for which the wide kernel is chosen by default
+// shortest reduction for which the wide kernel is chosen by default, with and without a GeLU in the epilogue (pairs of
+// GEMMs on E = 32, M = 2048 back to back: with the GeLU level at K = 6144, 2 % slower at 5120; without it 1.6 % faster
+// at 5120, level at 4096)
+constexpr int kWideMinK = 6144, kWideMinKPlain = 5120;
 constexpr uint32_t AW_BYTES = 2 * A_BYTES, STAGE_W_BYTES = AW_BYTES + B_BYTES;
 constexpr size_t kFfnWideSmem = (size_t)NSTAGE_W * STAGE_W_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 
@@ -847,14 +850,14 @@ void plan_expert_ffn(const locmoe_shape_t& s, int64_t rows, int F, int kernels[2
         return;
     }
     const long long m1 = (M + BM - 1) / BM, m2 = (M + 2 * BM - 1) / (2 * BM), G = sm_count() > 0 ? sm_count() : 1;
-    auto pays = [&](int N, int K) {
+    auto pays = [&](int N, int K, bool gelu) {
         const long long n = (N + BN - 1) / BN;
         const long long tw = E * m2 * n, tail = tw % G;
         const long long waves_narrow = (E * m1 * n + G - 1) / G;                      // in 128-row tiles
         const long long waves_wide = tw / G * 2 + (tail == 0 ? 0 : (tw >= G && 2 * tail <= G) ? 1 : 2);   // the same unit
-        return K >= kWideMinK && m2 * 2 == m1 && waves_wide * 19 <= waves_narrow * 20;
+        return K >= (gelu ? kWideMinK : kWideMinKPlain) && m2 * 2 == m1 && waves_wide * 19 <= waves_narrow * 20;
     };
-    bool wide1 = pays(F, s.H), wide2 = pays(s.H, F);
+    bool wide1 = pays(F, s.H, true), wide2 = pays(s.H, F, false);
     if (mode && mode[0] == '1') wide1 = wide2 = false;
     if (mode && mode[0] == 'w') { wide1 = mode[1] != '2'; wide2 = mode[1] != '1'; }
     kernels[0] = wide1 ? 1 : 0;

@@ -195,7 +195,8 @@ def test_ffn_kernel_choice_is_a_host_side_query(B, monkeypatch):
     assert B.locmoe_ffn_kernels(sh, 8, 10240) == (0, 1)          # 256 rows per expert: 320 wide tiles, the last 24 as halves
     assert B.locmoe_ffn_kernels(sh, 4, 10240) == (0, 0)          # 128 rows per expert: half of every 256-row tile would be empty
     assert B.locmoe_ffn_kernels(sh, 32, 10240) == (0, 1)         # 1024 rows per expert
-    assert B.locmoe_ffn_kernels(sh, 64, 4096) == (0, 0)          # no reduction of 6144 or more
+    assert B.locmoe_ffn_kernels(sh, 64, 4096) == (0, 0)          # no reduction long enough
+    assert B.locmoe_ffn_kernels(sh, 64, 5120) == (0, 1)          # 5120 is, without a GeLU in the epilogue
     sh3 = B.make_shape(65536, 2560, 32, 4, 8, B.BF16, B.LAYOUT_RECV)
     assert B.locmoe_ffn_kernels(sh3, 3, 10240) == (0, 0)         # 96 rows per expert: a 256-row tile would be mostly empty
     monkeypatch.setenv("LOCMOE_FFN", "w")
