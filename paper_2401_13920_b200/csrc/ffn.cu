@@ -11,8 +11,10 @@
 //   - eight epilogue warps read the accumulator with tcgen05.ld (one row per thread, half of the columns per
 //     warp), apply GeLU (first GEMM), convert and store.
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = epilogue.  Persistent CTAs, one per SM.
-// Two kernels share these pieces: ffn_gemm_kernel (one CTA per 128 x 256 tile, the default) and
-// ffn_gemm2_kernel (a cluster of two CTAs per 256 x 256 tile, tcgen05 cta_group::2; described at the kernel).
+// Three kernels share these pieces: ffn_gemm_kernel (one CTA per 128 x 256 tile, as described above),
+// ffn_gemm_wide_kernel (one CTA per 256 x 256 tile, both accumulators on it; chosen for long reductions) and
+// ffn_gemm2_kernel (a cluster of two CTAs per 256 x 256 tile, tcgen05 cta_group::2; opt-in); the latter two are
+// described where they are defined, the choice between them at plan_expert_ffn.
 // Every barrier wait is bounded; on a timeout the kernel raises the device diagnostics flag, leaves its
 // loops, frees its TMEM and returns.
 #include <cuda.h>
