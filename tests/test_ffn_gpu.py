@@ -56,6 +56,7 @@ def _check_rows(P, buf, w_in, w_out, y, E, M, rows, y_is_bf16=True):
     (8, 1, 8, 40, 512, 1024, torch.bfloat16),    # M = 320, several k-blocks and n-tiles
     (2, 1, 2, 300, 320, 512, torch.bfloat16),    # M = 600: three 256-row tiles, the last one with an empty lower half
     (4, 1, 2, 256, 64, 5120, torch.bfloat16),    # first GEMM: 160 tiles of 256 x 256 -- on 148 SMs the wide kernel splits the last 12 into halves
+    (4, 1, 2, 300, 64, 3328, torch.bfloat16),    # M = 600 and 156 wide tiles: split halves that lie wholly beyond an expert's rows
 ])
 @pytest.mark.parametrize("kernel", ["one_sm", "wide", pytest.param("two_sm_single_acc", marks=two_sm), pytest.param("two_sm", marks=two_sm)])
 def test_expert_ffn_small_shapes_all_rows(P, monkeypatch, kernel, E, N, Dn, C, H, F, ydt):
